@@ -1,0 +1,166 @@
+/*
+ * libgrawa -- the distributed averaging update of GRAWA, MGRAWA and LGRAWA
+ * (Dimlioglu & Choromanska, "GRAWA: Gradient-based Weighted Averaging for Distributed
+ * Training of Deep Learning Models") for M worker replicas resident on one NVIDIA B200.
+ *
+ * The update, for workers m = 1..M with flat fp32 parameters x_m and accumulated gradients
+ * g_m of n elements cut into K layers, layer k = [layer_offsets[k], layer_offsets[k+1]):
+ *
+ *   1. S[k][m]  = sum_{j in layer k} g_m[j]^2                      (||G_k||_F^2, Eq. 3 / Eq. 5)
+ *   2. score    LGRAWA  A^k_m = sqrt(S[k][m])                      (Eq. 5-6)
+ *               MGRAWA  A_m   = sum_k sqrt(S[k][m])                (Eq. 3)
+ *               GRAWA   A_m   = sqrt(sum_k S[k][m])                (Eq. 2, flattened gradient)
+ *   3. weights  beta_m = (1/A_m) / sum_i (1/A_i), sum_m beta_m = 1 (Eq. 2, Eq. 4); LGRAWA does
+ *               this separately in every layer (Eq. 7)
+ *   4. centre   x_C[j] = sum_m beta_{m,layer(j)} x_m[j]            (display under Eq. 2; Eq. 7)
+ *   5. pull     x_m[j] <- (1-pull) x_m[j] + pull x_C[j]            (same display; last line of
+ *               Algorithms 1 and 2), x_C taken from the values before the pull.
+ *
+ * Conventions common to every entry point
+ *   - `params`, `grads`: HOST arrays of M DEVICE pointers, each to n contiguous fp32 values.
+ *   - `layer_offsets`: HOST array of n_layers+1 int64, offsets[0] = 0, non-decreasing,
+ *     offsets[n_layers] = n.  Empty layers are allowed.
+ *   - `center_out`: DEVICE pointer to n fp32 values, fully overwritten; may be NULL.
+ *   - The caller owns every buffer.  params[m] are updated in place, grads[m] are only read.
+ *     No two of {params[*], center_out} may overlap and grads may not overlap params or
+ *     center_out; overlap visible from the pointer ranges is rejected.
+ *   - Work is enqueued on `stream` (a cudaStream_t; NULL is the default stream) and the call
+ *     returns without synchronising.  The first call with a new (device, stream, n, M, layer
+ *     table) builds and caches a plan (device allocations and a small upload); later calls
+ *     allocate nothing.
+ *   - Arithmetic: fp32 loads; sums of squares accumulated in short fp32 runs combined in fp64
+ *     in a fixed order (bitwise reproducible run to run); scores and weights in fp64, rounded
+ *     once to fp32; centre as an fp32 fused-multiply-add chain over m = 0..M-1; pull as
+ *     fmaf(pull, x_C, (1-pull) * x_m).
+ *   - Scores that are exactly zero take the limit of 1/A: inside a normalisation group the Z
+ *     workers with zero score get 1/Z each, all others 0.  A non-finite score (NaN/Inf
+ *     gradients) gives that worker weight 0, the rest are normalised among themselves (uniform
+ *     1/M if none is finite), and the step's status word is set; see grawa_last_step_status.
+ *   - Errors detectable on the host return a negative code before anything is enqueued.
+ *     Nothing on the device traps or waits.
+ *   - There is no CPU implementation behind this interface.
+ */
+#ifndef GRAWA_H
+#define GRAWA_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define GRAWA_MAX_WORKERS 64
+
+typedef struct CUstream_st *grawa_stream_t; /* identical to cudaStream_t */
+
+typedef enum grawa_status {
+    GRAWA_OK = 0,
+    GRAWA_ERR_INVALID_ARG = -1, /* NULL pointer, bad M/n/offsets/pull, overlapping buffers        */
+    GRAWA_ERR_CUDA = -2,        /* a CUDA runtime call failed; text in grawa_last_cuda_error()    */
+    GRAWA_ERR_NONFINITE = -3,   /* a gradient score was NaN/Inf (fallback weights were applied)   */
+    GRAWA_ERR_WORKSPACE = -4,   /* caller-supplied workspace missing, misaligned or too small     */
+    GRAWA_ERR_TIMEOUT = -5      /* a bounded device-side wait ran out (bulk-copy variant only)    */
+} grawa_status;
+
+typedef enum grawa_variant { GRAWA_VARIANT_GRAWA = 0, GRAWA_VARIANT_MGRAWA = 1, GRAWA_VARIANT_LGRAWA = 2 } grawa_variant;
+
+/* Optional arguments; a NULL `options` pointer means all defaults.  Zero-initialise before use. */
+typedef struct grawa_options {
+    float  *weights_out;   /* DEVICE, fp32: beta, [M] for GRAWA/MGRAWA, [n_layers][M] for LGRAWA    */
+    double *scores_out;    /* DEVICE, fp64: A, same shape as weights_out                            */
+    double *sumsq_out;     /* DEVICE, fp64: S, [n_layers][M] (one row when there is no layer table) */
+    void   *workspace;     /* DEVICE scratch, 256-byte aligned; NULL = the cached plan owns one     */
+    size_t  workspace_bytes; /* size of `workspace`; at least grawa_workspace_bytes(...)            */
+} grawa_options;
+
+/* Library version, major*10000 + minor*100 + patch. */
+int grawa_version(void);
+
+/* Static text for a status code. */
+const char *grawa_status_string(grawa_status status);
+
+/* Text of the last CUDA error seen by the calling thread ("" if none). */
+const char *grawa_last_cuda_error(void);
+
+/* Bytes of device scratch a step needs for this problem (partial sums, S, A, beta, status).
+ * layer_offsets may be NULL with n_layers = 0 (one layer).  Returns 0 on invalid arguments. */
+size_t grawa_workspace_bytes(int64_t n, int M, const int64_t *layer_offsets, int n_layers);
+
+/* MGRAWA step (Eq. 3-4, then centre and pull): one weight per worker from the sum of its
+ * per-layer gradient norms.  With layer_offsets = NULL / n_layers = 0 the whole vector is one
+ * layer and the score is the flat norm, i.e. vanilla GRAWA (Eq. 2).
+ * pull must lie in [0, 1].  M in [1, GRAWA_MAX_WORKERS].  n = 0 is a no-op returning GRAWA_OK.
+ * M = 1: the single worker is left untouched and copied to center_out. */
+grawa_status grawa_mgrawa_step(float *const *params, const float *const *grads, int64_t n, int M,
+                               float pull, const int64_t *layer_offsets, int n_layers,
+                               float *center_out, const grawa_options *options, grawa_stream_t stream);
+
+/* Vanilla GRAWA step (Eq. 2): one weight per worker from the norm of the flattened gradient.
+ * A layer table, if given, only shapes sumsq_out; the weights do not depend on it. */
+grawa_status grawa_grawa_step(float *const *params, const float *const *grads, int64_t n, int M,
+                              float pull, const int64_t *layer_offsets, int n_layers,
+                              float *center_out, const grawa_options *options, grawa_stream_t stream);
+
+/* LGRAWA step (Eq. 5-7, construct, pull): in every layer k separate weights beta^k_m from the
+ * layer's gradient norms; the centre is the concatenation of the per-layer weighted averages.
+ * Empty layers form no group. */
+grawa_status grawa_lgrawa_step(float *const *params, const float *const *grads, int64_t n, int M,
+                               float pull, const int64_t *layer_offsets, int n_layers,
+                               float *center_out, const grawa_options *options, grawa_stream_t stream);
+
+/* Same update with HOST buffers: params[m], grads[m] and center_out are HOST pointers (pinned
+ * memory gives asynchronous copies; pageable memory works and is slower).  The call uploads the
+ * M gradient and parameter vectors to device staging buffers owned by the cached plan, runs the
+ * step of `variant`, downloads the updated parameters and the centre, and synchronises `stream`
+ * before returning, so the results are in the host buffers on return.  The staging buffers take
+ * (2M+1)*n*4 bytes of device memory and are allocated on the first call for a problem shape. */
+grawa_status grawa_step_host(grawa_variant variant, float *const *params, const float *const *grads,
+                             int64_t n, int M, float pull, const int64_t *layer_offsets, int n_layers,
+                             float *center_out, grawa_stream_t stream);
+
+/* Synchronises `stream` and reports the status word of the last step enqueued on it by the
+ * calling process: GRAWA_OK, GRAWA_ERR_NONFINITE or GRAWA_ERR_TIMEOUT (GRAWA_ERR_CUDA if the
+ * synchronisation itself fails, GRAWA_ERR_INVALID_ARG if no step was enqueued on it). */
+grawa_status grawa_last_step_status(grawa_stream_t stream);
+
+/* Proximity-search step of the local phase (the line marked "Prox." in Algorithms 1 and 2):
+ * x_m[j] <- (1 - mu_over_tau) x_m[j] + mu_over_tau * center[j] for all M workers in one pass,
+ * with `center` (DEVICE, n fp32, read only) the centre stored by the last averaging step.
+ * mu_over_tau must lie in [0, 1]. */
+grawa_status grawa_prox_step(float *const *params, const float *center, int64_t n, int M,
+                             float mu_over_tau, grawa_stream_t stream);
+
+/* Tuning knobs, process wide; they change speed, never results beyond fp32 summation order
+ * of the sums of squares ("sumsq_tile").  Returns GRAWA_ERR_INVALID_ARG for an unknown name
+ * or a value out of range.
+ *   "sumsq_tile"   elements per sum-of-squares work item (multiple of 1024, 1024..1048576)
+ *   "pull_tile"    elements per centre+pull work item (multiple of 1024, 1024..1048576)
+ *   "pull_variant" 0 = automatic, 1 = register kernel (vector loads), 2 = bulk-copy kernel
+ *                  (shared-memory staging by 1-D bulk asynchronous copies)
+ *   "kernel_timing" 1 = every device-buffer step also records CUDA events around its three
+ *                  phases on the step's stream (see grawa_collect_kernel_times); do not use
+ *                  while capturing a CUDA graph.  Default 0.
+ * Changing a tile size drops the cached plans. */
+grawa_status grawa_set_option(const char *name, int64_t value);
+
+/* Current value of a tuning knob, or -1 for an unknown name. */
+int64_t grawa_get_option(const char *name);
+
+/* Number of kernels this library has launched in the calling process since it was loaded. */
+int64_t grawa_launch_count(void);
+
+/* Sums, in milliseconds, of the device time of the three phases (sum-of-squares kernel; partial
+ * reduction + scores + weights kernel; centre+pull kernel) over the steps enqueued while
+ * "kernel_timing" was 1 since the previous call, and the number of those steps.  Any output
+ * pointer may be NULL.  Synchronises the device. */
+grawa_status grawa_collect_kernel_times(double *sumsq_ms, double *finalize_ms, double *center_pull_ms,
+                                        int64_t *steps);
+
+/* Frees every cached plan (device allocations included) on every device.  Synchronises. */
+void grawa_clear_plans(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GRAWA_H */

@@ -108,9 +108,11 @@ def weights(A):
     return beta, bool(flagged)
 
 
-def center_pull(params, beta, pull, layer_offsets=None, j0=0, j1=None, want_workers=True):
+def center_pull(params, beta, pull, layer_offsets=None, j0=0, j1=None, want_workers=True, out=None):
     """Steps 4-5 on [j0, j1): x_C = sum_m beta_m x_m, then x_m <- (1-pull) x_m + pull x_C.
-    ``beta`` is [K, M] (per layer, Eq. 7) or [M].  Returns (center, workers) in float64."""
+    ``beta`` is [K, M] (per layer, Eq. 7) or [M].  Returns (center, workers) in float64.
+    ``out``: optional (center_buffer, [worker_buffers]) of float64 arrays with at least j1-j0
+    elements that are reused instead of allocating fresh outputs (views of them are returned)."""
     x = _f32_list(params)
     n, M = x[0].size, len(x)
     j1 = n if j1 is None else j1
@@ -122,8 +124,13 @@ def center_pull(params, beta, pull, layer_offsets=None, j0=0, j1=None, want_work
         assert beta.shape == (K, M)
     else:
         assert beta.shape == (M,)
-    center = np.zeros(j1 - j0, dtype=np.float64)
-    outs = [np.zeros(j1 - j0, dtype=np.float64) for _ in range(M)] if want_workers else None
+    if out is not None:
+        center = out[0][:j1 - j0]
+        outs = [b[:j1 - j0] for b in out[1]] if want_workers else None
+        assert center.dtype == np.float64 and center.flags["C_CONTIGUOUS"] and center.size == j1 - j0
+    else:
+        center = np.zeros(j1 - j0, dtype=np.float64)
+        outs = [np.zeros(j1 - j0, dtype=np.float64) for _ in range(M)] if want_workers else None
     _load().grawa_oracle_center_pull(_ptr_array(x), M, beta.ctypes.data, int(per_layer),
                                      off.ctypes.data, K, j0, j1, float(pull), center.ctypes.data,
                                      _ptr_array(outs) if want_workers else None)

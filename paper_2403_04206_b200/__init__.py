@@ -1,0 +1,26 @@
+"""B200-native GRAWA / MGRAWA / LGRAWA averaging update.
+
+The product is the CUDA library ``libgrawa.so`` (C ABI in ``include/grawa.h``); this package is
+its thin ctypes binding.  Importing the package does not load the library; the first call does,
+and fails loudly when the library cannot be built or loaded.  There is no CPU fallback.
+"""
+from .binding import (  # noqa: F401
+    GrawaError,
+    GRAWA_MAX_WORKERS,
+    grawa_clear_plans,
+    grawa_collect_kernel_times,
+    grawa_get_option,
+    grawa_grawa_step,
+    grawa_last_cuda_error,
+    grawa_last_step_status,
+    grawa_launch_count,
+    grawa_lgrawa_step,
+    grawa_mgrawa_step,
+    grawa_prox_step,
+    grawa_set_option,
+    grawa_status_string,
+    grawa_step_host,
+    grawa_version,
+    grawa_workspace_bytes,
+    library,
+)

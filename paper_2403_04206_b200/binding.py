@@ -1,0 +1,246 @@
+"""ctypes binding of libgrawa.so: argument marshalling only.
+
+Each function has the name of the C entry point it calls (see ``include/grawa.h`` for the
+meaning of every argument).  Device buffers are passed as torch CUDA tensors (float32,
+contiguous, 1-D) or as raw integer device addresses; torch is used for device memory and
+streams only.  Every step of the update runs in the library's CUDA kernels.
+"""
+from __future__ import annotations
+
+import ctypes
+from typing import Optional, Sequence
+
+import numpy as np
+
+from . import build as _build
+
+GRAWA_MAX_WORKERS = 64
+_VARIANTS = {"grawa": 0, "mgrawa": 1, "lgrawa": 2}
+
+
+class GrawaError(RuntimeError):
+    """A libgrawa entry point returned a negative status."""
+
+    def __init__(self, status: int, where: str):
+        self.status = status
+        text = library().grawa_status_string(status).decode()
+        detail = library().grawa_last_cuda_error().decode() if status == -2 else ""
+        super().__init__(f"{where}: {text} ({status})" + (f": {detail}" if detail else ""))
+
+
+class _Options(ctypes.Structure):
+    _fields_ = [("weights_out", ctypes.c_void_p), ("scores_out", ctypes.c_void_p), ("sumsq_out", ctypes.c_void_p),
+                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
+
+
+_lib = None
+
+
+def library() -> ctypes.CDLL:
+    """Loads (building first when missing or stale) libgrawa.so.  Raises if that is impossible."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    path = _build.build()
+    lib = ctypes.CDLL(path)
+    vp, i64, ci, cf = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_float
+    step_args = [vp, vp, i64, ci, cf, vp, ci, vp, vp, vp]
+    for name in ("grawa_mgrawa_step", "grawa_grawa_step", "grawa_lgrawa_step"):
+        getattr(lib, name).argtypes = step_args
+        getattr(lib, name).restype = ci
+    lib.grawa_step_host.argtypes = [ci, vp, vp, i64, ci, cf, vp, ci, vp, vp]
+    lib.grawa_step_host.restype = ci
+    lib.grawa_prox_step.argtypes = [vp, vp, i64, ci, cf, vp]
+    lib.grawa_prox_step.restype = ci
+    lib.grawa_workspace_bytes.argtypes = [i64, ci, vp, ci]
+    lib.grawa_workspace_bytes.restype = ctypes.c_size_t
+    lib.grawa_last_step_status.argtypes = [vp]
+    lib.grawa_last_step_status.restype = ci
+    lib.grawa_status_string.argtypes = [ci]
+    lib.grawa_status_string.restype = ctypes.c_char_p
+    lib.grawa_last_cuda_error.argtypes = []
+    lib.grawa_last_cuda_error.restype = ctypes.c_char_p
+    lib.grawa_version.restype = ci
+    lib.grawa_set_option.argtypes = [ctypes.c_char_p, i64]
+    lib.grawa_set_option.restype = ci
+    lib.grawa_get_option.argtypes = [ctypes.c_char_p]
+    lib.grawa_get_option.restype = i64
+    lib.grawa_launch_count.restype = i64
+    lib.grawa_clear_plans.restype = None
+    lib.grawa_collect_kernel_times.argtypes = [vp, vp, vp, vp]
+    lib.grawa_collect_kernel_times.restype = ci
+    _lib = lib
+    return lib
+
+
+# ------------------------------------------------------------------ marshalling helpers
+
+def _addr(buf) -> int:
+    """Device (or host) address of a torch tensor / numpy array / integer / None."""
+    if buf is None:
+        return 0
+    if isinstance(buf, int):
+        return buf
+    if isinstance(buf, np.ndarray):
+        if not buf.flags["C_CONTIGUOUS"]:
+            raise ValueError("numpy buffers must be C-contiguous")
+        return buf.ctypes.data
+    if hasattr(buf, "data_ptr"):
+        if not buf.is_contiguous():
+            raise ValueError("tensors must be contiguous")
+        return buf.data_ptr()
+    raise TypeError(f"cannot take the address of {type(buf)!r}")
+
+
+def _numel(buf) -> int:
+    if isinstance(buf, np.ndarray):
+        return buf.size
+    return buf.numel()
+
+
+def _check_f32(bufs):
+    for b in bufs:
+        if hasattr(b, "dtype") and str(b.dtype) not in ("torch.float32", "float32"):
+            raise TypeError(f"expected float32 buffers, got {b.dtype}")
+
+
+def _ptr_array(bufs: Sequence) -> ctypes.Array:
+    return (ctypes.c_void_p * len(bufs))(*[_addr(b) for b in bufs])
+
+
+def _stream(stream) -> int:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+def _offsets(layer_offsets):
+    if layer_offsets is None:
+        return None, 0
+    off = np.ascontiguousarray(np.asarray(layer_offsets), dtype=np.int64)
+    return off, off.size - 1
+
+
+def _raise(status: int, where: str):
+    if status < 0:
+        raise GrawaError(status, where)
+
+
+def _step(name, params, grads, pull, layer_offsets, center_out, weights_out, scores_out, sumsq_out,
+          workspace, stream, n):
+    lib = library()
+    if len(params) != len(grads):
+        raise ValueError("params and grads must have one entry per worker")
+    _check_f32(list(params) + list(grads) + ([center_out] if center_out is not None else []))
+    M = len(params)
+    if n is None:
+        n = _numel(params[0]) if M else 0
+    off, K = _offsets(layer_offsets)
+    opt = None
+    if any(b is not None for b in (weights_out, scores_out, sumsq_out, workspace)):
+        ws_bytes = 0
+        if workspace is not None:
+            ws_bytes = workspace.numel() * workspace.element_size()
+        opt = _Options(_addr(weights_out), _addr(scores_out), _addr(sumsq_out), _addr(workspace), ws_bytes)
+    status = getattr(lib, name)(_ptr_array(params), _ptr_array(grads), n, M, float(pull),
+                                off.ctypes.data if off is not None else None, K, _addr(center_out),
+                                ctypes.byref(opt) if opt is not None else None, _stream(stream))
+    _raise(status, name)
+
+
+# ------------------------------------------------------------------ entry points (same names as the C ABI)
+
+def grawa_mgrawa_step(params, grads, pull, layer_offsets=None, center_out=None, *, weights_out=None,
+                      scores_out=None, sumsq_out=None, workspace=None, stream=None, n=None) -> None:
+    """MGRAWA step (Eq. 3-4, centre, pull) in place on ``params``; see grawa_mgrawa_step in grawa.h."""
+    _step("grawa_mgrawa_step", params, grads, pull, layer_offsets, center_out, weights_out, scores_out,
+          sumsq_out, workspace, stream, n)
+
+
+def grawa_grawa_step(params, grads, pull, layer_offsets=None, center_out=None, *, weights_out=None,
+                     scores_out=None, sumsq_out=None, workspace=None, stream=None, n=None) -> None:
+    """Vanilla GRAWA step (Eq. 2: flat gradient norm); see grawa_grawa_step in grawa.h."""
+    _step("grawa_grawa_step", params, grads, pull, layer_offsets, center_out, weights_out, scores_out,
+          sumsq_out, workspace, stream, n)
+
+
+def grawa_lgrawa_step(params, grads, pull, layer_offsets, center_out=None, *, weights_out=None,
+                      scores_out=None, sumsq_out=None, workspace=None, stream=None, n=None) -> None:
+    """LGRAWA step (Eq. 5-7: per-layer weights); see grawa_lgrawa_step in grawa.h."""
+    _step("grawa_lgrawa_step", params, grads, pull, layer_offsets, center_out, weights_out, scores_out,
+          sumsq_out, workspace, stream, n)
+
+
+def grawa_step_host(variant, params, grads, pull, layer_offsets=None, center_out=None, *, stream=None, n=None) -> None:
+    """Whole step with HOST buffers (numpy arrays or pinned CPU tensors); synchronises before returning."""
+    lib = library()
+    v = _VARIANTS[variant] if isinstance(variant, str) else int(variant)
+    _check_f32(list(params) + list(grads) + ([center_out] if center_out is not None else []))
+    M = len(params)
+    if n is None:
+        n = _numel(params[0]) if M else 0
+    off, K = _offsets(layer_offsets)
+    status = lib.grawa_step_host(v, _ptr_array(params), _ptr_array(grads), n, M, float(pull),
+                                 off.ctypes.data if off is not None else None, K, _addr(center_out), _stream(stream))
+    _raise(status, "grawa_step_host")
+
+
+def grawa_prox_step(params, center, mu_over_tau, *, stream=None, n=None) -> None:
+    """Proximity step x_m <- (1 - mu/tau) x_m + (mu/tau) x_C for all workers in one pass."""
+    lib = library()
+    _check_f32(list(params) + [center])
+    M = len(params)
+    if n is None:
+        n = _numel(center)
+    _raise(lib.grawa_prox_step(_ptr_array(params), _addr(center), n, M, float(mu_over_tau), _stream(stream)),
+           "grawa_prox_step")
+
+
+def grawa_workspace_bytes(n: int, M: int, layer_offsets=None) -> int:
+    off, K = _offsets(layer_offsets)
+    return int(library().grawa_workspace_bytes(n, M, off.ctypes.data if off is not None else None, K))
+
+
+def grawa_last_step_status(stream=None) -> int:
+    """Synchronises the stream and returns the status code of the last step enqueued on it."""
+    return int(library().grawa_last_step_status(_stream(stream)))
+
+
+def grawa_status_string(status: int) -> str:
+    return library().grawa_status_string(int(status)).decode()
+
+
+def grawa_last_cuda_error() -> str:
+    return library().grawa_last_cuda_error().decode()
+
+
+def grawa_version() -> int:
+    return int(library().grawa_version())
+
+
+def grawa_set_option(name: str, value: int) -> None:
+    _raise(library().grawa_set_option(name.encode(), int(value)), f"grawa_set_option({name})")
+
+
+def grawa_get_option(name: str) -> int:
+    return int(library().grawa_get_option(name.encode()))
+
+
+def grawa_launch_count() -> int:
+    return int(library().grawa_launch_count())
+
+
+def grawa_collect_kernel_times() -> dict:
+    """Per-phase device time (ms, summed) of the steps run while option "kernel_timing" was 1."""
+    a, b, c = ctypes.c_double(), ctypes.c_double(), ctypes.c_double()
+    k = ctypes.c_int64()
+    _raise(library().grawa_collect_kernel_times(ctypes.byref(a), ctypes.byref(b), ctypes.byref(c), ctypes.byref(k)),
+           "grawa_collect_kernel_times")
+    return {"sumsq_ms": a.value, "finalize_ms": b.value, "center_pull_ms": c.value, "steps": k.value}
+
+
+def grawa_clear_plans() -> None:
+    library().grawa_clear_plans()

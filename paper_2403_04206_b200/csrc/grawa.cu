@@ -1,0 +1,547 @@
+// Host side of libgrawa: argument validation, the cached work-list plan, kernel launches and
+// the C ABI declared in include/grawa.h.  There is no CPU implementation of the update here.
+#include "../../include/grawa.h"
+
+#include <cuda_runtime.h>
+
+#include <atomic>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <memory>
+#include <mutex>
+#include <string>
+#include <vector>
+
+#include "kernels.cuh"
+
+namespace grawa {
+
+static_assert(kMaxWorkers == GRAWA_MAX_WORKERS, "header and kernels disagree on the worker limit");
+
+// ------------------------------------------------------------------ process-wide state
+static std::mutex g_mutex;
+static std::atomic<int64_t> g_launches{0};
+static int64_t g_sumsq_tile = 8192;
+static int64_t g_pull_tile = 4096;
+static int64_t g_pull_variant = 0;
+static int64_t g_kernel_timing = 0;
+static thread_local std::string t_cuda_error;
+
+static grawa_status cuda_fail(cudaError_t err, const char* what)
+{
+    char buf[512];
+    std::snprintf(buf, sizeof buf, "%s: %s (%s)", what, cudaGetErrorString(err), cudaGetErrorName(err));
+    t_cuda_error = buf;
+    return GRAWA_ERR_CUDA;
+}
+
+#define GRAWA_CUDA_TRY(expr)                                        \
+    do {                                                            \
+        cudaError_t err__ = (expr);                                 \
+        if (err__ != cudaSuccess) return cuda_fail(err__, #expr);   \
+    } while (0)
+
+static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// ------------------------------------------------------------------ work list
+// Cuts every non-empty layer at the absolute multiples of `tile` that fall inside it.
+static void build_segments(const std::vector<int64_t>& off, int64_t tile, std::vector<Segment>* segs,
+                           std::vector<int>* layer_first)
+{
+    const int K = static_cast<int>(off.size()) - 1;
+    if (layer_first) layer_first->assign(K + 1, 0);
+    int64_t count = 0;
+    for (int k = 0; k < K; ++k) {
+        if (layer_first) (*layer_first)[k] = static_cast<int>(count);
+        int64_t pos = off[k];
+        const int64_t end = off[k + 1];
+        while (pos < end) {
+            const int64_t next = std::min(end, (pos / tile + 1) * tile);
+            if (segs) segs->push_back(Segment{pos, static_cast<int>(next - pos), k});
+            ++count;
+            pos = next;
+        }
+    }
+    if (layer_first) (*layer_first)[K] = static_cast<int>(count);
+}
+
+static int64_t count_segments(const std::vector<int64_t>& off, int64_t tile)
+{
+    int64_t count = 0;
+    for (size_t k = 0; k + 1 < off.size(); ++k) {
+        if (off[k + 1] > off[k]) count += (off[k + 1] - 1) / tile - off[k] / tile + 1;
+    }
+    return count;
+}
+
+// Scratch layout (all offsets 256-byte aligned).
+struct WorkspaceLayout {
+    size_t partials, S, A, beta, words, total;
+};
+
+static WorkspaceLayout workspace_layout(int64_t C1, int K, int M)
+{
+    WorkspaceLayout w{};
+    size_t p = 0;
+    w.partials = p; p = align_up(p + sizeof(double) * static_cast<size_t>(C1) * M, 256);
+    w.S = p;        p = align_up(p + sizeof(double) * static_cast<size_t>(K) * M, 256);
+    w.A = p;        p = align_up(p + sizeof(double) * static_cast<size_t>(K) * M, 256);
+    w.beta = p;     p = align_up(p + sizeof(float) * static_cast<size_t>(K) * M, 256);
+    w.words = p;    p = align_up(p + 256, 256);   // [0] ticket (unsigned), [1] status (int)
+    w.total = p;
+    return w;
+}
+
+struct Plan {
+    int device = 0;
+    cudaStream_t stream = nullptr;
+    int64_t n = 0;
+    int M = 0, K = 0;
+    std::vector<int64_t> off;
+    int64_t tile1 = 0, tile2 = 0;
+    int C1 = 0, C2 = 0;
+    Segment* d_segs1 = nullptr;      // sum-of-squares items
+    Segment* d_segs2 = nullptr;      // per-layer centre+pull items
+    int* d_layer_first = nullptr;    // first sum-of-squares item of each layer, K+1 entries
+    void* d_ws = nullptr;            // owned scratch (used when the caller passes none)
+    WorkspaceLayout ws{};
+    float* d_stage = nullptr;        // owned staging for the host-buffer entry point
+    ~Plan()
+    {
+        cudaFree(d_segs1); cudaFree(d_segs2); cudaFree(d_layer_first); cudaFree(d_ws); cudaFree(d_stage);
+    }
+};
+
+struct PlanKey {
+    int device; cudaStream_t stream; int64_t n; int M; std::vector<int64_t> off;
+    bool operator<(const PlanKey& o) const
+    {
+        if (device != o.device) return device < o.device;
+        if (stream != o.stream) return stream < o.stream;
+        if (n != o.n) return n < o.n;
+        if (M != o.M) return M < o.M;
+        return off < o.off;
+    }
+};
+
+// Event quads recorded around the three phases of a step while "kernel_timing" is on.
+struct TimedStep { cudaEvent_t e[4]; };
+static auto& g_timed_pool = *new std::vector<TimedStep>;   // created once, reused
+static size_t g_timed_used = 0;
+
+// Heap-allocated and never destroyed: at process exit the CUDA runtime may already be gone.
+static auto& g_plans = *new std::map<PlanKey, std::unique_ptr<Plan>>;
+static auto& g_last_status = *new std::map<std::pair<int, cudaStream_t>, int*>;   // (device, stream) -> status word
+
+static grawa_status get_plan(int64_t n, int M, const std::vector<int64_t>& off, cudaStream_t stream, Plan** out)
+{
+    int device = 0;
+    GRAWA_CUDA_TRY(cudaGetDevice(&device));
+    PlanKey key{device, stream, n, M, off};
+    auto it = g_plans.find(key);
+    if (it != g_plans.end()) { *out = it->second.get(); return GRAWA_OK; }
+
+    std::unique_ptr<Plan> p(new Plan);
+    p->device = device; p->stream = stream; p->n = n; p->M = M; p->off = off;
+    p->K = static_cast<int>(off.size()) - 1;
+    p->tile1 = g_sumsq_tile; p->tile2 = g_pull_tile;
+    std::vector<Segment> s1, s2;
+    std::vector<int> first;
+    build_segments(off, p->tile1, &s1, &first);
+    build_segments(off, p->tile2, &s2, nullptr);
+    if (s1.size() * static_cast<size_t>(M) > 0x7fffffffull || s2.size() > 0x7fffffffull) return GRAWA_ERR_INVALID_ARG;
+    p->C1 = static_cast<int>(s1.size()); p->C2 = static_cast<int>(s2.size());
+    p->ws = workspace_layout(p->C1, p->K, M);
+    GRAWA_CUDA_TRY(cudaMalloc(&p->d_segs1, sizeof(Segment) * std::max<size_t>(1, s1.size())));
+    GRAWA_CUDA_TRY(cudaMalloc(&p->d_segs2, sizeof(Segment) * std::max<size_t>(1, s2.size())));
+    GRAWA_CUDA_TRY(cudaMalloc(&p->d_layer_first, sizeof(int) * first.size()));
+    GRAWA_CUDA_TRY(cudaMemcpy(p->d_segs1, s1.data(), sizeof(Segment) * s1.size(), cudaMemcpyHostToDevice));
+    GRAWA_CUDA_TRY(cudaMemcpy(p->d_segs2, s2.data(), sizeof(Segment) * s2.size(), cudaMemcpyHostToDevice));
+    GRAWA_CUDA_TRY(cudaMemcpy(p->d_layer_first, first.data(), sizeof(int) * first.size(), cudaMemcpyHostToDevice));
+    *out = p.get();
+    g_plans[key] = std::move(p);
+    return GRAWA_OK;
+}
+
+// ------------------------------------------------------------------ validation
+static bool ranges_overlap(const void* a, const void* b, size_t bytes)
+{
+    const uintptr_t x = reinterpret_cast<uintptr_t>(a), y = reinterpret_cast<uintptr_t>(b);
+    return x < y + bytes && y < x + bytes;
+}
+
+static grawa_status validate(float* const* params, const float* const* grads, int64_t n, int M, float pull,
+                             const int64_t* layer_offsets, int n_layers, const float* center_out,
+                             std::vector<int64_t>* off)
+{
+    if (M < 1 || M > GRAWA_MAX_WORKERS || n < 0 || n_layers < 0) return GRAWA_ERR_INVALID_ARG;
+    if (!(pull >= 0.0f && pull <= 1.0f)) return GRAWA_ERR_INVALID_ARG;   // also rejects NaN
+    if (params == nullptr) return GRAWA_ERR_INVALID_ARG;
+    if ((layer_offsets == nullptr) != (n_layers == 0)) return GRAWA_ERR_INVALID_ARG;
+    if (layer_offsets) {
+        if (layer_offsets[0] != 0 || layer_offsets[n_layers] != n) return GRAWA_ERR_INVALID_ARG;
+        for (int k = 0; k < n_layers; ++k)
+            if (layer_offsets[k + 1] < layer_offsets[k]) return GRAWA_ERR_INVALID_ARG;
+        off->assign(layer_offsets, layer_offsets + n_layers + 1);
+    } else {
+        off->assign({0, n});
+    }
+    if (n == 0) return GRAWA_OK;
+    const size_t bytes = static_cast<size_t>(n) * sizeof(float);
+    for (int m = 0; m < M; ++m) {
+        if (params[m] == nullptr || (grads && grads[m] == nullptr)) return GRAWA_ERR_INVALID_ARG;
+        if ((reinterpret_cast<uintptr_t>(params[m]) & 3u) || (grads && (reinterpret_cast<uintptr_t>(grads[m]) & 3u)))
+            return GRAWA_ERR_INVALID_ARG;
+    }
+    if (reinterpret_cast<uintptr_t>(center_out) & 3u) return GRAWA_ERR_INVALID_ARG;
+    for (int a = 0; a < M; ++a) {
+        for (int b = a + 1; b < M; ++b)
+            if (ranges_overlap(params[a], params[b], bytes)) return GRAWA_ERR_INVALID_ARG;
+        if (center_out && ranges_overlap(params[a], center_out, bytes)) return GRAWA_ERR_INVALID_ARG;
+        if (grads) {
+            for (int b = 0; b < M; ++b)
+                if (ranges_overlap(params[a], grads[b], bytes)) return GRAWA_ERR_INVALID_ARG;
+            if (center_out && ranges_overlap(grads[a], center_out, bytes)) return GRAWA_ERR_INVALID_ARG;
+        }
+    }
+    return GRAWA_OK;
+}
+
+static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// ------------------------------------------------------------------ launches
+template <int M>
+static void launch_center_pull(bool per_layer, int grid, cudaStream_t stream, const MutPtrs& x, float* center,
+                               const float* beta, const Segment* segs, long long n, int tile, float pull)
+{
+    if (per_layer) center_pull_kernel<M, true><<<grid, kThreads, 0, stream>>>(x, center, beta, segs, n, tile, pull, 1);
+    else center_pull_kernel<M, false><<<grid, kThreads, 0, stream>>>(x, center, beta, segs, n, tile, pull, 1);
+}
+
+template <int M>
+struct CenterPullDispatch {
+    static void run(int m, bool per_layer, int grid, cudaStream_t stream, const MutPtrs& x, float* center,
+                    const float* beta, const Segment* segs, long long n, int tile, float pull)
+    {
+        if (m == M) launch_center_pull<M>(per_layer, grid, stream, x, center, beta, segs, n, tile, pull);
+        else CenterPullDispatch<M - 1>::run(m, per_layer, grid, stream, x, center, beta, segs, n, tile, pull);
+    }
+};
+template <>
+struct CenterPullDispatch<1> {
+    static void run(int, bool, int, cudaStream_t, const MutPtrs&, float*, const float*, const Segment*, long long, int, float) {}
+};
+
+static grawa_status enqueue_step(int variant, float* const* params, const float* const* grads, int64_t n, int M,
+                                 float pull, const std::vector<int64_t>& off, float* center_out,
+                                 const grawa_options* opt, cudaStream_t stream, Plan* plan)
+{
+    const int K = plan->K;
+    // scratch
+    char* ws = static_cast<char*>(opt ? opt->workspace : nullptr);
+    if (ws) {
+        if ((reinterpret_cast<uintptr_t>(ws) & 255u) || opt->workspace_bytes < plan->ws.total) return GRAWA_ERR_WORKSPACE;
+    } else {
+        if (opt && opt->workspace_bytes != 0) return GRAWA_ERR_WORKSPACE;
+        if (!plan->d_ws) GRAWA_CUDA_TRY(cudaMalloc(&plan->d_ws, plan->ws.total));
+        ws = static_cast<char*>(plan->d_ws);
+    }
+    double* partials = reinterpret_cast<double*>(ws + plan->ws.partials);
+    double* S = reinterpret_cast<double*>(ws + plan->ws.S);
+    double* A = reinterpret_cast<double*>(ws + plan->ws.A);
+    float* beta = reinterpret_cast<float*>(ws + plan->ws.beta);
+    unsigned* ticket = reinterpret_cast<unsigned*>(ws + plan->ws.words);
+    int* status = reinterpret_cast<int*>(ws + plan->ws.words) + 1;
+    g_last_status[{plan->device, stream}] = status;
+
+    ConstPtrs gp{};
+    MutPtrs xp{};
+    bool vec_g = true, vec_x = center_out == nullptr || aligned16(center_out);
+    for (int m = 0; m < M; ++m) {
+        gp.p[m] = grads[m]; xp.p[m] = params[m];
+        vec_g = vec_g && aligned16(grads[m]);
+        vec_x = vec_x && aligned16(params[m]);
+    }
+
+    TimedStep* ts = nullptr;
+    if (g_kernel_timing) {
+        if (g_timed_used == g_timed_pool.size()) {
+            TimedStep fresh{};
+            for (auto& ev : fresh.e) GRAWA_CUDA_TRY(cudaEventCreate(&ev));
+            g_timed_pool.push_back(fresh);
+        }
+        ts = &g_timed_pool[g_timed_used++];
+        GRAWA_CUDA_TRY(cudaEventRecord(ts->e[0], stream));
+    }
+    // step 1: partial sums of squares, one CTA per (worker, item)
+    sumsq_kernel<8><<<plan->C1 * M, kThreads, 0, stream>>>(gp, plan->d_segs1, plan->C1, partials, vec_g ? 1 : 0, ticket, status);
+    ++g_launches;
+    GRAWA_CUDA_TRY(cudaGetLastError());
+    if (ts) GRAWA_CUDA_TRY(cudaEventRecord(ts->e[1], stream));
+    // steps 1b-3: S, scores, weights
+    finalize_kernel<<<K * M, kFinalizeThreads, 0, stream>>>(partials, plan->d_layer_first, plan->C1, K, M, variant, S, A, beta,
+                                                           ticket, status, opt ? opt->weights_out : nullptr,
+                                                           opt ? opt->scores_out : nullptr, opt ? opt->sumsq_out : nullptr);
+    ++g_launches;
+    GRAWA_CUDA_TRY(cudaGetLastError());
+    if (ts) GRAWA_CUDA_TRY(cudaEventRecord(ts->e[2], stream));
+    // steps 4-5
+    if (M == 1) {
+        if (center_out) {
+            const bool v = aligned16(center_out) && aligned16(params[0]);
+            const int grid = static_cast<int>(std::min<int64_t>((n + kThreads * 4 - 1) / (kThreads * 4), 148 * 16));
+            copy_kernel<<<grid, kThreads, 0, stream>>>(params[0], center_out, n, v ? 1 : 0);
+            ++g_launches;
+            GRAWA_CUDA_TRY(cudaGetLastError());
+        }
+        if (ts) GRAWA_CUDA_TRY(cudaEventRecord(ts->e[3], stream));
+        return GRAWA_OK;
+    }
+    const bool per_layer = variant == kLgrawa;
+    const int64_t tiles = per_layer ? plan->C2 : (n + plan->tile2 - 1) / plan->tile2;
+    if (tiles > 0x7fffffffll) return GRAWA_ERR_INVALID_ARG;
+    const int grid = static_cast<int>(tiles);
+    if (vec_x && M <= kMaxRegWorkers) {
+        CenterPullDispatch<kMaxRegWorkers>::run(M, per_layer, grid, stream, xp, center_out, beta, plan->d_segs2, n,
+                                                static_cast<int>(plan->tile2), pull);
+    } else {
+        center_pull_generic_kernel<<<grid, kThreads, 0, stream>>>(xp, center_out, beta, plan->d_segs2, per_layer ? 1 : 0, n,
+                                                                 static_cast<int>(plan->tile2), pull, M);
+    }
+    ++g_launches;
+    GRAWA_CUDA_TRY(cudaGetLastError());
+    if (ts) GRAWA_CUDA_TRY(cudaEventRecord(ts->e[3], stream));
+    return GRAWA_OK;
+}
+
+static grawa_status step_entry(int variant, float* const* params, const float* const* grads, int64_t n, int M, float pull,
+                               const int64_t* layer_offsets, int n_layers, float* center_out, const grawa_options* opt,
+                               cudaStream_t stream)
+{
+    if (grads == nullptr) return GRAWA_ERR_INVALID_ARG;
+    std::vector<int64_t> off;
+    grawa_status st = validate(params, grads, n, M, pull, layer_offsets, n_layers, center_out, &off);
+    if (st != GRAWA_OK || n == 0) return st;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    Plan* plan = nullptr;
+    st = get_plan(n, M, off, stream, &plan);
+    if (st != GRAWA_OK) return st;
+    return enqueue_step(variant, params, grads, n, M, pull, off, center_out, opt, stream, plan);
+}
+
+}  // namespace grawa
+
+using namespace grawa;
+
+extern "C" {
+
+int grawa_version(void) { return 100; }
+
+const char* grawa_status_string(grawa_status status)
+{
+    switch (status) {
+        case GRAWA_OK: return "ok";
+        case GRAWA_ERR_INVALID_ARG: return "invalid argument";
+        case GRAWA_ERR_CUDA: return "CUDA runtime error";
+        case GRAWA_ERR_NONFINITE: return "non-finite gradient score";
+        case GRAWA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
+        case GRAWA_ERR_TIMEOUT: return "bounded device wait ran out";
+    }
+    return "unknown status";
+}
+
+const char* grawa_last_cuda_error(void) { return t_cuda_error.c_str(); }
+
+size_t grawa_workspace_bytes(int64_t n, int M, const int64_t* layer_offsets, int n_layers)
+{
+    if (M < 1 || M > GRAWA_MAX_WORKERS || n < 0 || n_layers < 0 || (layer_offsets == nullptr) != (n_layers == 0)) return 0;
+    std::vector<int64_t> off;
+    if (layer_offsets) {
+        if (layer_offsets[0] != 0 || layer_offsets[n_layers] != n) return 0;
+        for (int k = 0; k < n_layers; ++k)
+            if (layer_offsets[k + 1] < layer_offsets[k]) return 0;
+        off.assign(layer_offsets, layer_offsets + n_layers + 1);
+    } else {
+        off.assign({0, n});
+    }
+    std::lock_guard<std::mutex> lock(g_mutex);
+    return workspace_layout(count_segments(off, g_sumsq_tile), static_cast<int>(off.size()) - 1, M).total;
+}
+
+grawa_status grawa_mgrawa_step(float* const* params, const float* const* grads, int64_t n, int M, float pull,
+                               const int64_t* layer_offsets, int n_layers, float* center_out,
+                               const grawa_options* options, grawa_stream_t stream)
+{
+    return step_entry(kMgrawa, params, grads, n, M, pull, layer_offsets, n_layers, center_out, options, stream);
+}
+
+grawa_status grawa_grawa_step(float* const* params, const float* const* grads, int64_t n, int M, float pull,
+                              const int64_t* layer_offsets, int n_layers, float* center_out,
+                              const grawa_options* options, grawa_stream_t stream)
+{
+    return step_entry(kGrawa, params, grads, n, M, pull, layer_offsets, n_layers, center_out, options, stream);
+}
+
+grawa_status grawa_lgrawa_step(float* const* params, const float* const* grads, int64_t n, int M, float pull,
+                               const int64_t* layer_offsets, int n_layers, float* center_out,
+                               const grawa_options* options, grawa_stream_t stream)
+{
+    return step_entry(kLgrawa, params, grads, n, M, pull, layer_offsets, n_layers, center_out, options, stream);
+}
+
+grawa_status grawa_step_host(grawa_variant variant, float* const* params, const float* const* grads, int64_t n, int M,
+                             float pull, const int64_t* layer_offsets, int n_layers, float* center_out,
+                             grawa_stream_t stream)
+{
+    if (variant != GRAWA_VARIANT_GRAWA && variant != GRAWA_VARIANT_MGRAWA && variant != GRAWA_VARIANT_LGRAWA)
+        return GRAWA_ERR_INVALID_ARG;
+    if (grads == nullptr) return GRAWA_ERR_INVALID_ARG;
+    std::vector<int64_t> off;
+    grawa_status st = validate(params, grads, n, M, pull, layer_offsets, n_layers, center_out, &off);
+    if (st != GRAWA_OK || n == 0) return st;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    Plan* plan = nullptr;
+    st = get_plan(n, M, off, stream, &plan);
+    if (st != GRAWA_OK) return st;
+    const size_t nn = align_up(static_cast<size_t>(n), 64);      // keeps every staged vector 256-byte aligned
+    if (!plan->d_stage) GRAWA_CUDA_TRY(cudaMalloc(&plan->d_stage, sizeof(float) * nn * (2 * static_cast<size_t>(M) + 1)));
+    std::vector<float*> dx(M);
+    std::vector<const float*> dg(M);
+    float* dc = plan->d_stage + nn * 2 * M;
+    const size_t bytes = sizeof(float) * static_cast<size_t>(n);
+    for (int m = 0; m < M; ++m) {
+        dg[m] = plan->d_stage + nn * m;
+        GRAWA_CUDA_TRY(cudaMemcpyAsync(plan->d_stage + nn * m, grads[m], bytes, cudaMemcpyHostToDevice, stream));
+    }
+    for (int m = 0; m < M; ++m) {
+        dx[m] = plan->d_stage + nn * (M + m);
+        GRAWA_CUDA_TRY(cudaMemcpyAsync(dx[m], params[m], bytes, cudaMemcpyHostToDevice, stream));
+    }
+    st = enqueue_step(variant, dx.data(), dg.data(), n, M, pull, off, center_out ? dc : nullptr, nullptr, stream, plan);
+    if (st != GRAWA_OK) return st;
+    if (M > 1)
+        for (int m = 0; m < M; ++m)
+            GRAWA_CUDA_TRY(cudaMemcpyAsync(params[m], dx[m], bytes, cudaMemcpyDeviceToHost, stream));
+    if (center_out) GRAWA_CUDA_TRY(cudaMemcpyAsync(center_out, dc, bytes, cudaMemcpyDeviceToHost, stream));
+    GRAWA_CUDA_TRY(cudaStreamSynchronize(stream));
+    return GRAWA_OK;
+}
+
+grawa_status grawa_last_step_status(grawa_stream_t stream)
+{
+    int device = 0;
+    GRAWA_CUDA_TRY(cudaGetDevice(&device));
+    int* status = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        auto it = g_last_status.find({device, stream});
+        if (it == g_last_status.end()) return GRAWA_ERR_INVALID_ARG;
+        status = it->second;
+    }
+    GRAWA_CUDA_TRY(cudaStreamSynchronize(stream));
+    int word = 0;
+    GRAWA_CUDA_TRY(cudaMemcpy(&word, status, sizeof word, cudaMemcpyDeviceToHost));
+    if (word & kStatusTimeout) return GRAWA_ERR_TIMEOUT;
+    if (word & kStatusNonFinite) return GRAWA_ERR_NONFINITE;
+    return GRAWA_OK;
+}
+
+grawa_status grawa_prox_step(float* const* params, const float* center, int64_t n, int M, float mu_over_tau,
+                             grawa_stream_t stream)
+{
+    if (center == nullptr && n > 0) return GRAWA_ERR_INVALID_ARG;
+    std::vector<int64_t> off;
+    grawa_status st = validate(params, nullptr, n, M, mu_over_tau, nullptr, 0, center, &off);
+    if (st != GRAWA_OK || n == 0) return st;
+    MutPtrs xp{};
+    bool vec = aligned16(center);
+    for (int m = 0; m < M; ++m) { xp.p[m] = params[m]; vec = vec && aligned16(params[m]); }
+    int64_t tile;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        tile = g_pull_tile;
+    }
+    const int64_t tiles = (n + tile - 1) / tile;
+    if (tiles > 0x7fffffffll) return GRAWA_ERR_INVALID_ARG;
+    prox_kernel<<<static_cast<int>(tiles), kThreads, 0, stream>>>(xp, center, n, static_cast<int>(tile), mu_over_tau, M, vec ? 1 : 0);
+    ++g_launches;
+    GRAWA_CUDA_TRY(cudaGetLastError());
+    return GRAWA_OK;
+}
+
+static void clear_plans_locked()
+{
+    cudaDeviceSynchronize();
+    g_plans.clear();
+    g_last_status.clear();
+}
+
+grawa_status grawa_set_option(const char* name, int64_t value)
+{
+    if (name == nullptr) return GRAWA_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    const bool tile_ok = value >= 1024 && value <= 1048576 && value % 1024 == 0;
+    if (std::strcmp(name, "sumsq_tile") == 0) {
+        if (!tile_ok) return GRAWA_ERR_INVALID_ARG;
+        if (value != g_sumsq_tile) { g_sumsq_tile = value; clear_plans_locked(); }
+        return GRAWA_OK;
+    }
+    if (std::strcmp(name, "pull_tile") == 0) {
+        if (!tile_ok) return GRAWA_ERR_INVALID_ARG;
+        if (value != g_pull_tile) { g_pull_tile = value; clear_plans_locked(); }
+        return GRAWA_OK;
+    }
+    if (std::strcmp(name, "pull_variant") == 0) {
+        if (value < 0 || value > 2) return GRAWA_ERR_INVALID_ARG;
+        g_pull_variant = value;
+        return GRAWA_OK;
+    }
+    if (std::strcmp(name, "kernel_timing") == 0) {
+        if (value < 0 || value > 1) return GRAWA_ERR_INVALID_ARG;
+        g_kernel_timing = value;
+        return GRAWA_OK;
+    }
+    return GRAWA_ERR_INVALID_ARG;
+}
+
+int64_t grawa_get_option(const char* name)
+{
+    if (name == nullptr) return -1;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (std::strcmp(name, "sumsq_tile") == 0) return g_sumsq_tile;
+    if (std::strcmp(name, "pull_tile") == 0) return g_pull_tile;
+    if (std::strcmp(name, "pull_variant") == 0) return g_pull_variant;
+    if (std::strcmp(name, "kernel_timing") == 0) return g_kernel_timing;
+    return -1;
+}
+
+int64_t grawa_launch_count(void) { return g_launches.load(); }
+
+grawa_status grawa_collect_kernel_times(double* sumsq_ms, double* finalize_ms, double* center_pull_ms, int64_t* steps)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    GRAWA_CUDA_TRY(cudaDeviceSynchronize());
+    double sum[3] = {0.0, 0.0, 0.0};
+    for (size_t i = 0; i < g_timed_used; ++i)
+        for (int ph = 0; ph < 3; ++ph) {
+            float ms = 0.f;
+            GRAWA_CUDA_TRY(cudaEventElapsedTime(&ms, g_timed_pool[i].e[ph], g_timed_pool[i].e[ph + 1]));
+            sum[ph] += ms;
+        }
+    if (sumsq_ms) *sumsq_ms = sum[0];
+    if (finalize_ms) *finalize_ms = sum[1];
+    if (center_pull_ms) *center_pull_ms = sum[2];
+    if (steps) *steps = static_cast<int64_t>(g_timed_used);
+    g_timed_used = 0;
+    return GRAWA_OK;
+}
+
+void grawa_clear_plans(void)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    clear_plans_locked();
+}
+
+}  // extern "C"

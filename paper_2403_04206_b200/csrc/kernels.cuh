@@ -1,0 +1,382 @@
+// Device code of libgrawa: segmented sum of squares, score/weight finalisation,
+// fused centre + pull, proximity step.  Written for sm_100a; HBM-bandwidth bound,
+// plain ALU arithmetic (a small-M weighted sum is not a dense contraction).
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace grawa {
+
+constexpr int kMaxWorkers = 64;
+constexpr int kThreads = 256;          // threads per CTA of the streaming kernels
+constexpr int kFinalizeThreads = 128;
+constexpr int kMaxRegWorkers = 16;     // largest M the register-resident centre+pull kernel is built for
+
+enum Variant { kGrawa = 0, kMgrawa = 1, kLgrawa = 2 };
+enum StatusBits { kStatusNonFinite = 1, kStatusTimeout = 2 };
+
+struct ConstPtrs { const float* p[kMaxWorkers]; };
+struct MutPtrs { float* p[kMaxWorkers]; };
+
+// One work item: elements [begin, begin+len) of the flat vector, all inside layer `layer`.
+// Items are cut at layer boundaries and at absolute multiples of the tile size, so every
+// interior boundary is 16-byte aligned relative to the base pointer.
+struct Segment {
+    long long begin;
+    int len;
+    int layer;
+};
+
+// Streaming accesses: every byte is touched once per step, so keep it out of the way in L1/L2.
+__device__ __forceinline__ float4 ld_stream4(const float4* p) { return __ldcs(p); }
+__device__ __forceinline__ float ld_stream1(const float* p) { return __ldcs(p); }
+__device__ __forceinline__ void st_stream4(float4* p, float4 v) { __stcs(p, v); }
+__device__ __forceinline__ void st_stream1(float* p, float v) { __stcs(p, v); }
+
+// Splits [b, e) into scalar head [b, hb), 16-byte aligned body [hb, te), scalar tail [te, e).
+// With vec_ok == 0 (a base pointer that is not 16-byte aligned) everything is head.
+__device__ __forceinline__ void split_range(long long b, long long e, int vec_ok, long long& hb, long long& te)
+{
+    if (vec_ok) {
+        hb = min((b + 3) & ~3LL, e);
+        te = max(e & ~3LL, hb);
+    } else {
+        hb = e;
+        te = e;
+    }
+}
+
+// Deterministic block sum of one double per thread: xor-free shuffle-down tree inside each warp,
+// then thread 0 adds the warp results in warp order.  Result valid in thread 0.
+template <int THREADS>
+__device__ __forceinline__ double block_sum_fixed_order(double v)
+{
+    __shared__ double warp_part[THREADS / 32];
+#pragma unroll
+    for (int d = 16; d > 0; d >>= 1) v += __shfl_down_sync(0xffffffffu, v, d);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (lane == 0) warp_part[warp] = v;
+    __syncthreads();
+    double total = 0.0;
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int w = 0; w < THREADS / 32; ++w) total += warp_part[w];
+    }
+    return total;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Step 1 (Eq. 3 / Eq. 5): partial[m][s] = sum of g_m[j]^2 over segment s.  One CTA per
+// (worker, segment).  fp32 squares are accumulated in runs of UNROLL terms per accumulator and
+// the runs are combined in fp64, in an order fixed by the launch shape only.
+// CTA 0 also clears the ticket and status words for the finalisation that follows on the stream.
+// ---------------------------------------------------------------------------------------------
+template <int UNROLL>
+__global__ void __launch_bounds__(kThreads)
+sumsq_kernel(ConstPtrs grads, const Segment* __restrict__ segs, int C, double* __restrict__ partials,
+             int vec_ok, unsigned* __restrict__ ticket, int* __restrict__ status)
+{
+    const int item = blockIdx.x;
+    const int m = item / C;
+    const int s = item - m * C;
+    const Segment sg = segs[s];
+    const float* __restrict__ g = grads.p[m];
+    const long long b = sg.begin, e = b + sg.len;
+    const int tid = threadIdx.x;
+    if (item == 0 && tid == 0) { *ticket = 0u; *status = 0; }
+
+    long long hb, te;
+    split_range(b, e, vec_ok, hb, te);
+    double dacc = 0.0;
+
+    const float4* __restrict__ g4 = reinterpret_cast<const float4*>(g + hb);
+    const int ncol = static_cast<int>((te - hb) >> 2);
+    for (int c0 = 0; c0 < ncol; c0 += kThreads * UNROLL) {
+        float4 v[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const int c = c0 + u * kThreads + tid;
+            v[u] = (c < ncol) ? ld_stream4(g4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            a0 = fmaf(v[u].x, v[u].x, a0);
+            a1 = fmaf(v[u].y, v[u].y, a1);
+            a2 = fmaf(v[u].z, v[u].z, a2);
+            a3 = fmaf(v[u].w, v[u].w, a3);
+        }
+        dacc += (static_cast<double>(a0) + static_cast<double>(a1)) +
+                (static_cast<double>(a2) + static_cast<double>(a3));
+    }
+    for (long long i = b + tid; i < hb; i += kThreads) {
+        const double v = static_cast<double>(ld_stream1(g + i));
+        dacc += v * v;
+    }
+    for (long long i = te + tid; i < e; i += kThreads) {
+        const double v = static_cast<double>(ld_stream1(g + i));
+        dacc += v * v;
+    }
+    const double total = block_sum_fixed_order<kThreads>(dacc);
+    if (tid == 0) partials[static_cast<size_t>(m) * C + s] = total;
+}
+
+// Step 3 for one group of M scores (Eq. 2 / 4 / 7) with the zero-score limit and the non-finite
+// fallback.  A has stride 1.  Returns 1 if a non-finite score was met.
+__device__ inline int weights_group(const double* A, int M, float* beta, float* beta_copy)
+{
+    int zeros = 0, finite = 0, flagged = 0;
+    for (int m = 0; m < M; ++m) {
+        const double a = A[m];
+        if (!isfinite(a)) flagged = 1;
+        else { ++finite; if (a == 0.0) ++zeros; }
+    }
+    double z = 0.0;
+    if (finite > 0 && zeros == 0)
+        for (int m = 0; m < M; ++m)
+            if (isfinite(A[m])) z += 1.0 / A[m];
+    for (int m = 0; m < M; ++m) {
+        const double a = A[m];
+        double w;
+        if (finite == 0) w = 1.0 / M;
+        else if (zeros > 0) w = (isfinite(a) && a == 0.0) ? 1.0 / zeros : 0.0;
+        else w = isfinite(a) ? (1.0 / a) / z : 0.0;
+        const float wf = static_cast<float>(w);
+        beta[m] = wf;
+        if (beta_copy) beta_copy[m] = wf;
+    }
+    return flagged;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Steps 1b-3: one CTA per (layer, worker) adds that pair's partials in a fixed order into
+// S[k][m]; the CTA that takes the last ticket then turns S into scores and weights.
+// No CTA waits for another: the last arrival is found with one atomic ticket.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kFinalizeThreads)
+finalize_kernel(const double* __restrict__ partials, const int* __restrict__ layer_seg_first, int C, int K, int M,
+                int variant, double* S, double* A, float* beta, unsigned* ticket, int* status,
+                float* weights_out, double* scores_out, double* sumsq_out)
+{
+    const int k = blockIdx.x / M;
+    const int m = blockIdx.x - k * M;
+    const int tid = threadIdx.x;
+    const int s0 = layer_seg_first[k], s1 = layer_seg_first[k + 1];
+    const double* __restrict__ row = partials + static_cast<size_t>(m) * C;
+    double acc = 0.0;
+    for (int s = s0 + tid; s < s1; s += kFinalizeThreads) acc += row[s];
+    const double total = block_sum_fixed_order<kFinalizeThreads>(acc);
+
+    __shared__ int is_last;
+    if (tid == 0) {
+        S[static_cast<size_t>(k) * M + m] = total;
+        if (sumsq_out) sumsq_out[static_cast<size_t>(k) * M + m] = total;
+        __threadfence();
+        const unsigned t = atomicAdd(ticket, 1u);
+        is_last = (t == static_cast<unsigned>(K) * M - 1u);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+
+    const volatile double* Sv = S;
+    int flagged = 0;
+    if (variant == kLgrawa) {
+        for (int kk = tid; kk < K; kk += kFinalizeThreads) {
+            double* Arow = A + static_cast<size_t>(kk) * M;
+            for (int mm = 0; mm < M; ++mm) {
+                const double a = sqrt(Sv[static_cast<size_t>(kk) * M + mm]);
+                Arow[mm] = a;
+                if (scores_out) scores_out[static_cast<size_t>(kk) * M + mm] = a;
+            }
+            flagged |= weights_group(Arow, M, beta + static_cast<size_t>(kk) * M,
+                                     weights_out ? weights_out + static_cast<size_t>(kk) * M : nullptr);
+        }
+    } else {
+        if (tid < M) {
+            double a = 0.0;
+            if (variant == kMgrawa) {
+                for (int kk = 0; kk < K; ++kk) a += sqrt(Sv[static_cast<size_t>(kk) * M + tid]);
+            } else {
+                for (int kk = 0; kk < K; ++kk) a += Sv[static_cast<size_t>(kk) * M + tid];
+                a = sqrt(a);
+            }
+            A[tid] = a;
+            if (scores_out) scores_out[tid] = a;
+        }
+        __syncthreads();
+        if (tid == 0) flagged = weights_group(A, M, beta, weights_out);
+    }
+    if (flagged) atomicOr(status, kStatusNonFinite);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Steps 4-5, register variant: one thread owns a 16-byte column of all M workers, so each
+// parameter is read once and M independent vector loads are in flight per column.
+//   x_C = sum_m beta_m x_m   (fp32 FMA chain, m = 0..M-1)      x_m <- fmaf(pull, x_C, (1-pull) x_m)
+// PER_LAYER: one CTA per Segment, weights of the segment's layer (Eq. 7); otherwise flat tiles of
+// `tile` elements and one weight per worker (Eq. 2 / Eq. 4).
+// ---------------------------------------------------------------------------------------------
+template <int M>
+__device__ __forceinline__ void pull_scalar(const MutPtrs& x, float* center, const float (&w)[M],
+                                            float lambda, float oml, long long i)
+{
+    float v[M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) v[m] = ld_stream1(x.p[m] + i);
+    float c = w[0] * v[0];
+#pragma unroll
+    for (int m = 1; m < M; ++m) c = fmaf(w[m], v[m], c);
+    if (center) st_stream1(center + i, c);
+#pragma unroll
+    for (int m = 0; m < M; ++m) st_stream1(x.p[m] + i, fmaf(lambda, c, oml * v[m]));
+}
+
+template <int M, bool PER_LAYER>
+__global__ void __launch_bounds__(kThreads)
+center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restrict__ beta,
+                   const Segment* __restrict__ segs, long long n, int tile, float lambda, int vec_ok)
+{
+    constexpr int COLS = (M <= 4) ? 4 : (M <= 8) ? 2 : 1;
+    long long b, e;
+    const float* __restrict__ bt = beta;
+    if (PER_LAYER) {
+        const Segment sg = segs[blockIdx.x];
+        b = sg.begin;
+        e = b + sg.len;
+        bt = beta + static_cast<size_t>(sg.layer) * M;
+    } else {
+        b = static_cast<long long>(blockIdx.x) * tile;
+        e = min(n, b + tile);
+    }
+    float w[M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) w[m] = bt[m];
+    const float oml = 1.0f - lambda;
+    const int tid = threadIdx.x;
+
+    long long hb, te;
+    split_range(b, e, vec_ok, hb, te);
+    const int ncol = static_cast<int>((te - hb) >> 2);
+    for (int c0 = 0; c0 < ncol; c0 += kThreads * COLS) {
+        float4 v[COLS][M];
+#pragma unroll
+        for (int q = 0; q < COLS; ++q) {
+            const int c = c0 + q * kThreads + tid;
+            if (c < ncol) {
+#pragma unroll
+                for (int m = 0; m < M; ++m) v[q][m] = ld_stream4(reinterpret_cast<const float4*>(x.p[m] + hb) + c);
+            }
+        }
+#pragma unroll
+        for (int q = 0; q < COLS; ++q) {
+            const int c = c0 + q * kThreads + tid;
+            if (c < ncol) {
+                float4 cc;
+                cc.x = w[0] * v[q][0].x; cc.y = w[0] * v[q][0].y; cc.z = w[0] * v[q][0].z; cc.w = w[0] * v[q][0].w;
+#pragma unroll
+                for (int m = 1; m < M; ++m) {
+                    cc.x = fmaf(w[m], v[q][m].x, cc.x); cc.y = fmaf(w[m], v[q][m].y, cc.y);
+                    cc.z = fmaf(w[m], v[q][m].z, cc.z); cc.w = fmaf(w[m], v[q][m].w, cc.w);
+                }
+                if (center) st_stream4(reinterpret_cast<float4*>(center + hb) + c, cc);
+#pragma unroll
+                for (int m = 0; m < M; ++m) {
+                    float4 o;
+                    o.x = fmaf(lambda, cc.x, oml * v[q][m].x); o.y = fmaf(lambda, cc.y, oml * v[q][m].y);
+                    o.z = fmaf(lambda, cc.z, oml * v[q][m].z); o.w = fmaf(lambda, cc.w, oml * v[q][m].w);
+                    st_stream4(reinterpret_cast<float4*>(x.p[m] + hb) + c, o);
+                }
+            }
+        }
+    }
+    for (long long i = b + tid; i < hb; i += kThreads) pull_scalar<M>(x, center, w, lambda, oml, i);
+    for (long long i = te + tid; i < e; i += kThreads) pull_scalar<M>(x, center, w, lambda, oml, i);
+}
+
+// Steps 4-5 for any M up to kMaxWorkers and any alignment: scalar, two passes over the workers
+// (the second pass re-reads the elements the same thread has just read, from cache).
+__global__ void __launch_bounds__(kThreads)
+center_pull_generic_kernel(MutPtrs x, float* __restrict__ center, const float* __restrict__ beta,
+                           const Segment* __restrict__ segs, int per_layer, long long n, int tile,
+                           float lambda, int M)
+{
+    long long b, e;
+    const float* __restrict__ bt = beta;
+    if (per_layer) {
+        const Segment sg = segs[blockIdx.x];
+        b = sg.begin;
+        e = b + sg.len;
+        bt = beta + static_cast<size_t>(sg.layer) * M;
+    } else {
+        b = static_cast<long long>(blockIdx.x) * tile;
+        e = min(n, b + tile);
+    }
+    __shared__ float w[kMaxWorkers];
+    if (threadIdx.x < M) w[threadIdx.x] = bt[threadIdx.x];
+    __syncthreads();
+    const float oml = 1.0f - lambda;
+    for (long long i = b + threadIdx.x; i < e; i += kThreads) {
+        float c = w[0] * x.p[0][i];
+        for (int m = 1; m < M; ++m) c = fmaf(w[m], x.p[m][i], c);
+        if (center) center[i] = c;
+        for (int m = 0; m < M; ++m) x.p[m][i] = fmaf(lambda, c, oml * x.p[m][i]);
+    }
+}
+
+// M = 1: the centre is the single worker; the worker itself is left untouched.
+__global__ void __launch_bounds__(kThreads)
+copy_kernel(const float* __restrict__ src, float* __restrict__ dst, long long n, int vec_ok)
+{
+    const long long stride = static_cast<long long>(gridDim.x) * kThreads;
+    const long long t = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x;
+    const long long n4 = vec_ok ? (n >> 2) : 0;
+    for (long long c = t; c < n4; c += stride)
+        st_stream4(reinterpret_cast<float4*>(dst) + c, ld_stream4(reinterpret_cast<const float4*>(src) + c));
+    for (long long i = (n4 << 2) + t; i < n; i += stride) dst[i] = src[i];
+}
+
+// Proximity step ("Prox." line of Algorithms 1-2): x_m <- fmaf(a, x_C, (1-a) x_m), a = mu/tau.
+// One CTA per flat tile; the centre column is loaded once and reused for all M workers.
+__global__ void __launch_bounds__(kThreads)
+prox_kernel(MutPtrs x, const float* __restrict__ center, long long n, int tile, float a, int M, int vec_ok)
+{
+    const long long b = static_cast<long long>(blockIdx.x) * tile;
+    const long long e = min(n, b + tile);
+    const float oma = 1.0f - a;
+    long long hb, te;
+    split_range(b, e, vec_ok, hb, te);
+    const int ncol = static_cast<int>((te - hb) >> 2);
+    for (int c = threadIdx.x; c < ncol; c += kThreads) {
+        const float4 cc = ld_stream4(reinterpret_cast<const float4*>(center + hb) + c);
+        int m = 0;
+        for (; m + 4 <= M; m += 4) {
+            float4 v[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) v[q] = ld_stream4(reinterpret_cast<const float4*>(x.p[m + q] + hb) + c);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                float4 o;
+                o.x = fmaf(a, cc.x, oma * v[q].x); o.y = fmaf(a, cc.y, oma * v[q].y);
+                o.z = fmaf(a, cc.z, oma * v[q].z); o.w = fmaf(a, cc.w, oma * v[q].w);
+                st_stream4(reinterpret_cast<float4*>(x.p[m + q] + hb) + c, o);
+            }
+        }
+        for (; m < M; ++m) {
+            const float4 v = ld_stream4(reinterpret_cast<const float4*>(x.p[m] + hb) + c);
+            float4 o;
+            o.x = fmaf(a, cc.x, oma * v.x); o.y = fmaf(a, cc.y, oma * v.y);
+            o.z = fmaf(a, cc.z, oma * v.z); o.w = fmaf(a, cc.w, oma * v.w);
+            st_stream4(reinterpret_cast<float4*>(x.p[m] + hb) + c, o);
+        }
+    }
+    for (int pass = 0; pass < 2; ++pass) {
+        const long long lo = pass ? te : b, hi = pass ? e : hb;
+        for (long long i = lo + threadIdx.x; i < hi; i += kThreads) {
+            const float c = center[i];
+            for (int m = 0; m < M; ++m) x.p[m][i] = fmaf(a, c, oma * x.p[m][i]);
+        }
+    }
+}
+
+}  // namespace grawa

@@ -1,0 +1,375 @@
+"""GPU parity: the CUDA path, called through the C ABI, against the float64 oracle on the same
+seeded inputs, element by element; plus the exact-arithmetic, determinism and edge-case checks."""
+import numpy as np
+import pytest
+
+import gen
+import oracle
+from gpu_util import compare_with_oracle, gpu_step, to_device
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def grawa():
+    import torch
+    assert torch.cuda.is_available()
+    import paper_2403_04206_b200 as g
+    g.library()          # fails loudly if the CUDA library cannot be built or loaded
+    return g
+
+
+_inputs_cache = {}
+
+
+def inputs(name):
+    """Seeded inputs of a named benchmark workload (kept for the module: the big ones are costly)."""
+    if name not in _inputs_cache:
+        _inputs_cache.clear()           # hold one big workload at a time
+        _inputs_cache[name] = gen.make_inputs(gen.CONFIGS[name])
+    return _inputs_cache[name]
+
+
+# ------------------------------------------------------------------ the five benchmark workloads, full size
+
+@pytest.mark.parametrize("variant", ["mgrawa", "lgrawa", "grawa"])
+@pytest.mark.parametrize("name", ["toy10", "resnet20_cifar", "resnet18_imagenet"])
+def test_parity_small_and_medium_workloads(grawa, name, variant):
+    cfg = gen.CONFIGS[name]
+    p, g = inputs(name)
+    res = gpu_step(grawa, variant, p, g, cfg.pull, cfg.offsets())
+    compare_with_oracle(res, variant, p, g, cfg.pull, cfg.offsets())
+    assert grawa.grawa_last_step_status() == 0
+
+
+@pytest.mark.parametrize("variant", ["mgrawa", "lgrawa"])
+@pytest.mark.parametrize("name", ["vgg16", "vit_b16"])
+def test_parity_large_workloads(grawa, name, variant):
+    cfg = gen.CONFIGS[name]
+    p, g = inputs(name)
+    res = gpu_step(grawa, variant, p, g, cfg.pull, cfg.offsets())
+    stats = compare_with_oracle(res, variant, p, g, cfg.pull, cfg.offsets())
+    print(name, variant, stats)
+    if name == "vit_b16" and variant == "mgrawa":
+        # the worker with 100x larger gradients gets about 1/100 of a peer's weight
+        assert 50 < res["beta"][1] / res["beta"][0] < 200
+
+
+@pytest.mark.parametrize("pull", [0.3, 0.7])
+@pytest.mark.parametrize("variant", ["mgrawa", "lgrawa"])
+def test_parity_other_pull_strengths(grawa, variant, pull):
+    cfg = gen.CONFIGS["resnet20_cifar"]
+    p, g = inputs("resnet20_cifar")
+    res = gpu_step(grawa, variant, p, g, pull, cfg.offsets())
+    compare_with_oracle(res, variant, p, g, pull, cfg.offsets())
+
+
+# ------------------------------------------------------------------ adversarial layer tables and worker counts
+
+TABLES = [
+    [1], [3], [5], [7], [4], [8192], [8193], [4096, 4096], [4095, 4097],
+    [1, 3, 5, 7], [7, 5, 3, 1, 2, 6], [0, 5, 0, 0, 9, 0], [10, 1000, 10, 8192, 3, 20000, 1],
+    [16384, 1, 16383, 2, 4094, 4098], [33000], [1023, 1025, 2047, 2049, 4095, 4097, 8191, 8193],
+]
+
+
+@pytest.mark.parametrize("variant", ["mgrawa", "lgrawa", "grawa"])
+@pytest.mark.parametrize("sizes", TABLES, ids=lambda s: "-".join(map(str, s)))
+def test_parity_adversarial_layer_tables(grawa, sizes, variant):
+    cfg = gen.custom_config(sizes, 3, seed=11)
+    p, g = gen.make_inputs(cfg)
+    res = gpu_step(grawa, variant, p, g, 0.5, cfg.offsets())
+    compare_with_oracle(res, variant, p, g, 0.5, cfg.offsets())
+
+
+@pytest.mark.parametrize("variant", ["mgrawa", "lgrawa"])
+@pytest.mark.parametrize("M", list(range(1, 18)) + [24, 33, 64])
+def test_parity_worker_counts(grawa, M, variant):
+    cfg = gen.custom_config([10, 5000, 3, 12000, 777], M, seed=100 + M, log10_sigma=(-2.0, 0.0))
+    p, g = gen.make_inputs(cfg)
+    before = [a.copy() for a in p]
+    res = gpu_step(grawa, variant, p, g, 0.5, cfg.offsets())
+    compare_with_oracle(res, variant, p, g, 0.5, cfg.offsets(), check_workers=(M > 1))
+    if M == 1:   # identity: the worker is untouched, the centre is the worker
+        assert np.array_equal(res["workers"][0].cpu().numpy(), before[0])
+        assert np.array_equal(res["center"].cpu().numpy(), before[0])
+
+
+def test_parity_without_layer_table_is_the_flat_norm(grawa):
+    cfg = gen.custom_config([30000], 5, seed=5)
+    p, g = gen.make_inputs(cfg)
+    res = gpu_step(grawa, "mgrawa", p, g, 0.5, None)
+    compare_with_oracle(res, "grawa", p, g, 0.5, None)
+
+
+def test_parity_unaligned_base_pointers(grawa):
+    """Workers that start 4 bytes into an allocation take the scalar kernels; results are the same."""
+    import torch
+    cfg = gen.custom_config([10, 5000, 3, 9000], 4, seed=21)
+    p, g = gen.make_inputs(cfg)
+    n = cfg.n
+    xs = [torch.zeros(n + 1, device="cuda")[1:] for _ in range(4)]
+    gs = [torch.zeros(n + 1, device="cuda")[1:] for _ in range(4)]
+    for variant in ("mgrawa", "lgrawa"):
+        for t, a in zip(xs + gs, p + g):
+            t.copy_(torch.from_numpy(a))
+        res = gpu_step(grawa, variant, p, g, 0.5, cfg.offsets(), params_dev=xs, grads_dev=gs)
+        compare_with_oracle(res, variant, p, g, 0.5, cfg.offsets())
+
+
+# ------------------------------------------------------------------ exact arithmetic: indexing is bit-exact
+
+def test_sumsq_bit_exact_on_integer_gradients(grawa):
+    """Small-integer gradients make every partial sum exact in fp32 and fp64: the S table must be
+    bit-identical to the oracle's, which exposes any off-by-one, gap or overlap between work items."""
+    sizes = [10, 1000, 8192, 3, 20000, 1, 4097, 70000]
+    rng = np.random.default_rng(3)
+    off = np.concatenate([[0], np.cumsum(sizes)])
+    g = [rng.integers(-3, 4, size=off[-1]).astype(np.float32) for _ in range(3)]
+    p = [rng.normal(size=off[-1]).astype(np.float32) for _ in range(3)]
+    res = gpu_step(grawa, "lgrawa", p, g, 0.5, off)
+    assert np.array_equal(res["S"], oracle.sumsq(g, off))
+    # a single 1 at every layer's first and last element
+    for k in range(len(sizes)):
+        for pos in {off[k], off[k + 1] - 1}:
+            g1 = [np.zeros(off[-1], np.float32) for _ in range(2)]
+            g1[0][pos] = 1.0
+            g1[1][pos] = 2.0
+            S = gpu_step(grawa, "lgrawa", p[:2], g1, 0.5, off)["S"]
+            expect = np.zeros((len(sizes), 2)); expect[k] = [1, 4]
+            assert np.array_equal(S, expect), (k, pos)
+
+
+def test_centre_bit_exact_with_dyadic_weights(grawa):
+    """Gradient norms 1, 1, 2, 4 per layer give weights with short binary expansions only when
+    they are dyadic; use norms (1, 1, 1, 1) -> 1/4 each and (1, 1) -> 1/2: with integer parameters
+    every product and sum is exact, so centre and workers must match the oracle bit for bit."""
+    sizes = [5, 4096, 3, 9001]
+    off = np.concatenate([[0], np.cumsum(sizes)])
+    n = int(off[-1])
+    rng = np.random.default_rng(4)
+    for M in (2, 4, 8):
+        g = []
+        for m in range(M):
+            gm = np.zeros(n, np.float32)
+            for k in range(len(sizes)):
+                gm[off[k] + (m % sizes[k])] = 1.0 if m % 2 == 0 else -1.0     # every layer norm is 1
+            g.append(gm)
+        p = [rng.integers(-1000, 1000, size=n).astype(np.float32) for _ in range(M)]
+        for variant in ("mgrawa", "lgrawa"):
+            res = gpu_step(grawa, variant, p, g, 0.5, off)
+            ref = oracle.step(p, g, 0.5, variant, off)
+            assert np.array_equal(res["beta"].astype(np.float64), ref["beta"])
+            assert np.array_equal(res["center"].cpu().numpy().astype(np.float64), ref["center"])
+            for m in range(M):
+                assert np.array_equal(res["workers"][m].cpu().numpy().astype(np.float64), ref["workers"][m])
+
+
+def test_layer_boundaries_select_the_right_weights(grawa):
+    """LGRAWA with one-hot weights that alternate between workers from layer to layer: every
+    element of the centre must be bit-equal to the worker that owns its layer."""
+    sizes = [1, 2, 3, 4097, 5, 8191, 1, 8193, 7]
+    off = np.concatenate([[0], np.cumsum(sizes)])
+    n = int(off[-1])
+    rng = np.random.default_rng(5)
+    p = [rng.normal(size=n).astype(np.float32) for _ in range(3)]
+    g = [rng.normal(size=n).astype(np.float32) for _ in range(3)]
+    owner = np.zeros(n, dtype=np.int64)
+    for k in range(len(sizes)):
+        g[k % 3][off[k]:off[k + 1]] = 0.0       # zero gradient in layer k -> that worker takes weight 1
+        owner[off[k]:off[k + 1]] = k % 3
+    res = gpu_step(grawa, "lgrawa", p, g, 1.0, off)
+    want = np.choose(owner, p)
+    assert np.array_equal(res["center"].cpu().numpy(), want)
+    for m in range(3):
+        assert np.array_equal(res["workers"][m].cpu().numpy(), want)      # full pull
+
+
+# ------------------------------------------------------------------ invariants on the GPU result itself
+
+@pytest.mark.parametrize("variant", ["mgrawa", "lgrawa"])
+def test_pull_extremes_are_bit_exact(grawa, variant):
+    cfg = gen.CONFIGS["toy10"]
+    p, g = inputs("toy10")
+    r1 = gpu_step(grawa, variant, p, g, 1.0, cfg.offsets())
+    c = r1["center"].cpu().numpy()
+    for w in r1["workers"]:
+        assert np.array_equal(w.cpu().numpy(), c)
+    r0 = gpu_step(grawa, variant, p, g, 0.0, cfg.offsets())
+    for w, a in zip(r0["workers"], p):
+        assert np.array_equal(w.cpu().numpy(), a)
+    assert np.array_equal(r0["center"].cpu().numpy(), c)
+
+
+@pytest.mark.parametrize("variant", ["mgrawa", "lgrawa"])
+def test_run_to_run_bitwise_determinism(grawa, variant):
+    cfg = gen.CONFIGS["resnet18_imagenet"]
+    p, g = inputs("resnet18_imagenet")
+    a = gpu_step(grawa, variant, p, g, 0.5, cfg.offsets())
+    b = gpu_step(grawa, variant, p, g, 0.5, cfg.offsets())
+    assert np.array_equal(a["S"], b["S"]) and np.array_equal(a["beta"], b["beta"])
+    assert np.array_equal(a["center"].cpu().numpy(), b["center"].cpu().numpy())
+    for u, v in zip(a["workers"], b["workers"]):
+        assert bool((u == v).all())
+
+
+def test_weights_sum_to_one_and_equal_norms_give_the_mean(grawa):
+    import torch
+    cfg = gen.custom_config([3000, 17, 9000], 6, seed=8)
+    p, g = gen.make_inputs(cfg)
+    res = gpu_step(grawa, "lgrawa", p, g, 0.5, cfg.offsets())
+    assert np.allclose(res["beta"].sum(axis=1), 1.0, atol=3e-7)
+    g_same = [g[0].copy() * (-1) ** m for m in range(6)]          # equal norms
+    res = gpu_step(grawa, "mgrawa", p, g_same, 0.5, cfg.offsets())
+    assert np.array_equal(res["beta"], np.full(6, np.float32(1 / 6)))
+    mean = torch.stack(to_device(p)).double().mean(dim=0).cpu().numpy()
+    assert np.abs(res["center"].cpu().numpy() - mean).max() <= 2e-6 * max(np.abs(a).max() for a in p)
+
+
+def test_centre_invariant_to_worker_permutation(grawa):
+    cfg = gen.custom_config([5000, 33, 7000], 5, seed=9)
+    p, g = gen.make_inputs(cfg)
+    ref = gpu_step(grawa, "lgrawa", p, g, 0.5, cfg.offsets())["center"].cpu().numpy()
+    perm = [3, 0, 4, 2, 1]
+    got = gpu_step(grawa, "lgrawa", [p[i] for i in perm], [g[i] for i in perm], 0.5, cfg.offsets())["center"].cpu().numpy()
+    assert np.abs(got - ref).max() <= 2e-6 * max(np.abs(a).max() for a in p)
+
+
+# ------------------------------------------------------------------ zero and non-finite scores
+
+def test_zero_and_nonfinite_scores_follow_the_stated_policy(grawa):
+    sizes = [100, 5000, 64]
+    off = np.concatenate([[0], np.cumsum(sizes)])
+    cfg = gen.custom_config(sizes, 4, seed=13)
+    p, g = gen.make_inputs(cfg)
+    g[1][off[1]:off[2]] = 0.0                       # worker 1 has zero gradient in layer 1
+    g[2][:] = 0.0                                   # worker 2 has zero gradient everywhere
+    res = gpu_step(grawa, "lgrawa", p, g, 0.5, off)
+    compare_with_oracle(res, "lgrawa", p, g, 0.5, off)
+    assert np.array_equal(res["beta"][1], [0, 0.5, 0.5, 0]) and np.array_equal(res["beta"][0], [0, 0, 1, 0])
+    assert grawa.grawa_last_step_status() == 0
+    res = gpu_step(grawa, "mgrawa", p, g, 0.5, off)
+    assert np.array_equal(res["beta"], [0, 0, 1, 0])
+    # NaN / Inf gradients: flagged, that worker gets weight 0, nothing traps
+    g[0][off[1] + 7] = np.nan
+    g[3][5] = np.inf
+    for variant in ("lgrawa", "mgrawa"):
+        res = gpu_step(grawa, variant, p, g, 0.5, off)
+        ref_beta, flagged = oracle.weights(oracle.scores(oracle.sumsq(g, off), variant))
+        assert flagged and grawa.grawa_last_step_status() == -3
+        assert np.allclose(res["beta"], ref_beta, rtol=1e-5)
+        assert np.isfinite(res["center"].cpu().numpy()).all()
+    # a clean step afterwards clears the status
+    g[0][off[1] + 7] = 0.5
+    g[3][5] = 0.5
+    gpu_step(grawa, "mgrawa", p, g, 0.5, off)
+    assert grawa.grawa_last_step_status() == 0
+
+
+# ------------------------------------------------------------------ optional arguments and the other entry points
+
+def test_caller_workspace_and_no_centre(grawa):
+    import torch
+    cfg = gen.CONFIGS["resnet20_cifar"]
+    p, g = inputs("resnet20_cifar")
+    off = cfg.offsets()
+    need = grawa.grawa_workspace_bytes(cfg.n, cfg.M, off)
+    ws = torch.empty(need + 256, dtype=torch.uint8, device="cuda")
+    ws.fill_(0xFF)                                   # scratch contents must not matter
+    ref = gpu_step(grawa, "lgrawa", p, g, 0.5, off)
+    res = gpu_step(grawa, "lgrawa", p, g, 0.5, off, workspace=ws[:need], want_center=False)
+    assert res["center"] is None
+    for u, v in zip(ref["workers"], res["workers"]):
+        assert bool((u == v).all())
+    with pytest.raises(grawa.GrawaError) as e:
+        gpu_step(grawa, "lgrawa", p, g, 0.5, off, workspace=ws[:need - 256])
+    assert e.value.status == -4
+    with pytest.raises(grawa.GrawaError):
+        gpu_step(grawa, "lgrawa", p, g, 0.5, off, workspace=ws[1:need + 1])       # misaligned
+
+
+@pytest.mark.parametrize("tiles", [(1024, 1024), (4096, 16384), (65536, 2048)])
+def test_tile_options_do_not_change_the_result(grawa, tiles):
+    cfg = gen.CONFIGS["toy10"]
+    p, g = inputs("toy10")
+    old = grawa.grawa_get_option("sumsq_tile"), grawa.grawa_get_option("pull_tile")
+    try:
+        grawa.grawa_set_option("sumsq_tile", tiles[0])
+        grawa.grawa_set_option("pull_tile", tiles[1])
+        for variant in ("mgrawa", "lgrawa"):
+            res = gpu_step(grawa, variant, p, g, 0.5, cfg.offsets())
+            compare_with_oracle(res, variant, p, g, 0.5, cfg.offsets())
+    finally:
+        grawa.grawa_set_option("sumsq_tile", old[0])
+        grawa.grawa_set_option("pull_tile", old[1])
+
+
+@pytest.mark.parametrize("M", [1, 3, 4, 9])
+def test_prox_step_parity(grawa, M):
+    import torch
+    cfg = gen.custom_config([10, 5000, 3, 12001], M, seed=31)
+    p, _ = gen.make_inputs(cfg)
+    c = gen.make_inputs(gen.custom_config([cfg.n], 1, seed=32))[0][0]
+    for a in (0.05 / 16, 0.01 / 32, 0.0, 1.0):
+        x = to_device(p)
+        grawa.grawa_prox_step(x, torch.from_numpy(c).cuda(), a)
+        torch.cuda.synchronize()
+        ref = oracle.prox(p, c, a)
+        tol = 2e-6 * max(np.abs(q).max() for q in p + [c])
+        for m in range(M):
+            got = x[m].cpu().numpy()
+            assert np.abs(got - ref[m]).max() <= tol
+            if a == 0.0:
+                assert np.array_equal(got, p[m])
+            if a == 1.0:
+                assert np.array_equal(got, c)
+
+
+@pytest.mark.parametrize("variant", ["mgrawa", "lgrawa", "grawa"])
+def test_host_buffer_entry_point(grawa, variant):
+    import torch
+    cfg = gen.CONFIGS["resnet20_cifar"]
+    p, g = inputs("resnet20_cifar")
+    off = cfg.offsets()
+    hp = [torch.from_numpy(a.copy()).pin_memory() for a in p]
+    hg = [torch.from_numpy(a.copy()).pin_memory() for a in g]
+    hc = torch.empty(cfg.n, dtype=torch.float32).pin_memory()
+    grawa.grawa_step_host(variant, hp, hg, 0.5, off, hc)
+    dev = gpu_step(grawa, variant, p, g, 0.5, off)
+    assert np.array_equal(hc.numpy(), dev["center"].cpu().numpy())
+    for m in range(cfg.M):
+        assert np.array_equal(hp[m].numpy(), dev["workers"][m].cpu().numpy())
+        assert np.array_equal(hg[m].numpy(), g[m])
+    # pageable numpy buffers work too
+    np_p = [a.copy() for a in p]
+    np_c = np.empty(cfg.n, np.float32)
+    grawa.grawa_step_host(variant, np_p, g, 0.5, off, np_c)
+    assert np.array_equal(np_c, hc.numpy())
+
+
+def test_step_inside_a_cuda_graph(grawa):
+    """After one eager call has built the plan, a step allocates nothing and can be captured."""
+    import torch
+    cfg = gen.CONFIGS["resnet20_cifar"]
+    p, g = inputs("resnet20_cifar")
+    off = cfg.offsets()
+    stream = torch.cuda.Stream()
+    x, gr = to_device(p), to_device(g)
+    center = torch.empty(cfg.n, device="cuda")
+    with torch.cuda.stream(stream):
+        grawa.grawa_lgrawa_step(x, gr, 0.5, off, center)          # builds the plan for this stream
+        stream.synchronize()
+        for t, a in zip(x, p):
+            t.copy_(torch.from_numpy(a))
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            grawa.grawa_lgrawa_step(x, gr, 0.5, off, center, stream=torch.cuda.current_stream())
+    for t, a in zip(x, p):
+        t.copy_(torch.from_numpy(a))
+    torch.cuda.synchronize()
+    graph.replay()
+    torch.cuda.synchronize()
+    ref = gpu_step(grawa, "lgrawa", p, g, 0.5, off)
+    assert bool((center == ref["center"]).all())
+    for u, v in zip(x, ref["workers"]):
+        assert bool((u == v).all())
