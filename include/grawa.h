@@ -60,7 +60,8 @@ typedef enum grawa_status {
     GRAWA_ERR_CUDA = -2,        /* a CUDA runtime call failed; text in grawa_last_cuda_error()    */
     GRAWA_ERR_NONFINITE = -3,   /* a gradient score was NaN/Inf (fallback weights were applied)   */
     GRAWA_ERR_WORKSPACE = -4,   /* caller-supplied workspace missing, misaligned or too small     */
-    GRAWA_ERR_TIMEOUT = -5      /* a bounded device-side wait ran out (bulk-copy variant only)    */
+    GRAWA_ERR_TIMEOUT = -5,     /* a bounded device-side wait ran out (bulk-copy variant only)    */
+    GRAWA_ERR_TOO_LARGE = -6    /* problem larger than the built-in scratch of grawa_sumsq_static */
 } grawa_status;
 
 typedef enum grawa_variant { GRAWA_VARIANT_GRAWA = 0, GRAWA_VARIANT_MGRAWA = 1, GRAWA_VARIANT_LGRAWA = 2 } grawa_variant;
@@ -130,6 +131,41 @@ grawa_status grawa_last_step_status(grawa_stream_t stream);
  * mu_over_tau must lie in [0, 1]. */
 grawa_status grawa_prox_step(float *const *params, const float *center, int64_t n, int M,
                              float mu_over_tau, grawa_stream_t stream);
+
+/* Largest number of partial sums grawa_sumsq_static can hold: M * ceil(n / 16384) must not
+ * exceed it (for example M = 16 workers of up to 134 million elements each). */
+#define GRAWA_STATIC_MAX_PARTIALS 131072
+
+/* Squared gradient norms without any allocation (the paper has no counterpart of this entry
+ * point; it exists for the sake of callers, not of the method): sumsq_out[m] = sum_j grads[m][j]^2
+ * for m = 0..M-1, the quantity under the square root of Eq. 2.
+ *
+ * Who needs it: a host program whose device memory is already fully claimed by another
+ * allocator (a training framework's caching pool, a fixed partition handed out at start-up),
+ * where a raw cudaMalloc inside a library fails or fragments that pool; and a latency-bound
+ * loop that cannot afford the device-wide synchronisation cudaMalloc and cudaFree imply.  The
+ * step entry points above build a plan on their first call for a shape (device allocations);
+ * this one never calls cudaMalloc, cudaFree or any allocating routine, on any call.
+ *
+ * Its scratch for the per-tile partial sums is a fixed array of GRAWA_STATIC_MAX_PARTIALS
+ * doubles (1 MiB) compiled into the library; every GPU that loads the library holds that
+ * megabyte until the process exits.  grads: HOST array of M DEVICE pointers to n fp32 values
+ * (read only).  sumsq_out: DEVICE, M doubles, overwritten.  Same arithmetic as step 1 of the
+ * step entry points with tiles of 16384 elements: fp32 runs combined in fp64 in a fixed order,
+ * bitwise reproducible.
+ *
+ * Errors: GRAWA_ERR_INVALID_ARG for NULL pointers, M outside [1, GRAWA_MAX_WORKERS] or n < 0;
+ * GRAWA_ERR_TOO_LARGE when M * ceil(n / 16384) > GRAWA_STATIC_MAX_PARTIALS (nothing is
+ * enqueued); GRAWA_ERR_CUDA for a failed launch or address look-up.  n = 0 writes zeros.
+ *
+ * The first call on each device looks up the device address of the built-in array (the device
+ * must be current); make that first call outside any stream capture.  All calls on a device
+ * share the one array and it keeps the previous call's contents (every slot a call reads it
+ * has first overwritten, so nothing needs clearing): two calls whose kernels can overlap on
+ * the GPU, for instance on different streams without an ordering between them, race on it
+ * and give wrong sums.  Calls on one stream are safe. */
+grawa_status grawa_sumsq_static(const float *const *grads, int64_t n, int M, double *sumsq_out,
+                                grawa_stream_t stream);
 
 /* Tuning knobs, process wide; they change speed, never results beyond fp32 summation order
  * of the sums of squares ("sumsq_tile").  Returns GRAWA_ERR_INVALID_ARG for an unknown name

@@ -20,6 +20,7 @@ from .binding import (  # noqa: F401
     grawa_set_option,
     grawa_status_string,
     grawa_step_host,
+    grawa_sumsq_static,
     grawa_version,
     grawa_workspace_bytes,
     library,

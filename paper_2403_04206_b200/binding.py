@@ -67,6 +67,8 @@ def library() -> ctypes.CDLL:
     lib.grawa_get_option.restype = i64
     lib.grawa_launch_count.restype = i64
     lib.grawa_clear_plans.restype = None
+    lib.grawa_sumsq_static.argtypes = [vp, i64, ci, vp, vp]
+    lib.grawa_sumsq_static.restype = ci
     lib.grawa_collect_kernel_times.argtypes = [vp, vp, vp, vp]
     lib.grawa_collect_kernel_times.restype = ci
     _lib = lib
@@ -197,6 +199,19 @@ def grawa_prox_step(params, center, mu_over_tau, *, stream=None, n=None) -> None
         n = _numel(center)
     _raise(lib.grawa_prox_step(_ptr_array(params), _addr(center), n, M, float(mu_over_tau), _stream(stream)),
            "grawa_prox_step")
+
+
+def grawa_sumsq_static(grads, sumsq_out, *, stream=None, n=None) -> None:
+    """Squared gradient norms of the M workers into ``sumsq_out`` (device, M float64) using only
+    the scratch array built into the library: for callers whose device memory belongs to another
+    allocator, or who cannot afford the synchronisation an allocation implies.  Calls that may
+    overlap on the GPU share that array and race; keep them on one stream."""
+    _check_f32(list(grads))
+    M = len(grads)
+    if n is None:
+        n = _numel(grads[0]) if M else 0
+    _raise(library().grawa_sumsq_static(_ptr_array(grads), n, M, _addr(sumsq_out), _stream(stream)),
+           "grawa_sumsq_static")
 
 
 def grawa_workspace_bytes(n: int, M: int, layer_offsets=None) -> int:

@@ -331,6 +331,75 @@ static grawa_status step_entry(int variant, float* const* params, const float* c
     return enqueue_step(variant, params, grads, n, M, pull, off, center_out, opt, stream, plan);
 }
 
+// ------------------------------------------------------------------ allocation-free sum of squares
+// Scratch that lives in the library image instead of in an allocation: one array per GPU that
+// loads the library, held until the process exits.  In host code `g_static_partials` is only a
+// handle for cudaGetSymbolAddress; kernels are given the address that call returns.
+constexpr int kStaticTile = 16384;
+static_assert(kStaticTile % 4 == 0, "tiles must keep 16-byte alignment");
+static __device__ __align__(256) double g_static_partials[GRAWA_STATIC_MAX_PARTIALS];
+
+constexpr int kMaxDevices = 64;
+static double* g_static_partials_addr[kMaxDevices] = {};   // per device, filled on first use
+
+// Variant of sumsq_kernel for one flat layer: items are (worker, tile of `tile` elements) found
+// by arithmetic, so no work list has to exist in device memory.
+template <int UNROLL>
+__global__ void __launch_bounds__(kThreads)
+sumsq_flat_kernel(ConstPtrs grads, long long n, int tiles, int tile, double* __restrict__ partials, int vec_ok)
+{
+    const int item = blockIdx.x;
+    const int m = item / tiles;
+    const int t = item - m * tiles;
+    const float* __restrict__ g = grads.p[m];
+    const long long b = static_cast<long long>(t) * tile, e = min(n, b + tile);
+    const int tid = threadIdx.x;
+    long long hb, te;
+    split_range(b, e, vec_ok, hb, te);
+    double dacc = 0.0;
+    const float4* __restrict__ g4 = reinterpret_cast<const float4*>(g + hb);
+    const int ncol = static_cast<int>((te - hb) >> 2);
+    for (int c0 = 0; c0 < ncol; c0 += kThreads * UNROLL) {
+        float4 v[UNROLL];
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            const int c = c0 + u * kThreads + tid;
+            v[u] = (c < ncol) ? ld_stream4(g4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+        }
+        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+#pragma unroll
+        for (int u = 0; u < UNROLL; ++u) {
+            a0 = fmaf(v[u].x, v[u].x, a0);
+            a1 = fmaf(v[u].y, v[u].y, a1);
+            a2 = fmaf(v[u].z, v[u].z, a2);
+            a3 = fmaf(v[u].w, v[u].w, a3);
+        }
+        dacc += (static_cast<double>(a0) + static_cast<double>(a1)) +
+                (static_cast<double>(a2) + static_cast<double>(a3));
+    }
+    for (long long i = b + tid; i < hb; i += kThreads) {
+        const double v = static_cast<double>(ld_stream1(g + i));
+        dacc += v * v;
+    }
+    for (long long i = te + tid; i < e; i += kThreads) {
+        const double v = static_cast<double>(ld_stream1(g + i));
+        dacc += v * v;
+    }
+    const double total = block_sum_fixed_order<kThreads>(dacc);
+    if (tid == 0) partials[static_cast<size_t>(m) * tiles + t] = total;
+}
+
+// One CTA per worker adds that worker's `tiles` partial sums in a fixed order.
+__global__ void __launch_bounds__(kFinalizeThreads)
+sum_partials_kernel(const double* __restrict__ partials, int tiles, double* __restrict__ out)
+{
+    const double* __restrict__ row = partials + static_cast<size_t>(blockIdx.x) * tiles;
+    double acc = 0.0;
+    for (int s = threadIdx.x; s < tiles; s += kFinalizeThreads) acc += row[s];
+    const double total = block_sum_fixed_order<kFinalizeThreads>(acc);
+    if (threadIdx.x == 0) out[blockIdx.x] = total;
+}
+
 }  // namespace grawa
 
 using namespace grawa;
@@ -348,6 +417,7 @@ const char* grawa_status_string(grawa_status status)
         case GRAWA_ERR_NONFINITE: return "non-finite gradient score";
         case GRAWA_ERR_WORKSPACE: return "workspace missing, misaligned or too small";
         case GRAWA_ERR_TIMEOUT: return "bounded device wait ran out";
+        case GRAWA_ERR_TOO_LARGE: return "problem exceeds the built-in scratch (GRAWA_STATIC_MAX_PARTIALS)";
     }
     return "unknown status";
 }
@@ -466,6 +536,46 @@ grawa_status grawa_prox_step(float* const* params, const float* center, int64_t 
     const int64_t tiles = (n + tile - 1) / tile;
     if (tiles > 0x7fffffffll) return GRAWA_ERR_INVALID_ARG;
     prox_kernel<<<static_cast<int>(tiles), kThreads, 0, stream>>>(xp, center, n, static_cast<int>(tile), mu_over_tau, M, vec ? 1 : 0);
+    ++g_launches;
+    GRAWA_CUDA_TRY(cudaGetLastError());
+    return GRAWA_OK;
+}
+
+grawa_status grawa_sumsq_static(const float* const* grads, int64_t n, int M, double* sumsq_out, grawa_stream_t stream)
+{
+    if (grads == nullptr || sumsq_out == nullptr || M < 1 || M > GRAWA_MAX_WORKERS || n < 0) return GRAWA_ERR_INVALID_ARG;
+    ConstPtrs gp{};
+    bool vec = true;
+    for (int m = 0; m < M; ++m) {
+        if (n > 0 && (grads[m] == nullptr || (reinterpret_cast<uintptr_t>(grads[m]) & 3u))) return GRAWA_ERR_INVALID_ARG;
+        gp.p[m] = grads[m];
+        vec = vec && aligned16(grads[m]);
+    }
+    const int64_t tiles64 = (n + kStaticTile - 1) / kStaticTile;
+    if (tiles64 * M > GRAWA_STATIC_MAX_PARTIALS) return GRAWA_ERR_TOO_LARGE;
+    const int tiles = static_cast<int>(tiles64);
+
+    // Once per device, with that device current: the device address of the built-in array.
+    int device = 0;
+    GRAWA_CUDA_TRY(cudaGetDevice(&device));
+    if (device < 0 || device >= kMaxDevices) return GRAWA_ERR_INVALID_ARG;
+    double* partials = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (g_static_partials_addr[device] == nullptr) {
+            double* addr = nullptr;
+            GRAWA_CUDA_TRY(cudaGetSymbolAddress(reinterpret_cast<void**>(&addr), g_static_partials));
+            g_static_partials_addr[device] = addr;
+        }
+        partials = g_static_partials_addr[device];
+    }
+    if (tiles > 0) {
+        sumsq_flat_kernel<8><<<tiles * M, kThreads, 0, stream>>>(gp, n, tiles, kStaticTile, partials, vec ? 1 : 0);
+        ++g_launches;
+        GRAWA_CUDA_TRY(cudaGetLastError());
+    }
+    // with tiles == 0 every row is empty and the sums are written as zeros
+    sum_partials_kernel<<<M, kFinalizeThreads, 0, stream>>>(partials, tiles, sumsq_out);
     ++g_launches;
     GRAWA_CUDA_TRY(cudaGetLastError());
     return GRAWA_OK;
