@@ -172,12 +172,22 @@ grawa_status grawa_sumsq_static(const float *const *grads, int64_t n, int M, dou
  * or a value out of range.
  *   "sumsq_tile"   elements per sum-of-squares work item (multiple of 1024, 1024..1048576)
  *   "pull_tile"    elements per centre+pull work item (multiple of 1024, 1024..1048576)
- *   "pull_variant" 0 = automatic, 1 = register kernel (vector loads), 2 = bulk-copy kernel
- *                  (shared-memory staging by 1-D bulk asynchronous copies)
+ *   "pull_variant" 0 = automatic (register kernel up to 16 workers, bulk-copy kernel above),
+ *                  1 = register kernel (vector loads), 2 = bulk-copy kernel (shared-memory
+ *                  staging by 1-D bulk asynchronous copies and bulk stores)
+ *   "bulk_tile"    elements per slice of a bulk-copy stage (multiple of 256, up to 16384);
+ *                  0 = chosen from M so that three stages fit in shared memory
  *   "kernel_timing" 1 = every device-buffer step also records CUDA events around its three
  *                  phases on the step's stream (see grawa_collect_kernel_times); do not use
  *                  while capturing a CUDA graph.  Default 0.
- * Changing a tile size drops the cached plans. */
+ *   "dependent_launch" 1 (default) = the kernels of a step are launched with programmatic
+ *                  stream serialisation, so each one's launch overlaps the tail of the one
+ *                  before it on the stream (it still waits for that kernel's results);
+ *                  0 = plain stream order.
+ *   "sumsq_ctas_per_sm", "pull_ctas_per_sm" (0..32) CTAs per SM of the grid that streams
+ *                  through the work items of the sum-of-squares / centre+pull kernel;
+ *                  0 = one CTA per work item.
+ * Changing a tile size or the variant drops the cached plans. */
 grawa_status grawa_set_option(const char *name, int64_t value);
 
 /* Current value of a tuning knob, or -1 for an unknown name. */

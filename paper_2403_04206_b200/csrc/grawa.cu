@@ -15,6 +15,7 @@
 #include <vector>
 
 #include "kernels.cuh"
+#include "center_pull_bulk.cuh"
 
 namespace grawa {
 
@@ -26,7 +27,11 @@ static std::atomic<int64_t> g_launches{0};
 static int64_t g_sumsq_tile = 8192;
 static int64_t g_pull_tile = 4096;
 static int64_t g_pull_variant = 0;
+static int64_t g_bulk_tile = 0;           // 0 = chosen from M so that at least three stages fit
 static int64_t g_kernel_timing = 0;
+static int64_t g_pdl = 1;
+static int64_t g_sumsq_ctas_per_sm = 0;   // 0 = one CTA per work item
+static int64_t g_pull_ctas_per_sm = 0;    // 0 = one CTA per work item
 static thread_local std::string t_cuda_error;
 
 static grawa_status cuda_fail(cudaError_t err, const char* what)
@@ -44,6 +49,21 @@ static grawa_status cuda_fail(cudaError_t err, const char* what)
     } while (0)
 
 static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Dynamic shared memory the bulk-copy centre+pull kernel may use (one CTA per SM).
+constexpr size_t kBulkSmemBudget = 200 * 1024;
+
+// Does the centre+pull of an M-worker problem take the bulk-copy kernel?
+static bool wants_bulk(int M) { return g_pull_variant == 2 || (g_pull_variant == 0 && M > kMaxRegWorkers); }
+
+// Elements per slice of a bulk-copy stage: the option, or the largest multiple of 256 up to 4096
+// that leaves room for three stages of M+1 slices.
+static int64_t bulk_tile_for(int M)
+{
+    if (g_bulk_tile > 0) return g_bulk_tile;
+    const int64_t fit = static_cast<int64_t>(kBulkSmemBudget / (3 * sizeof(float) * (static_cast<size_t>(M) + 1)));
+    return std::max<int64_t>(256, std::min<int64_t>(4096, fit / 256 * 256));
+}
 
 // ------------------------------------------------------------------ work list
 // Cuts every non-empty layer at the absolute multiples of `tile` that fall inside it.
@@ -87,9 +107,9 @@ static WorkspaceLayout workspace_layout(int64_t C1, int K, int M)
     size_t p = 0;
     w.partials = p; p = align_up(p + sizeof(double) * static_cast<size_t>(C1) * M, 256);
     w.S = p;        p = align_up(p + sizeof(double) * static_cast<size_t>(K) * M, 256);
-    w.A = p;        p = align_up(p + sizeof(double) * static_cast<size_t>(K) * M, 256);
+    w.A = p;        p = align_up(p + sizeof(double) * (static_cast<size_t>(K) + 1) * M, 256);   // K rows of terms + scores
     w.beta = p;     p = align_up(p + sizeof(float) * static_cast<size_t>(K) * M, 256);
-    w.words = p;    p = align_up(p + 256, 256);   // [0] ticket (unsigned), [1] status (int)
+    w.words = p;    p = align_up(p + 256, 256);   // [0] ticket (unsigned), [1] status (int), [2] work counter (unsigned)
     w.total = p;
     return w;
 }
@@ -108,6 +128,8 @@ struct Plan {
     void* d_ws = nullptr;            // owned scratch (used when the caller passes none)
     WorkspaceLayout ws{};
     float* d_stage = nullptr;        // owned staging for the host-buffer entry point
+    int sm_count = 148;
+    bool bulk = false;               // centre+pull items are cut for the bulk-copy kernel
     ~Plan()
     {
         cudaFree(d_segs1); cudaFree(d_segs2); cudaFree(d_layer_first); cudaFree(d_ws); cudaFree(d_stage);
@@ -146,7 +168,9 @@ static grawa_status get_plan(int64_t n, int M, const std::vector<int64_t>& off, 
     std::unique_ptr<Plan> p(new Plan);
     p->device = device; p->stream = stream; p->n = n; p->M = M; p->off = off;
     p->K = static_cast<int>(off.size()) - 1;
-    p->tile1 = g_sumsq_tile; p->tile2 = g_pull_tile;
+    p->bulk = wants_bulk(M);
+    p->tile1 = g_sumsq_tile; p->tile2 = p->bulk ? bulk_tile_for(M) : g_pull_tile;
+    GRAWA_CUDA_TRY(cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, device));
     std::vector<Segment> s1, s2;
     std::vector<int> first;
     build_segments(off, p->tile1, &s1, &first);
@@ -212,26 +236,88 @@ static grawa_status validate(float* const* params, const float* const* grads, in
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // ------------------------------------------------------------------ launches
-template <int M>
-static void launch_center_pull(bool per_layer, int grid, cudaStream_t stream, const MutPtrs& x, float* center,
-                               const float* beta, const Segment* segs, long long n, int tile, float pull)
+// One launch, optionally with programmatic stream serialisation (the kernel may start launching
+// while its predecessor on the stream drains; it waits for it in grid_dependency_sync()).
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_kernel_smem(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t stream, bool pdl,
+                                      Args&&... args)
 {
-    if (per_layer) center_pull_kernel<M, true><<<grid, kThreads, 0, stream>>>(x, center, beta, segs, n, tile, pull, 1);
-    else center_pull_kernel<M, false><<<grid, kThreads, 0, stream>>>(x, center, beta, segs, n, tile, pull, 1);
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(static_cast<unsigned>(grid));
+    cfg.blockDim = dim3(static_cast<unsigned>(block));
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = pdl ? 1 : 0;
+    ++g_launches;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+template <typename... KArgs, typename... Args>
+static cudaError_t launch_kernel(void (*kernel)(KArgs...), int grid, int block, cudaStream_t stream, bool pdl, Args&&... args)
+{
+    return launch_kernel_smem(kernel, grid, block, 0, stream, pdl, static_cast<Args&&>(args)...);
+}
+
+// Bulk-copy centre+pull: MT = M for 2..16 (register column), MT = 0 for larger M.
+
+template <int MT>
+static cudaError_t launch_center_pull_bulk(bool per_layer, int grid, int items, size_t smem, cudaStream_t stream, bool pdl,
+                                           const MutPtrs& x, float* center, const float* beta, const Segment* segs, long long n,
+                                           int tile, int stages, int M, float pull, unsigned* counter, int* status)
+{
+    auto kernel = per_layer ? center_pull_bulk_kernel<MT, true> : center_pull_bulk_kernel<MT, false>;
+    cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kBulkSmemBudget));
+    if (err != cudaSuccess) return err;
+    return launch_kernel_smem(kernel, grid, kThreads, smem, stream, pdl, x, center, beta, segs, items, n, tile, stages, M, pull,
+                              counter, status);
+}
+
+template <int MT>
+struct CenterPullBulkDispatch {
+    template <typename... A>
+    static cudaError_t run(int m, A&&... a)
+    {
+        if (m == MT) return launch_center_pull_bulk<MT>(static_cast<A&&>(a)...);
+        return CenterPullBulkDispatch<MT - 1>::run(m, static_cast<A&&>(a)...);
+    }
+};
+template <>
+struct CenterPullBulkDispatch<1> {
+    template <typename... A>
+    static cudaError_t run(int, A&&... a)
+    {
+        return launch_center_pull_bulk<0>(static_cast<A&&>(a)...);
+    }
+};
+
+template <int M>
+static cudaError_t launch_center_pull(bool per_layer, int grid, int items, cudaStream_t stream, bool pdl, const MutPtrs& x,
+                                      float* center, const float* beta, const Segment* segs, long long n, int tile, float pull)
+{
+    if (per_layer) return launch_kernel(center_pull_kernel<M, true>, grid, kThreads, stream, pdl, x, center, beta, segs, items, n, tile, pull, 1);
+    return launch_kernel(center_pull_kernel<M, false>, grid, kThreads, stream, pdl, x, center, beta, segs, items, n, tile, pull, 1);
 }
 
 template <int M>
 struct CenterPullDispatch {
-    static void run(int m, bool per_layer, int grid, cudaStream_t stream, const MutPtrs& x, float* center,
-                    const float* beta, const Segment* segs, long long n, int tile, float pull)
+    static cudaError_t run(int m, bool per_layer, int grid, int items, cudaStream_t stream, bool pdl, const MutPtrs& x,
+                           float* center, const float* beta, const Segment* segs, long long n, int tile, float pull)
     {
-        if (m == M) launch_center_pull<M>(per_layer, grid, stream, x, center, beta, segs, n, tile, pull);
-        else CenterPullDispatch<M - 1>::run(m, per_layer, grid, stream, x, center, beta, segs, n, tile, pull);
+        if (m == M) return launch_center_pull<M>(per_layer, grid, items, stream, pdl, x, center, beta, segs, n, tile, pull);
+        return CenterPullDispatch<M - 1>::run(m, per_layer, grid, items, stream, pdl, x, center, beta, segs, n, tile, pull);
     }
 };
 template <>
 struct CenterPullDispatch<1> {
-    static void run(int, bool, int, cudaStream_t, const MutPtrs&, float*, const float*, const Segment*, long long, int, float) {}
+    static cudaError_t run(int, bool, int, int, cudaStream_t, bool, const MutPtrs&, float*, const float*, const Segment*,
+                           long long, int, float)
+    {
+        return cudaErrorInvalidValue;
+    }
 };
 
 static grawa_status enqueue_step(int variant, float* const* params, const float* const* grads, int64_t n, int M,
@@ -275,26 +361,25 @@ static grawa_status enqueue_step(int variant, float* const* params, const float*
         ts = &g_timed_pool[g_timed_used++];
         GRAWA_CUDA_TRY(cudaEventRecord(ts->e[0], stream));
     }
+    const bool pdl = g_pdl != 0 && ts == nullptr;   // event records between the kernels need plain ordering
     // step 1: partial sums of squares, one CTA per (worker, item)
-    sumsq_kernel<8><<<plan->C1 * M, kThreads, 0, stream>>>(gp, plan->d_segs1, plan->C1, partials, vec_g ? 1 : 0, ticket, status);
-    ++g_launches;
-    GRAWA_CUDA_TRY(cudaGetLastError());
+    const int items1 = plan->C1 * M;
+    const int grid1 = g_sumsq_ctas_per_sm > 0
+                          ? static_cast<int>(std::min<int64_t>(items1, g_sumsq_ctas_per_sm * plan->sm_count)) : items1;
+    GRAWA_CUDA_TRY(launch_kernel(sumsq_kernel<8>, grid1, kThreads, stream, pdl, gp, plan->d_segs1, plan->C1, items1, partials,
+                                 vec_g ? 1 : 0, ticket, status, ticket + 2));
     if (ts) GRAWA_CUDA_TRY(cudaEventRecord(ts->e[1], stream));
     // steps 1b-3: S, scores, weights
-    finalize_kernel<<<K * M, kFinalizeThreads, 0, stream>>>(partials, plan->d_layer_first, plan->C1, K, M, variant, S, A, beta,
-                                                           ticket, status, opt ? opt->weights_out : nullptr,
-                                                           opt ? opt->scores_out : nullptr, opt ? opt->sumsq_out : nullptr);
-    ++g_launches;
-    GRAWA_CUDA_TRY(cudaGetLastError());
+    GRAWA_CUDA_TRY(launch_kernel(finalize_kernel, K, kFinalizeThreads, stream, pdl, partials, plan->d_layer_first, plan->C1, K, M,
+                                 variant, S, A, beta, ticket, status, opt ? opt->weights_out : nullptr,
+                                 opt ? opt->scores_out : nullptr, opt ? opt->sumsq_out : nullptr));
     if (ts) GRAWA_CUDA_TRY(cudaEventRecord(ts->e[2], stream));
     // steps 4-5
     if (M == 1) {
         if (center_out) {
             const bool v = aligned16(center_out) && aligned16(params[0]);
             const int grid = static_cast<int>(std::min<int64_t>((n + kThreads * 4 - 1) / (kThreads * 4), 148 * 16));
-            copy_kernel<<<grid, kThreads, 0, stream>>>(params[0], center_out, n, v ? 1 : 0);
-            ++g_launches;
-            GRAWA_CUDA_TRY(cudaGetLastError());
+            GRAWA_CUDA_TRY(launch_kernel(copy_kernel, grid, kThreads, stream, pdl, params[0], center_out, n, v ? 1 : 0));
         }
         if (ts) GRAWA_CUDA_TRY(cudaEventRecord(ts->e[3], stream));
         return GRAWA_OK;
@@ -303,15 +388,24 @@ static grawa_status enqueue_step(int variant, float* const* params, const float*
     const int64_t tiles = per_layer ? plan->C2 : (n + plan->tile2 - 1) / plan->tile2;
     if (tiles > 0x7fffffffll) return GRAWA_ERR_INVALID_ARG;
     const int grid = static_cast<int>(tiles);
-    if (vec_x && M <= kMaxRegWorkers) {
-        CenterPullDispatch<kMaxRegWorkers>::run(M, per_layer, grid, stream, xp, center_out, beta, plan->d_segs2, n,
-                                                static_cast<int>(plan->tile2), pull);
+    // bulk-copy variant: asked for explicitly, or the only vector path for M > 16
+    const size_t stage_bytes = sizeof(float) * static_cast<size_t>(plan->tile2) * (M + 1);
+    const int stages = static_cast<int>(std::min<size_t>(kBulkMaxStages, kBulkSmemBudget / stage_bytes));
+    if (vec_x && plan->bulk && stages >= 2) {
+        const int gridb = static_cast<int>(std::min<int64_t>(grid, plan->sm_count));
+        GRAWA_CUDA_TRY(CenterPullBulkDispatch<kMaxRegWorkers>::run(M <= kMaxRegWorkers ? M : 1, per_layer, gridb, grid,
+                                                                   stage_bytes * stages, stream, pdl, xp, center_out, beta,
+                                                                   plan->d_segs2, n, static_cast<int>(plan->tile2), stages, M, pull,
+                                                                   ticket + 2, status));
+    } else if (vec_x && M <= kMaxRegWorkers) {
+        const int grid2 = g_pull_ctas_per_sm > 0
+                              ? static_cast<int>(std::min<int64_t>(grid, g_pull_ctas_per_sm * plan->sm_count)) : grid;
+        GRAWA_CUDA_TRY(CenterPullDispatch<kMaxRegWorkers>::run(M, per_layer, grid2, grid, stream, pdl, xp, center_out, beta,
+                                                               plan->d_segs2, n, static_cast<int>(plan->tile2), pull));
     } else {
-        center_pull_generic_kernel<<<grid, kThreads, 0, stream>>>(xp, center_out, beta, plan->d_segs2, per_layer ? 1 : 0, n,
-                                                                 static_cast<int>(plan->tile2), pull, M);
+        GRAWA_CUDA_TRY(launch_kernel(center_pull_generic_kernel, grid, kThreads, stream, pdl, xp, center_out, beta, plan->d_segs2,
+                                     per_layer ? 1 : 0, n, static_cast<int>(plan->tile2), pull, M));
     }
-    ++g_launches;
-    GRAWA_CUDA_TRY(cudaGetLastError());
     if (ts) GRAWA_CUDA_TRY(cudaEventRecord(ts->e[3], stream));
     return GRAWA_OK;
 }
@@ -605,12 +699,27 @@ grawa_status grawa_set_option(const char* name, int64_t value)
     }
     if (std::strcmp(name, "pull_variant") == 0) {
         if (value < 0 || value > 2) return GRAWA_ERR_INVALID_ARG;
-        g_pull_variant = value;
+        if (value != g_pull_variant) { g_pull_variant = value; clear_plans_locked(); }
+        return GRAWA_OK;
+    }
+    if (std::strcmp(name, "bulk_tile") == 0) {
+        if (value < 0 || value > 16384 || value % 256 != 0) return GRAWA_ERR_INVALID_ARG;
+        if (value != g_bulk_tile) { g_bulk_tile = value; clear_plans_locked(); }
         return GRAWA_OK;
     }
     if (std::strcmp(name, "kernel_timing") == 0) {
         if (value < 0 || value > 1) return GRAWA_ERR_INVALID_ARG;
         g_kernel_timing = value;
+        return GRAWA_OK;
+    }
+    if (std::strcmp(name, "dependent_launch") == 0) {
+        if (value < 0 || value > 1) return GRAWA_ERR_INVALID_ARG;
+        g_pdl = value;
+        return GRAWA_OK;
+    }
+    if (std::strcmp(name, "sumsq_ctas_per_sm") == 0 || std::strcmp(name, "pull_ctas_per_sm") == 0) {
+        if (value < 0 || value > 32) return GRAWA_ERR_INVALID_ARG;
+        (name[0] == 's' ? g_sumsq_ctas_per_sm : g_pull_ctas_per_sm) = value;
         return GRAWA_OK;
     }
     return GRAWA_ERR_INVALID_ARG;
@@ -623,7 +732,11 @@ int64_t grawa_get_option(const char* name)
     if (std::strcmp(name, "sumsq_tile") == 0) return g_sumsq_tile;
     if (std::strcmp(name, "pull_tile") == 0) return g_pull_tile;
     if (std::strcmp(name, "pull_variant") == 0) return g_pull_variant;
+    if (std::strcmp(name, "bulk_tile") == 0) return g_bulk_tile;
     if (std::strcmp(name, "kernel_timing") == 0) return g_kernel_timing;
+    if (std::strcmp(name, "dependent_launch") == 0) return g_pdl;
+    if (std::strcmp(name, "sumsq_ctas_per_sm") == 0) return g_sumsq_ctas_per_sm;
+    if (std::strcmp(name, "pull_ctas_per_sm") == 0) return g_pull_ctas_per_sm;
     return -1;
 }
 

@@ -9,7 +9,8 @@ namespace grawa {
 
 constexpr int kMaxWorkers = 64;
 constexpr int kThreads = 256;          // threads per CTA of the streaming kernels
-constexpr int kFinalizeThreads = 128;
+constexpr int kFinalizeThreads = 256;
+constexpr int kStageDoubles = 2048;    // shared-memory staging of the finalisation (16 KB)
 constexpr int kMaxRegWorkers = 16;     // largest M the register-resident centre+pull kernel is built for
 
 enum Variant { kGrawa = 0, kMgrawa = 1, kLgrawa = 2 };
@@ -26,6 +27,18 @@ struct Segment {
     int len;
     int layer;
 };
+
+// Programmatic dependent launch: every kernel first waits until the grids it depends on have
+// completed and their writes are visible, then lets its own dependents start launching.  The
+// dependents wait the same way, so only launch latency and CTA ramp-up overlap, never data.
+// Both instructions do nothing in a kernel launched without the attribute.
+__device__ __forceinline__ void grid_dependency_sync()
+{
+#ifndef GRAWA_NO_GRIDDEP
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+#endif
+}
 
 // Streaming accesses: every byte is touched once per step, so keep it out of the way in L1/L2.
 __device__ __forceinline__ float4 ld_stream4(const float4* p) { return __ldcs(p); }
@@ -66,156 +79,202 @@ __device__ __forceinline__ double block_sum_fixed_order(double v)
 }
 
 // ---------------------------------------------------------------------------------------------
-// Step 1 (Eq. 3 / Eq. 5): partial[m][s] = sum of g_m[j]^2 over segment s.  One CTA per
-// (worker, segment).  fp32 squares are accumulated in runs of UNROLL terms per accumulator and
-// the runs are combined in fp64, in an order fixed by the launch shape only.
-// CTA 0 also clears the ticket and status words for the finalisation that follows on the stream.
+// Step 1 (Eq. 3 / Eq. 5): partial[m][s] = sum of g_m[j]^2 over segment s.  Work items are the
+// (worker, segment) pairs, worker-major; CTA b takes items b, b + gridDim.x, ... (a grid of a few
+// CTAs per SM streams through the list; a grid of `items` CTAs gives one item each).  fp32
+// squares are accumulated in runs of UNROLL terms per accumulator and the runs are combined in
+// fp64; the order depends only on the item, never on the grid, so results are reproducible.
+// CTA 0 also clears the ticket, status and work-counter words for the kernels that follow on the stream.
 // ---------------------------------------------------------------------------------------------
 template <int UNROLL>
 __global__ void __launch_bounds__(kThreads)
-sumsq_kernel(ConstPtrs grads, const Segment* __restrict__ segs, int C, double* __restrict__ partials,
-             int vec_ok, unsigned* __restrict__ ticket, int* __restrict__ status)
+sumsq_kernel(ConstPtrs grads, const Segment* __restrict__ segs, int C, int items, double* __restrict__ partials,
+             int vec_ok, unsigned* __restrict__ ticket, int* __restrict__ status, unsigned* __restrict__ work_counter)
 {
-    const int item = blockIdx.x;
-    const int m = item / C;
-    const int s = item - m * C;
-    const Segment sg = segs[s];
-    const float* __restrict__ g = grads.p[m];
-    const long long b = sg.begin, e = b + sg.len;
-    const int tid = threadIdx.x;
-    if (item == 0 && tid == 0) { *ticket = 0u; *status = 0; }
+    grid_dependency_sync();
+    __shared__ double warp_part[2][kThreads / 32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (blockIdx.x == 0 && tid == 0) { *ticket = 0u; *status = 0; *work_counter = 0u; }
 
-    long long hb, te;
-    split_range(b, e, vec_ok, hb, te);
-    double dacc = 0.0;
+    int parity = 0;
+    for (int item = blockIdx.x; item < items; item += gridDim.x, parity ^= 1) {
+        const int m = item / C;
+        const int s = item - m * C;
+        const Segment sg = segs[s];
+        const float* __restrict__ g = grads.p[m];
+        const long long b = sg.begin, e = b + sg.len;
+        long long hb, te;
+        split_range(b, e, vec_ok, hb, te);
+        double dacc = 0.0;
 
-    const float4* __restrict__ g4 = reinterpret_cast<const float4*>(g + hb);
-    const int ncol = static_cast<int>((te - hb) >> 2);
-    for (int c0 = 0; c0 < ncol; c0 += kThreads * UNROLL) {
-        float4 v[UNROLL];
+        const float4* __restrict__ g4 = reinterpret_cast<const float4*>(g + hb);
+        const int ncol = static_cast<int>((te - hb) >> 2);
+        for (int c0 = 0; c0 < ncol; c0 += kThreads * UNROLL) {
+            float4 v[UNROLL];
 #pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-            const int c = c0 + u * kThreads + tid;
-            v[u] = (c < ncol) ? ld_stream4(g4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
-        }
-        float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
+            for (int u = 0; u < UNROLL; ++u) {
+                const int c = c0 + u * kThreads + tid;
+                v[u] = (c < ncol) ? ld_stream4(g4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+            float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
-        for (int u = 0; u < UNROLL; ++u) {
-            a0 = fmaf(v[u].x, v[u].x, a0);
-            a1 = fmaf(v[u].y, v[u].y, a1);
-            a2 = fmaf(v[u].z, v[u].z, a2);
-            a3 = fmaf(v[u].w, v[u].w, a3);
+            for (int u = 0; u < UNROLL; ++u) {
+                a0 = fmaf(v[u].x, v[u].x, a0);
+                a1 = fmaf(v[u].y, v[u].y, a1);
+                a2 = fmaf(v[u].z, v[u].z, a2);
+                a3 = fmaf(v[u].w, v[u].w, a3);
+            }
+            dacc += (static_cast<double>(a0) + static_cast<double>(a1)) +
+                    (static_cast<double>(a2) + static_cast<double>(a3));
         }
-        dacc += (static_cast<double>(a0) + static_cast<double>(a1)) +
-                (static_cast<double>(a2) + static_cast<double>(a3));
+        for (long long i = b + tid; i < hb; i += kThreads) {
+            const double v = static_cast<double>(ld_stream1(g + i));
+            dacc += v * v;
+        }
+        for (long long i = te + tid; i < e; i += kThreads) {
+            const double v = static_cast<double>(ld_stream1(g + i));
+            dacc += v * v;
+        }
+        // Fixed-order block sum.  Two alternating buffers need only one barrier per item: a warp
+        // can write buffer p again only after the barrier of the item in between, which thread 0
+        // reaches after it has read buffer p.
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) dacc += __shfl_down_sync(0xffffffffu, dacc, d);
+        if (lane == 0) warp_part[parity][warp] = dacc;
+        __syncthreads();
+        if (tid == 0) {
+            double total = 0.0;
+#pragma unroll
+            for (int w = 0; w < kThreads / 32; ++w) total += warp_part[parity][w];
+            partials[static_cast<size_t>(m) * C + s] = total;
+        }
     }
-    for (long long i = b + tid; i < hb; i += kThreads) {
-        const double v = static_cast<double>(ld_stream1(g + i));
-        dacc += v * v;
-    }
-    for (long long i = te + tid; i < e; i += kThreads) {
-        const double v = static_cast<double>(ld_stream1(g + i));
-        dacc += v * v;
-    }
-    const double total = block_sum_fixed_order<kThreads>(dacc);
-    if (tid == 0) partials[static_cast<size_t>(m) * C + s] = total;
 }
 
 // Step 3 for one group of M scores (Eq. 2 / 4 / 7) with the zero-score limit and the non-finite
-// fallback.  A has stride 1.  Returns 1 if a non-finite score was met.
-__device__ inline int weights_group(const double* A, int M, float* beta, float* beta_copy)
+// fallback, computed by the whole CTA: thread m < M passes its score `a` and gets beta_m back.
+// The reciprocals are taken in parallel and added by one thread in worker order, so the value is
+// the one a sequential loop over m = 0..M-1 gives.  Every thread of the CTA must call it.
+struct WeightsSmem {
+    double r[kMaxWorkers];
+    double z;
+};
+
+__device__ __forceinline__ float weights_parallel(double a, int M, WeightsSmem& sm, int& flagged)
 {
-    int zeros = 0, finite = 0, flagged = 0;
-    for (int m = 0; m < M; ++m) {
-        const double a = A[m];
-        if (!isfinite(a)) flagged = 1;
-        else { ++finite; if (a == 0.0) ++zeros; }
+    const int tid = threadIdx.x;
+    const bool active = tid < M;
+    const bool fin = active && isfinite(a);
+    const bool zero = fin && a == 0.0;
+    const int finite = __syncthreads_count(fin);
+    const int zeros = __syncthreads_count(zero);
+    if (active) sm.r[tid] = (fin && !zero) ? 1.0 / a : 0.0;
+    __syncthreads();
+    if (tid == 0) {
+        double z = 0.0;
+        for (int m = 0; m < M; ++m) z += sm.r[m];     // adding the 0.0 of a skipped worker is exact
+        sm.z = z;
     }
-    double z = 0.0;
-    if (finite > 0 && zeros == 0)
-        for (int m = 0; m < M; ++m)
-            if (isfinite(A[m])) z += 1.0 / A[m];
-    for (int m = 0; m < M; ++m) {
-        const double a = A[m];
-        double w;
+    __syncthreads();
+    flagged = finite < M;
+    double w = 0.0;
+    if (active) {
         if (finite == 0) w = 1.0 / M;
-        else if (zeros > 0) w = (isfinite(a) && a == 0.0) ? 1.0 / zeros : 0.0;
-        else w = isfinite(a) ? (1.0 / a) / z : 0.0;
-        const float wf = static_cast<float>(w);
-        beta[m] = wf;
-        if (beta_copy) beta_copy[m] = wf;
+        else if (zeros > 0) w = zero ? 1.0 / zeros : 0.0;
+        else w = fin ? sm.r[tid] / sm.z : 0.0;
     }
-    return flagged;
+    return static_cast<float>(w);
 }
 
 // ---------------------------------------------------------------------------------------------
-// Steps 1b-3: one CTA per (layer, worker) adds that pair's partials in a fixed order into
-// S[k][m]; the CTA that takes the last ticket then turns S into scores and weights.
-// No CTA waits for another: the last arrival is found with one atomic ticket.
+// Steps 1b-3: one CTA per layer.  Warp w adds the partials of workers w, w+8, ... of that layer
+// in a fixed order into S[k][m]; the layer's terms sqrt(S) (S itself for the flat norm) go to row k
+// of A.  LGRAWA: the same CTA turns them into the layer's weights (Eq. 7).  MGRAWA / GRAWA: the
+// CTA that draws the last ticket adds the K rows per worker in layer order (Eq. 3 / Eq. 2), writes
+// the scores to row K of A and computes the M weights (Eq. 4).  No CTA waits for another.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(kFinalizeThreads)
 finalize_kernel(const double* __restrict__ partials, const int* __restrict__ layer_seg_first, int C, int K, int M,
                 int variant, double* S, double* A, float* beta, unsigned* ticket, int* status,
                 float* weights_out, double* scores_out, double* sumsq_out)
 {
-    const int k = blockIdx.x / M;
-    const int m = blockIdx.x - k * M;
-    const int tid = threadIdx.x;
-    const int s0 = layer_seg_first[k], s1 = layer_seg_first[k + 1];
-    const double* __restrict__ row = partials + static_cast<size_t>(m) * C;
-    double acc = 0.0;
-    for (int s = s0 + tid; s < s1; s += kFinalizeThreads) acc += row[s];
-    const double total = block_sum_fixed_order<kFinalizeThreads>(acc);
-
+    grid_dependency_sync();
+    __shared__ double layer_sum[kMaxWorkers];
+    __shared__ WeightsSmem wsm;
     __shared__ int is_last;
-    if (tid == 0) {
-        S[static_cast<size_t>(k) * M + m] = total;
-        if (sumsq_out) sumsq_out[static_cast<size_t>(k) * M + m] = total;
-        __threadfence();
-        const unsigned t = atomicAdd(ticket, 1u);
-        is_last = (t == static_cast<unsigned>(K) * M - 1u);
+    const int k = blockIdx.x;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int s0 = layer_seg_first[k], s1 = layer_seg_first[k + 1];
+    for (int m = warp; m < M; m += kFinalizeThreads / 32) {
+        const double* __restrict__ row = partials + static_cast<size_t>(m) * C;
+        double acc = 0.0;
+        for (int s = s0 + lane; s < s1; s += 32) acc += row[s];
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, d);
+        if (lane == 0) layer_sum[m] = acc;
     }
+    __syncthreads();
+    double term = 0.0;
+    if (tid < M) {
+        const double s = layer_sum[tid];
+        const size_t idx = static_cast<size_t>(k) * M + tid;
+        S[idx] = s;
+        if (sumsq_out) sumsq_out[idx] = s;
+        term = (variant == kGrawa) ? s : sqrt(s);
+        A[idx] = term;
+    }
+    int flagged = 0;
+    if (variant == kLgrawa) {
+        const float w = weights_parallel(term, M, wsm, flagged);
+        if (tid < M) {
+            const size_t idx = static_cast<size_t>(k) * M + tid;
+            if (scores_out) scores_out[idx] = term;
+            beta[idx] = w;
+            if (weights_out) weights_out[idx] = w;
+        }
+        if (tid == 0 && flagged) atomicOr(status, kStatusNonFinite);
+        return;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) is_last = (atomicAdd(ticket, 1u) == static_cast<unsigned>(K) - 1u);
     __syncthreads();
     if (!is_last) return;
     __threadfence();
-
-    const volatile double* Sv = S;
-    int flagged = 0;
-    if (variant == kLgrawa) {
-        for (int kk = tid; kk < K; kk += kFinalizeThreads) {
-            double* Arow = A + static_cast<size_t>(kk) * M;
-            for (int mm = 0; mm < M; ++mm) {
-                const double a = sqrt(Sv[static_cast<size_t>(kk) * M + mm]);
-                Arow[mm] = a;
-                if (scores_out) scores_out[static_cast<size_t>(kk) * M + mm] = a;
-            }
-            flagged |= weights_group(Arow, M, beta + static_cast<size_t>(kk) * M,
-                                     weights_out ? weights_out + static_cast<size_t>(kk) * M : nullptr);
-        }
-    } else {
-        if (tid < M) {
-            double a = 0.0;
-            if (variant == kMgrawa) {
-                for (int kk = 0; kk < K; ++kk) a += sqrt(Sv[static_cast<size_t>(kk) * M + tid]);
-            } else {
-                for (int kk = 0; kk < K; ++kk) a += Sv[static_cast<size_t>(kk) * M + tid];
-                a = sqrt(a);
-            }
-            A[tid] = a;
-            if (scores_out) scores_out[tid] = a;
-        }
+    // Rows of A are staged through shared memory in blocks (parallel loads); thread m then adds
+    // its column in layer order.
+    __shared__ double stage[kStageDoubles];
+    const int rows_per_block = kStageDoubles / M;
+    double a = 0.0;
+    for (int k0 = 0; k0 < K; k0 += rows_per_block) {
+        const int rows = min(rows_per_block, K - k0);
+        const double* src = A + static_cast<size_t>(k0) * M;
+        for (int i = tid; i < rows * M; i += kFinalizeThreads) stage[i] = __ldcg(src + i);
         __syncthreads();
-        if (tid == 0) flagged = weights_group(A, M, beta, weights_out);
+        if (tid < M)
+            for (int r = 0; r < rows; ++r) a += stage[r * M + tid];
+        __syncthreads();
     }
-    if (flagged) atomicOr(status, kStatusNonFinite);
+    if (tid < M) {
+        if (variant == kGrawa) a = sqrt(a);
+        A[static_cast<size_t>(K) * M + tid] = a;
+        if (scores_out) scores_out[tid] = a;
+    }
+    const float w = weights_parallel(a, M, wsm, flagged);
+    if (tid < M) {
+        beta[tid] = w;
+        if (weights_out) weights_out[tid] = w;
+    }
+    if (tid == 0 && flagged) atomicOr(status, kStatusNonFinite);
 }
 
 // ---------------------------------------------------------------------------------------------
 // Steps 4-5, register variant: one thread owns a 16-byte column of all M workers, so each
 // parameter is read once and M independent vector loads are in flight per column.
 //   x_C = sum_m beta_m x_m   (fp32 FMA chain, m = 0..M-1)      x_m <- fmaf(pull, x_C, (1-pull) x_m)
-// PER_LAYER: one CTA per Segment, weights of the segment's layer (Eq. 7); otherwise flat tiles of
-// `tile` elements and one weight per worker (Eq. 2 / Eq. 4).
+// PER_LAYER: the items are the Segments, weights of the segment's layer (Eq. 7); otherwise flat
+// tiles of `tile` elements and one weight per worker (Eq. 2 / Eq. 4).  CTA b takes items b,
+// b + gridDim.x, ...
 // ---------------------------------------------------------------------------------------------
 template <int M>
 __device__ __forceinline__ void pull_scalar(const MutPtrs& x, float* center, const float (&w)[M],
@@ -232,66 +291,74 @@ __device__ __forceinline__ void pull_scalar(const MutPtrs& x, float* center, con
     for (int m = 0; m < M; ++m) st_stream1(x.p[m] + i, fmaf(lambda, c, oml * v[m]));
 }
 
+#ifndef GRAWA_PULL_MIN_BLOCKS
+#define GRAWA_PULL_MIN_BLOCKS 2
+#endif
 template <int M, bool PER_LAYER>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, GRAWA_PULL_MIN_BLOCKS)
 center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restrict__ beta,
-                   const Segment* __restrict__ segs, long long n, int tile, float lambda, int vec_ok)
+                   const Segment* __restrict__ segs, int items, long long n, int tile, float lambda, int vec_ok)
 {
+    grid_dependency_sync();
     constexpr int COLS = (M <= 4) ? 4 : (M <= 8) ? 2 : 1;
-    long long b, e;
-    const float* __restrict__ bt = beta;
-    if (PER_LAYER) {
-        const Segment sg = segs[blockIdx.x];
-        b = sg.begin;
-        e = b + sg.len;
-        bt = beta + static_cast<size_t>(sg.layer) * M;
-    } else {
-        b = static_cast<long long>(blockIdx.x) * tile;
-        e = min(n, b + tile);
-    }
-    float w[M];
-#pragma unroll
-    for (int m = 0; m < M; ++m) w[m] = bt[m];
     const float oml = 1.0f - lambda;
     const int tid = threadIdx.x;
-
-    long long hb, te;
-    split_range(b, e, vec_ok, hb, te);
-    const int ncol = static_cast<int>((te - hb) >> 2);
-    for (int c0 = 0; c0 < ncol; c0 += kThreads * COLS) {
-        float4 v[COLS][M];
+    float w[M];
+    if (!PER_LAYER) {
 #pragma unroll
-        for (int q = 0; q < COLS; ++q) {
-            const int c = c0 + q * kThreads + tid;
-            if (c < ncol) {
-#pragma unroll
-                for (int m = 0; m < M; ++m) v[q][m] = ld_stream4(reinterpret_cast<const float4*>(x.p[m] + hb) + c);
-            }
-        }
-#pragma unroll
-        for (int q = 0; q < COLS; ++q) {
-            const int c = c0 + q * kThreads + tid;
-            if (c < ncol) {
-                float4 cc;
-                cc.x = w[0] * v[q][0].x; cc.y = w[0] * v[q][0].y; cc.z = w[0] * v[q][0].z; cc.w = w[0] * v[q][0].w;
-#pragma unroll
-                for (int m = 1; m < M; ++m) {
-                    cc.x = fmaf(w[m], v[q][m].x, cc.x); cc.y = fmaf(w[m], v[q][m].y, cc.y);
-                    cc.z = fmaf(w[m], v[q][m].z, cc.z); cc.w = fmaf(w[m], v[q][m].w, cc.w);
-                }
-                if (center) st_stream4(reinterpret_cast<float4*>(center + hb) + c, cc);
-#pragma unroll
-                for (int m = 0; m < M; ++m) {
-                    float4 o;
-                    o.x = fmaf(lambda, cc.x, oml * v[q][m].x); o.y = fmaf(lambda, cc.y, oml * v[q][m].y);
-                    o.z = fmaf(lambda, cc.z, oml * v[q][m].z); o.w = fmaf(lambda, cc.w, oml * v[q][m].w);
-                    st_stream4(reinterpret_cast<float4*>(x.p[m] + hb) + c, o);
-                }
-            }
-        }
+        for (int m = 0; m < M; ++m) w[m] = beta[m];
     }
-    for (long long i = b + tid; i < hb; i += kThreads) pull_scalar<M>(x, center, w, lambda, oml, i);
-    for (long long i = te + tid; i < e; i += kThreads) pull_scalar<M>(x, center, w, lambda, oml, i);
+    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+        long long b, e;
+        if (PER_LAYER) {
+            const Segment sg = segs[item];
+            b = sg.begin;
+            e = b + sg.len;
+            const float* __restrict__ bt = beta + static_cast<size_t>(sg.layer) * M;
+#pragma unroll
+            for (int m = 0; m < M; ++m) w[m] = bt[m];
+        } else {
+            b = static_cast<long long>(item) * tile;
+            e = min(n, b + tile);
+        }
+        long long hb, te;
+        split_range(b, e, vec_ok, hb, te);
+        const int ncol = static_cast<int>((te - hb) >> 2);
+        for (int c0 = 0; c0 < ncol; c0 += kThreads * COLS) {
+            float4 v[COLS][M];
+#pragma unroll
+            for (int q = 0; q < COLS; ++q) {
+                const int c = c0 + q * kThreads + tid;
+                if (c < ncol) {
+#pragma unroll
+                    for (int m = 0; m < M; ++m) v[q][m] = ld_stream4(reinterpret_cast<const float4*>(x.p[m] + hb) + c);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < COLS; ++q) {
+                const int c = c0 + q * kThreads + tid;
+                if (c < ncol) {
+                    float4 cc;
+                    cc.x = w[0] * v[q][0].x; cc.y = w[0] * v[q][0].y; cc.z = w[0] * v[q][0].z; cc.w = w[0] * v[q][0].w;
+#pragma unroll
+                    for (int m = 1; m < M; ++m) {
+                        cc.x = fmaf(w[m], v[q][m].x, cc.x); cc.y = fmaf(w[m], v[q][m].y, cc.y);
+                        cc.z = fmaf(w[m], v[q][m].z, cc.z); cc.w = fmaf(w[m], v[q][m].w, cc.w);
+                    }
+                    if (center) st_stream4(reinterpret_cast<float4*>(center + hb) + c, cc);
+#pragma unroll
+                    for (int m = 0; m < M; ++m) {
+                        float4 o;
+                        o.x = fmaf(lambda, cc.x, oml * v[q][m].x); o.y = fmaf(lambda, cc.y, oml * v[q][m].y);
+                        o.z = fmaf(lambda, cc.z, oml * v[q][m].z); o.w = fmaf(lambda, cc.w, oml * v[q][m].w);
+                        st_stream4(reinterpret_cast<float4*>(x.p[m] + hb) + c, o);
+                    }
+                }
+            }
+        }
+        for (long long i = b + tid; i < hb; i += kThreads) pull_scalar<M>(x, center, w, lambda, oml, i);
+        for (long long i = te + tid; i < e; i += kThreads) pull_scalar<M>(x, center, w, lambda, oml, i);
+    }
 }
 
 // Steps 4-5 for any M up to kMaxWorkers and any alignment: scalar, two passes over the workers
@@ -301,6 +368,7 @@ center_pull_generic_kernel(MutPtrs x, float* __restrict__ center, const float* _
                            const Segment* __restrict__ segs, int per_layer, long long n, int tile,
                            float lambda, int M)
 {
+    grid_dependency_sync();
     long long b, e;
     const float* __restrict__ bt = beta;
     if (per_layer) {
@@ -328,6 +396,7 @@ center_pull_generic_kernel(MutPtrs x, float* __restrict__ center, const float* _
 __global__ void __launch_bounds__(kThreads)
 copy_kernel(const float* __restrict__ src, float* __restrict__ dst, long long n, int vec_ok)
 {
+    grid_dependency_sync();
     const long long stride = static_cast<long long>(gridDim.x) * kThreads;
     const long long t = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x;
     const long long n4 = vec_ok ? (n >> 2) : 0;
@@ -341,6 +410,7 @@ copy_kernel(const float* __restrict__ src, float* __restrict__ dst, long long n,
 __global__ void __launch_bounds__(kThreads)
 prox_kernel(MutPtrs x, const float* __restrict__ center, long long n, int tile, float a, int M, int vec_ok)
 {
+    grid_dependency_sync();
     const long long b = static_cast<long long>(blockIdx.x) * tile;
     const long long e = min(n, b + tile);
     const float oma = 1.0f - a;

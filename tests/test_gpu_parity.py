@@ -373,3 +373,73 @@ def test_step_inside_a_cuda_graph(grawa):
     assert bool((center == ref["center"]).all())
     for u, v in zip(x, ref["workers"]):
         assert bool((u == v).all())
+
+
+# ------------------------------------------------------------------ the bulk-copy centre+pull kernel
+
+@pytest.fixture
+def bulk_variant(grawa):
+    old = grawa.grawa_get_option("pull_variant")
+    grawa.grawa_set_option("pull_variant", 2)
+    yield grawa
+    grawa.grawa_set_option("pull_variant", old)
+    grawa.grawa_set_option("bulk_tile", 0)
+
+
+@pytest.mark.parametrize("variant", ["mgrawa", "lgrawa"])
+@pytest.mark.parametrize("name", ["toy10", "resnet20_cifar", "resnet18_imagenet"])
+def test_bulk_variant_parity_on_workloads(bulk_variant, name, variant):
+    cfg = gen.CONFIGS[name]
+    p, g = inputs(name)
+    res = gpu_step(bulk_variant, variant, p, g, cfg.pull, cfg.offsets())
+    compare_with_oracle(res, variant, p, g, cfg.pull, cfg.offsets())
+    assert bulk_variant.grawa_last_step_status() == 0
+
+
+@pytest.mark.parametrize("variant", ["mgrawa", "lgrawa"])
+@pytest.mark.parametrize("sizes", [[1], [3], [7, 5, 3, 1, 2, 6], [0, 5, 0, 0, 9, 0], [10, 1000, 10, 8192, 3, 20000, 1],
+                                   [1023, 1025, 2047, 2049, 4095, 4097, 8191, 8193], [33000]],
+                         ids=lambda s: "-".join(map(str, s)))
+def test_bulk_variant_parity_on_adversarial_tables(bulk_variant, sizes, variant):
+    cfg = gen.custom_config(sizes, 3, seed=11)
+    p, g = gen.make_inputs(cfg)
+    for tile in (0, 256, 2048):
+        bulk_variant.grawa_set_option("bulk_tile", tile)
+        res = gpu_step(bulk_variant, variant, p, g, 0.5, cfg.offsets())
+        compare_with_oracle(res, variant, p, g, 0.5, cfg.offsets())
+        assert bulk_variant.grawa_last_step_status() == 0
+
+
+@pytest.mark.parametrize("M", [2, 3, 5, 8, 13, 16, 17, 24, 33, 64])
+def test_bulk_variant_parity_on_worker_counts(bulk_variant, M):
+    cfg = gen.custom_config([10, 50000, 3, 120000, 777], M, seed=100 + M, log10_sigma=(-2.0, 0.0))
+    p, g = gen.make_inputs(cfg)
+    for variant in ("mgrawa", "lgrawa"):
+        res = gpu_step(bulk_variant, variant, p, g, 0.5, cfg.offsets())
+        compare_with_oracle(res, variant, p, g, 0.5, cfg.offsets())
+        assert bulk_variant.grawa_last_step_status() == 0
+
+
+def test_bulk_and_register_variants_agree_bit_for_bit(grawa):
+    """Same arithmetic in the same order: the two centre+pull kernels must give identical bytes."""
+    cfg = gen.CONFIGS["resnet18_imagenet"]
+    p, g = inputs("resnet18_imagenet")
+    ref = gpu_step(grawa, "lgrawa", p, g, 0.5, cfg.offsets())
+    old = grawa.grawa_get_option("pull_variant")
+    try:
+        grawa.grawa_set_option("pull_variant", 2)
+        got = gpu_step(grawa, "lgrawa", p, g, 0.5, cfg.offsets())
+    finally:
+        grawa.grawa_set_option("pull_variant", old)
+    assert bool((ref["center"] == got["center"]).all())
+    for u, v in zip(ref["workers"], got["workers"]):
+        assert bool((u == v).all())
+
+
+def test_many_workers_take_the_bulk_kernel_by_default(grawa):
+    """More than 16 workers: the automatic choice is the bulk-copy kernel (any M up to 64)."""
+    cfg = gen.custom_config([100000, 33, 200001], 40, seed=77, log10_sigma=(-2.0, 0.0))
+    p, g = gen.make_inputs(cfg)
+    res = gpu_step(grawa, "lgrawa", p, g, 0.3, cfg.offsets())
+    compare_with_oracle(res, "lgrawa", p, g, 0.3, cfg.offsets())
+    assert grawa.grawa_last_step_status() == 0
