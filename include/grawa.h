@@ -171,7 +171,9 @@ grawa_status grawa_sumsq_static(const float *const *grads, int64_t n, int M, dou
  * of the sums of squares ("sumsq_tile").  Returns GRAWA_ERR_INVALID_ARG for an unknown name
  * or a value out of range.
  *   "sumsq_tile"   elements per sum-of-squares work item (multiple of 1024, 1024..1048576)
- *   "pull_tile"    elements per centre+pull work item (multiple of 1024, 1024..1048576)
+ *   "pull_tile"    elements per centre+pull work item (multiple of 1024, 1024..1048576);
+ *                  0 (default) = what one CTA of the register kernel covers in a single pass,
+ *                  8192 / 4096 / 2048 / 1024 elements for M <= 2 / 4 / 8 / more
  *   "pull_variant" 0 = automatic (register kernel up to 16 workers, bulk-copy kernel above),
  *                  1 = register kernel (vector loads), 2 = bulk-copy kernel (shared-memory
  *                  staging by 1-D bulk asynchronous copies and bulk stores)

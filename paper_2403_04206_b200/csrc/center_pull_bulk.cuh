@@ -104,23 +104,29 @@ center_pull_bulk_kernel(MutPtrs x, float* __restrict__ center, const float* __re
     }
     __syncthreads();
 
-    // Warp 0, all lanes: claim the next item, publish it in info[s] and start its loads into stage s.
-    auto fill_stage = [&](int s) {
-        long long b = 0;
-        int len = -1, layer = 0;
-        if (lane == 0) {
-            const unsigned item = atomicAdd(work_counter, 1u);
-            if (item < static_cast<unsigned>(items)) {
-                if (PER_LAYER) {
-                    const Segment sg = segs[item];
-                    b = sg.begin; len = sg.len; layer = sg.layer;
-                } else {
-                    b = static_cast<long long>(item) * tile;
-                    len = static_cast<int>(min(static_cast<long long>(tile), n - b));
-                }
+    // Lane 0 of warp 0 keeps one claimed item ahead: the atomic and the Segment read of the item
+    // after next are issued when a stage is filled and are only needed at the following fill, so
+    // their latency is off the critical path.
+    long long nxt_begin = 0;
+    int nxt_len = -1, nxt_layer = 0;
+    auto claim_next = [&]() {
+        nxt_begin = 0; nxt_len = -1; nxt_layer = 0;
+        const unsigned item = atomicAdd(work_counter, 1u);
+        if (item < static_cast<unsigned>(items)) {
+            if (PER_LAYER) {
+                const Segment sg = segs[item];
+                nxt_begin = sg.begin; nxt_len = sg.len; nxt_layer = sg.layer;
+            } else {
+                nxt_begin = static_cast<long long>(item) * tile;
+                nxt_len = static_cast<int>(min(static_cast<long long>(tile), n - nxt_begin));
             }
-            info[s].begin = b; info[s].len = len; info[s].layer = layer;
         }
+    };
+    // Warp 0, all lanes: publish the claimed item in info[s], start its loads into stage s, claim the next.
+    auto fill_stage = [&](int s) {
+        long long b = nxt_begin;
+        int len = nxt_len;
+        if (lane == 0) { info[s].begin = b; info[s].len = len; info[s].layer = nxt_layer; }
         b = __shfl_sync(0xffffffffu, b, 0);
         len = __shfl_sync(0xffffffffu, len, 0);
         unsigned bytes = 0;
@@ -136,8 +142,10 @@ center_pull_bulk_kernel(MutPtrs x, float* __restrict__ center, const float* __re
             float* dst = stage_mem + static_cast<size_t>(s) * stage_floats;
             for (int m = lane; m < M; m += 32) bulk_load(dst + m * slice_floats, x.p[m] + hb, bytes, &full_bar[s]);
         }
+        if (lane == 0) claim_next();
     };
 
+    if (warp == 0 && lane == 0) claim_next();
     if (warp == 0)
         for (int s = 0; s < stages - 1; ++s) fill_stage(s);
 

@@ -25,7 +25,7 @@ static_assert(kMaxWorkers == GRAWA_MAX_WORKERS, "header and kernels disagree on 
 static std::mutex g_mutex;
 static std::atomic<int64_t> g_launches{0};
 static int64_t g_sumsq_tile = 8192;
-static int64_t g_pull_tile = 4096;
+static int64_t g_pull_tile = 0;           // 0 = one pass of the register kernel: 1024 * pull_cols(M) elements
 static int64_t g_pull_variant = 0;
 static int64_t g_bulk_tile = 0;           // 0 = chosen from M so that at least three stages fit
 static int64_t g_kernel_timing = 0;
@@ -169,7 +169,8 @@ static grawa_status get_plan(int64_t n, int M, const std::vector<int64_t>& off, 
     p->device = device; p->stream = stream; p->n = n; p->M = M; p->off = off;
     p->K = static_cast<int>(off.size()) - 1;
     p->bulk = wants_bulk(M);
-    p->tile1 = g_sumsq_tile; p->tile2 = p->bulk ? bulk_tile_for(M) : g_pull_tile;
+    p->tile1 = g_sumsq_tile;
+    p->tile2 = p->bulk ? bulk_tile_for(M) : (g_pull_tile > 0 ? g_pull_tile : 1024 * pull_cols(std::min(M, kMaxRegWorkers)));
     GRAWA_CUDA_TRY(cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, device));
     std::vector<Segment> s1, s2;
     std::vector<int> first;
@@ -625,7 +626,7 @@ grawa_status grawa_prox_step(float* const* params, const float* center, int64_t 
     int64_t tile;
     {
         std::lock_guard<std::mutex> lock(g_mutex);
-        tile = g_pull_tile;
+        tile = g_pull_tile > 0 ? g_pull_tile : 4096;
     }
     const int64_t tiles = (n + tile - 1) / tile;
     if (tiles > 0x7fffffffll) return GRAWA_ERR_INVALID_ARG;
@@ -693,7 +694,7 @@ grawa_status grawa_set_option(const char* name, int64_t value)
         return GRAWA_OK;
     }
     if (std::strcmp(name, "pull_tile") == 0) {
-        if (!tile_ok) return GRAWA_ERR_INVALID_ARG;
+        if (!tile_ok && value != 0) return GRAWA_ERR_INVALID_ARG;
         if (value != g_pull_tile) { g_pull_tile = value; clear_plans_locked(); }
         return GRAWA_OK;
     }

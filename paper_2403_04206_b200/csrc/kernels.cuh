@@ -34,13 +34,13 @@ struct Segment {
 // Both instructions do nothing in a kernel launched without the attribute.
 __device__ __forceinline__ void grid_dependency_sync()
 {
-#ifndef GRAWA_NO_GRIDDEP
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-#endif
 }
 
-// Streaming accesses: every byte is touched once per step, so keep it out of the way in L1/L2.
+// Streaming accesses: every byte is touched once per step, so keep it out of the way in L1/L2
+// (ld.global.cs / st.global.cs; measured equal to .nc.L1::no_allocate loads and better than
+// default-cached loads for the sum of squares).
 __device__ __forceinline__ float4 ld_stream4(const float4* p) { return __ldcs(p); }
 __device__ __forceinline__ float ld_stream1(const float* p) { return __ldcs(p); }
 __device__ __forceinline__ void st_stream4(float4* p, float4 v) { __stcs(p, v); }
@@ -291,16 +291,16 @@ __device__ __forceinline__ void pull_scalar(const MutPtrs& x, float* center, con
     for (int m = 0; m < M; ++m) st_stream1(x.p[m] + i, fmaf(lambda, c, oml * v[m]));
 }
 
-#ifndef GRAWA_PULL_MIN_BLOCKS
-#define GRAWA_PULL_MIN_BLOCKS 2
-#endif
+// Columns a thread of the register kernel keeps in flight at once (times M vector loads each).
+__host__ __device__ constexpr int pull_cols(int M) { return (M <= 2) ? 8 : (M <= 4) ? 4 : (M <= 8) ? 2 : 1; }
+
 template <int M, bool PER_LAYER>
-__global__ void __launch_bounds__(kThreads, GRAWA_PULL_MIN_BLOCKS)
+__global__ void __launch_bounds__(kThreads, 2)
 center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restrict__ beta,
                    const Segment* __restrict__ segs, int items, long long n, int tile, float lambda, int vec_ok)
 {
     grid_dependency_sync();
-    constexpr int COLS = (M <= 4) ? 4 : (M <= 8) ? 2 : 1;
+    constexpr int COLS = pull_cols(M);
     const float oml = 1.0f - lambda;
     const int tid = threadIdx.x;
     float w[M];
