@@ -109,7 +109,7 @@ static WorkspaceLayout workspace_layout(int64_t C1, int K, int M)
     w.S = p;        p = align_up(p + sizeof(double) * static_cast<size_t>(K) * M, 256);
     w.A = p;        p = align_up(p + sizeof(double) * (static_cast<size_t>(K) + 1) * M, 256);   // K rows of terms + scores
     w.beta = p;     p = align_up(p + sizeof(float) * static_cast<size_t>(K) * M, 256);
-    w.words = p;    p = align_up(p + 256, 256);   // [0] ticket (unsigned), [1] status (int), [2] work counter (unsigned)
+    w.words = p;    p = align_up(p + 256, 256);   // [1] status (int), [2] work counter (unsigned)
     w.total = p;
     return w;
 }
@@ -125,6 +125,8 @@ struct Plan {
     Segment* d_segs1 = nullptr;      // sum-of-squares items
     Segment* d_segs2 = nullptr;      // per-layer centre+pull items
     int* d_layer_first = nullptr;    // first sum-of-squares item of each layer, K+1 entries
+    unsigned* d_tickets = nullptr;   // the finalisation's arrival counter; zero between steps
+    int* d_layer_flag = nullptr;     // K per-layer non-finite flags
     void* d_ws = nullptr;            // owned scratch (used when the caller passes none)
     WorkspaceLayout ws{};
     float* d_stage = nullptr;        // owned staging for the host-buffer entry point
@@ -133,6 +135,7 @@ struct Plan {
     ~Plan()
     {
         cudaFree(d_segs1); cudaFree(d_segs2); cudaFree(d_layer_first); cudaFree(d_ws); cudaFree(d_stage);
+        cudaFree(d_tickets); cudaFree(d_layer_flag);
     }
 };
 
@@ -185,6 +188,10 @@ static grawa_status get_plan(int64_t n, int M, const std::vector<int64_t>& off, 
     GRAWA_CUDA_TRY(cudaMemcpy(p->d_segs1, s1.data(), sizeof(Segment) * s1.size(), cudaMemcpyHostToDevice));
     GRAWA_CUDA_TRY(cudaMemcpy(p->d_segs2, s2.data(), sizeof(Segment) * s2.size(), cudaMemcpyHostToDevice));
     GRAWA_CUDA_TRY(cudaMemcpy(p->d_layer_first, first.data(), sizeof(int) * first.size(), cudaMemcpyHostToDevice));
+    GRAWA_CUDA_TRY(cudaMalloc(&p->d_tickets, sizeof(unsigned)));
+    GRAWA_CUDA_TRY(cudaMemset(p->d_tickets, 0, sizeof(unsigned)));
+    GRAWA_CUDA_TRY(cudaMalloc(&p->d_layer_flag, sizeof(int) * static_cast<size_t>(p->K)));
+    GRAWA_CUDA_TRY(cudaMemset(p->d_layer_flag, 0, sizeof(int) * static_cast<size_t>(p->K)));
     *out = p.get();
     g_plans[key] = std::move(p);
     return GRAWA_OK;
@@ -339,8 +346,8 @@ static grawa_status enqueue_step(int variant, float* const* params, const float*
     double* S = reinterpret_cast<double*>(ws + plan->ws.S);
     double* A = reinterpret_cast<double*>(ws + plan->ws.A);
     float* beta = reinterpret_cast<float*>(ws + plan->ws.beta);
-    unsigned* ticket = reinterpret_cast<unsigned*>(ws + plan->ws.words);
     int* status = reinterpret_cast<int*>(ws + plan->ws.words) + 1;
+    unsigned* counter = reinterpret_cast<unsigned*>(ws + plan->ws.words) + 2;
     g_last_status[{plan->device, stream}] = status;
 
     ConstPtrs gp{};
@@ -363,17 +370,24 @@ static grawa_status enqueue_step(int variant, float* const* params, const float*
         GRAWA_CUDA_TRY(cudaEventRecord(ts->e[0], stream));
     }
     const bool pdl = g_pdl != 0 && ts == nullptr;   // event records between the kernels need plain ordering
+    StepScratch sc{};
+    sc.segs = plan->d_segs1; sc.layer_seg_first = plan->d_layer_first;
+    sc.C = plan->C1; sc.K = K; sc.M = M; sc.variant = variant;
+    sc.partials = partials; sc.S = S; sc.A = A; sc.beta = beta; sc.layer_flag = plan->d_layer_flag;
+    sc.global_ticket = plan->d_tickets;
+    sc.global_target = static_cast<unsigned>(K);
+    sc.status = status; sc.work_counter = counter;
+    sc.weights_out = opt ? opt->weights_out : nullptr;
+    sc.scores_out = opt ? opt->scores_out : nullptr;
+    sc.sumsq_out = opt ? opt->sumsq_out : nullptr;
     // step 1: partial sums of squares, one CTA per (worker, item)
     const int items1 = plan->C1 * M;
     const int grid1 = g_sumsq_ctas_per_sm > 0
                           ? static_cast<int>(std::min<int64_t>(items1, g_sumsq_ctas_per_sm * plan->sm_count)) : items1;
-    GRAWA_CUDA_TRY(launch_kernel(sumsq_kernel<8>, grid1, kThreads, stream, pdl, gp, plan->d_segs1, plan->C1, items1, partials,
-                                 vec_g ? 1 : 0, ticket, status, ticket + 2));
+    GRAWA_CUDA_TRY(launch_kernel(sumsq_kernel<8>, grid1, kThreads, stream, pdl, gp, sc, items1, vec_g ? 1 : 0));
     if (ts) GRAWA_CUDA_TRY(cudaEventRecord(ts->e[1], stream));
     // steps 1b-3: S, scores, weights
-    GRAWA_CUDA_TRY(launch_kernel(finalize_kernel, K, kFinalizeThreads, stream, pdl, partials, plan->d_layer_first, plan->C1, K, M,
-                                 variant, S, A, beta, ticket, status, opt ? opt->weights_out : nullptr,
-                                 opt ? opt->scores_out : nullptr, opt ? opt->sumsq_out : nullptr));
+    GRAWA_CUDA_TRY(launch_kernel(finalize_kernel, K, kThreads, stream, pdl, sc));
     if (ts) GRAWA_CUDA_TRY(cudaEventRecord(ts->e[2], stream));
     // steps 4-5
     if (M == 1) {
@@ -397,7 +411,7 @@ static grawa_status enqueue_step(int variant, float* const* params, const float*
         GRAWA_CUDA_TRY(CenterPullBulkDispatch<kMaxRegWorkers>::run(M <= kMaxRegWorkers ? M : 1, per_layer, gridb, grid,
                                                                    stage_bytes * stages, stream, pdl, xp, center_out, beta,
                                                                    plan->d_segs2, n, static_cast<int>(plan->tile2), stages, M, pull,
-                                                                   ticket + 2, status));
+                                                                   counter, status));
     } else if (vec_x && M <= kMaxRegWorkers) {
         const int grid2 = g_pull_ctas_per_sm > 0
                               ? static_cast<int>(std::min<int64_t>(grid, g_pull_ctas_per_sm * plan->sm_count)) : grid;

@@ -10,7 +10,7 @@ namespace grawa {
 constexpr int kMaxWorkers = 64;
 constexpr int kThreads = 256;          // threads per CTA of the streaming kernels
 constexpr int kFinalizeThreads = 256;
-constexpr int kStageDoubles = 2048;    // shared-memory staging of the finalisation (16 KB)
+constexpr int kStageDoubles = 256;     // shared-memory staging of the finalisation (2 KB)
 constexpr int kMaxRegWorkers = 16;     // largest M the register-resident centre+pull kernel is built for
 
 enum Variant { kGrawa = 0, kMgrawa = 1, kLgrawa = 2 };
@@ -78,29 +78,203 @@ __device__ __forceinline__ double block_sum_fixed_order(double v)
     return total;
 }
 
+// Everything the sum-of-squares and finalisation code needs to know about one step.
+struct StepScratch {
+    const Segment* segs;           // sum-of-squares work items of one worker, C of them
+    const int* layer_seg_first;    // first item of each layer, K+1 entries
+    int C, K, M, variant;
+    double* partials;              // [M][C]
+    double* S;                     // [K][M]
+    double* A;                     // [K+1][M]: per-layer terms, then the per-worker scores in row K
+    float* beta;                   // [K][M] (LGRAWA) or [M]
+    int* layer_flag;               // [K] non-finite flag of each layer's group (LGRAWA)
+    unsigned* global_ticket;       // zero between steps
+    unsigned global_target;        // arrivals that complete the step's finalisation
+    int* status;                   // written (not or-ed) when the finalisation completes
+    unsigned* work_counter;        // cleared for the bulk-copy centre+pull kernel
+    float* weights_out;            // optional copies
+    double* scores_out;
+    double* sumsq_out;
+};
+
+// Step 3 for one group of M scores (Eq. 2 / 4 / 7) with the zero-score limit and the non-finite
+// fallback, computed by the whole CTA: thread m < M passes its score `a` and gets beta_m back.
+// The reciprocals are taken in parallel and added by one thread in worker order, so the value is
+// the one a sequential loop over m = 0..M-1 gives.  Every thread of the CTA must call it.
+struct WeightsSmem {
+    double r[kMaxWorkers];
+    double z;
+};
+
+__device__ __forceinline__ float weights_parallel(double a, int M, WeightsSmem& sm, int& flagged)
+{
+    const int tid = threadIdx.x;
+    const bool active = tid < M;
+    const bool fin = active && isfinite(a);
+    const bool zero = fin && a == 0.0;
+    const int finite = __syncthreads_count(fin);
+    const int zeros = __syncthreads_count(zero);
+    if (active) sm.r[tid] = (fin && !zero) ? 1.0 / a : 0.0;
+    __syncthreads();
+    if (tid == 0) {
+        double z = 0.0;
+        for (int m = 0; m < M; ++m) z += sm.r[m];     // adding the 0.0 of a skipped worker is exact
+        sm.z = z;
+    }
+    __syncthreads();
+    flagged = finite < M;
+    double w = 0.0;
+    if (active) {
+        if (finite == 0) w = 1.0 / M;
+        else if (zeros > 0) w = zero ? 1.0 / zeros : 0.0;
+        else w = fin ? sm.r[tid] / sm.z : 0.0;
+    }
+    return static_cast<float>(w);
+}
+
+struct FinalizeSmem {
+    double layer_sum[kMaxWorkers];
+    WeightsSmem w;
+    double stage[kStageDoubles];
+    int flag;
+};
+
+// Steps 1b-3 for one non-empty layer, by a whole CTA of kThreads threads.  Warp w adds the partials
+// of workers w, w+8, ... of layer k in a fixed order into S[k][m]; the layer's terms sqrt(S) (S
+// itself for the flat norm) go to row k of A; LGRAWA turns them into the layer's weights (Eq. 7).
+__device__ __forceinline__ void finalize_layer(const StepScratch& sc, int k, FinalizeSmem& sm)
+{
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int M = sc.M;
+    const int s0 = sc.layer_seg_first[k], s1 = sc.layer_seg_first[k + 1];
+    for (int m = warp; m < M; m += kThreads / 32) {
+        const double* row = sc.partials + static_cast<size_t>(m) * sc.C;
+        double acc = 0.0;
+        for (int s = s0 + lane; s < s1; s += 32) acc += __ldcg(row + s);
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, d);
+        if (lane == 0) sm.layer_sum[m] = acc;
+    }
+    __syncthreads();
+    double term = 0.0;
+    const size_t idx = static_cast<size_t>(k) * M + tid;
+    if (tid < M) {
+        const double s = sm.layer_sum[tid];
+        sc.S[idx] = s;
+        if (sc.sumsq_out) sc.sumsq_out[idx] = s;
+        term = (sc.variant == kGrawa) ? s : sqrt(s);
+        sc.A[idx] = term;
+    }
+    if (sc.variant == kLgrawa) {
+        int flagged = 0;
+        const float w = weights_parallel(term, M, sm.w, flagged);
+        if (tid < M) {
+            if (sc.scores_out) sc.scores_out[idx] = term;
+            sc.beta[idx] = w;
+            if (sc.weights_out) sc.weights_out[idx] = w;
+        }
+        if (tid == 0) sc.layer_flag[k] = flagged;
+    }
+}
+
+// Called by a whole CTA after its part of the finalisation.  The CTA that makes the count reach
+// `global_target` finishes the step: rows of empty layers, MGRAWA / GRAWA scores (the K rows of A
+// added per worker in layer order, Eq. 3 / Eq. 2) and weights (Eq. 4), the status word, and the
+// reset of the counters for the next step.  No CTA waits for another.
+__device__ __forceinline__ void finalize_arrive(const StepScratch& sc, FinalizeSmem& sm)
+{
+    const int tid = threadIdx.x;
+    const int M = sc.M, K = sc.K;
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const bool last = atomicAdd(sc.global_ticket, 1u) == sc.global_target - 1u;
+        if (last) *sc.global_ticket = 0u;
+        sm.flag = last;
+    }
+    __syncthreads();
+    if (!sm.flag) return;
+    __threadfence();
+
+    // empty layers: zero sums and terms, uniform weights (they are never applied)
+    for (int k = tid; k < K; k += kThreads) {
+        if (sc.layer_seg_first[k] != sc.layer_seg_first[k + 1]) continue;
+        for (int m = 0; m < M; ++m) {
+            const size_t idx = static_cast<size_t>(k) * M + m;
+            sc.S[idx] = 0.0;
+            sc.A[idx] = 0.0;
+            if (sc.sumsq_out) sc.sumsq_out[idx] = 0.0;
+            if (sc.variant == kLgrawa) {
+                const float u = static_cast<float>(1.0 / M);
+                sc.beta[idx] = u;
+                if (sc.weights_out) sc.weights_out[idx] = u;
+                if (sc.scores_out) sc.scores_out[idx] = 0.0;
+            }
+        }
+    }
+    int flagged = 0;
+    if (sc.variant == kLgrawa) {
+        int f = 0;
+        for (int k = tid; k < K; k += kThreads)
+            if (sc.layer_seg_first[k] != sc.layer_seg_first[k + 1]) f |= __ldcg(sc.layer_flag + k);
+        flagged = __syncthreads_or(f);
+    } else {
+        // Rows of A are staged through shared memory in blocks (parallel loads); thread m then adds
+        // its column in layer order.  Rows of empty layers count as 0.
+        const int rows_per_block = kStageDoubles / M;
+        double a = 0.0;
+        for (int k0 = 0; k0 < K; k0 += rows_per_block) {
+            const int rows = min(rows_per_block, K - k0);
+            for (int i = tid; i < rows * M; i += kThreads) {
+                const int k = k0 + i / M;
+                const bool empty = sc.layer_seg_first[k] == sc.layer_seg_first[k + 1];
+                sm.stage[i] = empty ? 0.0 : __ldcg(sc.A + static_cast<size_t>(k0) * M + i);
+            }
+            __syncthreads();
+            if (tid < M)
+                for (int r = 0; r < rows; ++r) a += sm.stage[r * M + tid];
+            __syncthreads();
+        }
+        if (tid < M) {
+            if (sc.variant == kGrawa) a = sqrt(a);
+            sc.A[static_cast<size_t>(K) * M + tid] = a;
+            if (sc.scores_out) sc.scores_out[tid] = a;
+        }
+        const float w = weights_parallel(a, M, sm.w, flagged);
+        if (tid < M) {
+            sc.beta[tid] = w;
+            if (sc.weights_out) sc.weights_out[tid] = w;
+        }
+    }
+    if (tid == 0) {
+        *sc.status = flagged ? kStatusNonFinite : 0;
+        *sc.work_counter = 0u;
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Step 1 (Eq. 3 / Eq. 5): partial[m][s] = sum of g_m[j]^2 over segment s.  Work items are the
-// (worker, segment) pairs, worker-major; CTA b takes items b, b + gridDim.x, ... (a grid of a few
-// CTAs per SM streams through the list; a grid of `items` CTAs gives one item each).  fp32
-// squares are accumulated in runs of UNROLL terms per accumulator and the runs are combined in
-// fp64; the order depends only on the item, never on the grid, so results are reproducible.
-// CTA 0 also clears the ticket, status and work-counter words for the kernels that follow on the stream.
+// (worker, segment) pairs, worker-major; CTA b takes items b, b + gridDim.x, ...  fp32 squares
+// are accumulated in runs of UNROLL terms per accumulator and the runs are combined in fp64; the
+// order depends only on the item, never on the grid, so results are reproducible.
 // ---------------------------------------------------------------------------------------------
+#ifndef GRAWA_SUMSQ_MINB
+#define GRAWA_SUMSQ_MINB 1
+#endif
 template <int UNROLL>
-__global__ void __launch_bounds__(kThreads)
-sumsq_kernel(ConstPtrs grads, const Segment* __restrict__ segs, int C, int items, double* __restrict__ partials,
-             int vec_ok, unsigned* __restrict__ ticket, int* __restrict__ status, unsigned* __restrict__ work_counter)
+__global__ void __launch_bounds__(kThreads, GRAWA_SUMSQ_MINB)
+sumsq_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
 {
     grid_dependency_sync();
     __shared__ double warp_part[2][kThreads / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (blockIdx.x == 0 && tid == 0) { *ticket = 0u; *status = 0; *work_counter = 0u; }
+    const int C = sc.C;
 
     int parity = 0;
     for (int item = blockIdx.x; item < items; item += gridDim.x, parity ^= 1) {
         const int m = item / C;
         const int s = item - m * C;
-        const Segment sg = segs[s];
+        const Segment sg = sc.segs[s];
         const float* __restrict__ g = grads.p[m];
         const long long b = sg.begin, e = b + sg.len;
         long long hb, te;
@@ -146,126 +320,23 @@ sumsq_kernel(ConstPtrs grads, const Segment* __restrict__ segs, int C, int items
             double total = 0.0;
 #pragma unroll
             for (int w = 0; w < kThreads / 32; ++w) total += warp_part[parity][w];
-            partials[static_cast<size_t>(m) * C + s] = total;
+            sc.partials[static_cast<size_t>(m) * C + s] = total;
         }
     }
 }
 
-// Step 3 for one group of M scores (Eq. 2 / 4 / 7) with the zero-score limit and the non-finite
-// fallback, computed by the whole CTA: thread m < M passes its score `a` and gets beta_m back.
-// The reciprocals are taken in parallel and added by one thread in worker order, so the value is
-// the one a sequential loop over m = 0..M-1 gives.  Every thread of the CTA must call it.
-struct WeightsSmem {
-    double r[kMaxWorkers];
-    double z;
-};
-
-__device__ __forceinline__ float weights_parallel(double a, int M, WeightsSmem& sm, int& flagged)
-{
-    const int tid = threadIdx.x;
-    const bool active = tid < M;
-    const bool fin = active && isfinite(a);
-    const bool zero = fin && a == 0.0;
-    const int finite = __syncthreads_count(fin);
-    const int zeros = __syncthreads_count(zero);
-    if (active) sm.r[tid] = (fin && !zero) ? 1.0 / a : 0.0;
-    __syncthreads();
-    if (tid == 0) {
-        double z = 0.0;
-        for (int m = 0; m < M; ++m) z += sm.r[m];     // adding the 0.0 of a skipped worker is exact
-        sm.z = z;
-    }
-    __syncthreads();
-    flagged = finite < M;
-    double w = 0.0;
-    if (active) {
-        if (finite == 0) w = 1.0 / M;
-        else if (zeros > 0) w = zero ? 1.0 / zeros : 0.0;
-        else w = fin ? sm.r[tid] / sm.z : 0.0;
-    }
-    return static_cast<float>(w);
-}
-
-// ---------------------------------------------------------------------------------------------
-// Steps 1b-3: one CTA per layer.  Warp w adds the partials of workers w, w+8, ... of that layer
-// in a fixed order into S[k][m]; the layer's terms sqrt(S) (S itself for the flat norm) go to row k
-// of A.  LGRAWA: the same CTA turns them into the layer's weights (Eq. 7).  MGRAWA / GRAWA: the
-// CTA that draws the last ticket adds the K rows per worker in layer order (Eq. 3 / Eq. 2), writes
-// the scores to row K of A and computes the M weights (Eq. 4).  No CTA waits for another.
-// ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kFinalizeThreads)
-finalize_kernel(const double* __restrict__ partials, const int* __restrict__ layer_seg_first, int C, int K, int M,
-                int variant, double* S, double* A, float* beta, unsigned* ticket, int* status,
-                float* weights_out, double* scores_out, double* sumsq_out)
+// Steps 1b-3: one CTA per layer reduces the layer's partials and, for LGRAWA, computes its
+// weights; the CTA that arrives last completes the step (see finalize_arrive).
+// (Folding this into the sum-of-squares kernel with one ticket per layer was measured slower: the
+// fence and atomic each CTA then needs before it can retire cost more than the launch they save.)
+__global__ void __launch_bounds__(kThreads)
+finalize_kernel(StepScratch sc)
 {
     grid_dependency_sync();
-    __shared__ double layer_sum[kMaxWorkers];
-    __shared__ WeightsSmem wsm;
-    __shared__ int is_last;
+    __shared__ FinalizeSmem fsm;
     const int k = blockIdx.x;
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int s0 = layer_seg_first[k], s1 = layer_seg_first[k + 1];
-    for (int m = warp; m < M; m += kFinalizeThreads / 32) {
-        const double* __restrict__ row = partials + static_cast<size_t>(m) * C;
-        double acc = 0.0;
-        for (int s = s0 + lane; s < s1; s += 32) acc += row[s];
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, d);
-        if (lane == 0) layer_sum[m] = acc;
-    }
-    __syncthreads();
-    double term = 0.0;
-    if (tid < M) {
-        const double s = layer_sum[tid];
-        const size_t idx = static_cast<size_t>(k) * M + tid;
-        S[idx] = s;
-        if (sumsq_out) sumsq_out[idx] = s;
-        term = (variant == kGrawa) ? s : sqrt(s);
-        A[idx] = term;
-    }
-    int flagged = 0;
-    if (variant == kLgrawa) {
-        const float w = weights_parallel(term, M, wsm, flagged);
-        if (tid < M) {
-            const size_t idx = static_cast<size_t>(k) * M + tid;
-            if (scores_out) scores_out[idx] = term;
-            beta[idx] = w;
-            if (weights_out) weights_out[idx] = w;
-        }
-        if (tid == 0 && flagged) atomicOr(status, kStatusNonFinite);
-        return;
-    }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) is_last = (atomicAdd(ticket, 1u) == static_cast<unsigned>(K) - 1u);
-    __syncthreads();
-    if (!is_last) return;
-    __threadfence();
-    // Rows of A are staged through shared memory in blocks (parallel loads); thread m then adds
-    // its column in layer order.
-    __shared__ double stage[kStageDoubles];
-    const int rows_per_block = kStageDoubles / M;
-    double a = 0.0;
-    for (int k0 = 0; k0 < K; k0 += rows_per_block) {
-        const int rows = min(rows_per_block, K - k0);
-        const double* src = A + static_cast<size_t>(k0) * M;
-        for (int i = tid; i < rows * M; i += kFinalizeThreads) stage[i] = __ldcg(src + i);
-        __syncthreads();
-        if (tid < M)
-            for (int r = 0; r < rows; ++r) a += stage[r * M + tid];
-        __syncthreads();
-    }
-    if (tid < M) {
-        if (variant == kGrawa) a = sqrt(a);
-        A[static_cast<size_t>(K) * M + tid] = a;
-        if (scores_out) scores_out[tid] = a;
-    }
-    const float w = weights_parallel(a, M, wsm, flagged);
-    if (tid < M) {
-        beta[tid] = w;
-        if (weights_out) weights_out[tid] = w;
-    }
-    if (tid == 0 && flagged) atomicOr(status, kStatusNonFinite);
+    if (sc.layer_seg_first[k] != sc.layer_seg_first[k + 1]) finalize_layer(sc, k, fsm);
+    finalize_arrive(sc, fsm);
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -443,3 +443,21 @@ def test_many_workers_take_the_bulk_kernel_by_default(grawa):
     res = gpu_step(grawa, "lgrawa", p, g, 0.3, cfg.offsets())
     compare_with_oracle(res, "lgrawa", p, g, 0.3, cfg.offsets())
     assert grawa.grawa_last_step_status() == 0
+
+
+# ------------------------------------------------------------------ repeated steps on one plan
+
+@pytest.mark.parametrize("variant", ["mgrawa", "lgrawa", "grawa"])
+def test_repeated_steps_on_one_plan_leave_clean_counters(grawa, variant):
+    """The finalisation's arrival counter resets itself; step after step must give the same bytes."""
+    cfg = gen.custom_config([10, 50000, 0, 3, 120000, 777, 0], 7, seed=55, log10_sigma=(-2.0, 0.0))
+    p, g = gen.make_inputs(cfg)
+    off = cfg.offsets()
+    first = gpu_step(grawa, variant, p, g, 0.5, off)
+    compare_with_oracle(first, variant, p, g, 0.5, off)
+    for _ in range(4):
+        again = gpu_step(grawa, variant, p, g, 0.5, off)
+        for key in ("S", "A", "beta"):
+            assert np.array_equal(again[key], first[key]), key
+        assert bool((again["center"] == first["center"]).all())
+        assert grawa.grawa_last_step_status() == 0
