@@ -25,7 +25,7 @@ static_assert(kMaxWorkers == GRAWA_MAX_WORKERS, "header and kernels disagree on 
 static std::mutex g_mutex;
 static std::atomic<int64_t> g_launches{0};
 static int64_t g_sumsq_tile = 8192;
-static int64_t g_pull_tile = 0;           // 0 = one pass of the register kernel: 1024 * pull_cols(M) elements
+static int64_t g_pull_tile = 0;           // 0 = one pass of the register kernel, pull_pass_elems(M)
 static int64_t g_pull_variant = 0;
 static int64_t g_bulk_tile = 0;           // 0 = chosen from M so that at least three stages fit
 static int64_t g_kernel_timing = 0;
@@ -173,7 +173,7 @@ static grawa_status get_plan(int64_t n, int M, const std::vector<int64_t>& off, 
     p->K = static_cast<int>(off.size()) - 1;
     p->bulk = wants_bulk(M);
     p->tile1 = g_sumsq_tile;
-    p->tile2 = p->bulk ? bulk_tile_for(M) : (g_pull_tile > 0 ? g_pull_tile : 1024 * pull_cols(std::min(M, kMaxRegWorkers)));
+    p->tile2 = p->bulk ? bulk_tile_for(M) : (g_pull_tile > 0 ? g_pull_tile : pull_pass_elems(std::min(M, kMaxRegWorkers)));
     GRAWA_CUDA_TRY(cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, device));
     std::vector<Segment> s1, s2;
     std::vector<int> first;
