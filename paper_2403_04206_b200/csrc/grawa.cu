@@ -66,8 +66,20 @@ static int64_t bulk_tile_for(int M)
 }
 
 // ------------------------------------------------------------------ work list
-// Cuts every non-empty layer at the absolute multiples of `tile` that fall inside it.
-static void build_segments(const std::vector<int64_t>& off, int64_t tile, std::vector<Segment>* segs,
+// Tile used inside one layer: `tile`, doubled until the layer has at most `max_items` items (0 =
+// no limit).  Keeps the number of partial sums of a huge layer small enough for the one CTA that
+// adds them up, without giving up the fine grain that balances the many small layers.
+static int64_t layer_tile(int64_t layer_elems, int64_t tile, int64_t max_items)
+{
+    int64_t t = tile;
+    while (max_items > 0 && layer_elems / t > max_items && t < (int64_t{1} << 28)) t *= 2;
+    return t;
+}
+
+constexpr int64_t kMaxSumsqItemsPerLayer = 1024;
+
+// Cuts every non-empty layer at the absolute multiples of its tile that fall inside it.
+static void build_segments(const std::vector<int64_t>& off, int64_t tile, int64_t max_items, std::vector<Segment>* segs,
                            std::vector<int>* layer_first)
 {
     const int K = static_cast<int>(off.size()) - 1;
@@ -77,8 +89,9 @@ static void build_segments(const std::vector<int64_t>& off, int64_t tile, std::v
         if (layer_first) (*layer_first)[k] = static_cast<int>(count);
         int64_t pos = off[k];
         const int64_t end = off[k + 1];
+        const int64_t t = layer_tile(end - pos, tile, max_items);
         while (pos < end) {
-            const int64_t next = std::min(end, (pos / tile + 1) * tile);
+            const int64_t next = std::min(end, (pos / t + 1) * t);
             if (segs) segs->push_back(Segment{pos, static_cast<int>(next - pos), k});
             ++count;
             pos = next;
@@ -87,11 +100,14 @@ static void build_segments(const std::vector<int64_t>& off, int64_t tile, std::v
     if (layer_first) (*layer_first)[K] = static_cast<int>(count);
 }
 
-static int64_t count_segments(const std::vector<int64_t>& off, int64_t tile)
+static int64_t count_segments(const std::vector<int64_t>& off, int64_t tile, int64_t max_items)
 {
     int64_t count = 0;
     for (size_t k = 0; k + 1 < off.size(); ++k) {
-        if (off[k + 1] > off[k]) count += (off[k + 1] - 1) / tile - off[k] / tile + 1;
+        if (off[k + 1] > off[k]) {
+            const int64_t t = layer_tile(off[k + 1] - off[k], tile, max_items);
+            count += (off[k + 1] - 1) / t - off[k] / t + 1;
+        }
     }
     return count;
 }
@@ -177,8 +193,8 @@ static grawa_status get_plan(int64_t n, int M, const std::vector<int64_t>& off, 
     GRAWA_CUDA_TRY(cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, device));
     std::vector<Segment> s1, s2;
     std::vector<int> first;
-    build_segments(off, p->tile1, &s1, &first);
-    build_segments(off, p->tile2, &s2, nullptr);
+    build_segments(off, p->tile1, kMaxSumsqItemsPerLayer, &s1, &first);
+    build_segments(off, p->tile2, 0, &s2, nullptr);
     if (s1.size() * static_cast<size_t>(M) > 0x7fffffffull || s2.size() > 0x7fffffffull) return GRAWA_ERR_INVALID_ARG;
     p->C1 = static_cast<int>(s1.size()); p->C2 = static_cast<int>(s2.size());
     p->ws = workspace_layout(p->C1, p->K, M);
@@ -546,7 +562,7 @@ size_t grawa_workspace_bytes(int64_t n, int M, const int64_t* layer_offsets, int
         off.assign({0, n});
     }
     std::lock_guard<std::mutex> lock(g_mutex);
-    return workspace_layout(count_segments(off, g_sumsq_tile), static_cast<int>(off.size()) - 1, M).total;
+    return workspace_layout(count_segments(off, g_sumsq_tile, kMaxSumsqItemsPerLayer), static_cast<int>(off.size()) - 1, M).total;
 }
 
 grawa_status grawa_mgrawa_step(float* const* params, const float* const* grads, int64_t n, int M, float pull,

@@ -10,7 +10,7 @@ namespace grawa {
 constexpr int kMaxWorkers = 64;
 constexpr int kThreads = 256;          // threads per CTA of the streaming kernels
 constexpr int kFinalizeThreads = 256;
-constexpr int kStageDoubles = 256;     // shared-memory staging of the finalisation (2 KB)
+constexpr int kStageDoubles = 1024;    // shared-memory staging of the finalisation (8 KB)
 constexpr int kMaxRegWorkers = 16;     // largest M the register-resident centre+pull kernel is built for
 
 enum Variant { kGrawa = 0, kMgrawa = 1, kLgrawa = 2 };
@@ -149,8 +149,16 @@ __device__ __forceinline__ void finalize_layer(const StepScratch& sc, int k, Fin
     const int s0 = sc.layer_seg_first[k], s1 = sc.layer_seg_first[k + 1];
     for (int m = warp; m < M; m += kThreads / 32) {
         const double* row = sc.partials + static_cast<size_t>(m) * sc.C;
-        double acc = 0.0;
-        for (int s = s0 + lane; s < s1; s += 32) acc += __ldcg(row + s);
+        // eight independent running sums per lane keep eight loads in flight; the order in which
+        // they are combined is fixed, so the sum is the same on every run
+        double part[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
+        int s = s0 + lane;
+        for (; s + 7 * 32 < s1; s += 8 * 32) {
+#pragma unroll
+            for (int u = 0; u < 8; ++u) part[u] += __ldcg(row + s + u * 32);
+        }
+        for (int u = 0; s < s1; s += 32, ++u) part[u] += __ldcg(row + s);
+        double acc = ((part[0] + part[1]) + (part[2] + part[3])) + ((part[4] + part[5]) + (part[6] + part[7]));
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, d);
         if (lane == 0) sm.layer_sum[m] = acc;

@@ -461,3 +461,16 @@ def test_repeated_steps_on_one_plan_leave_clean_counters(grawa, variant):
             assert np.array_equal(again[key], first[key]), key
         assert bool((again["center"] == first["center"]).all())
         assert grawa.grawa_last_step_status() == 0
+
+
+def test_parity_one_huge_layer_among_small_ones(grawa):
+    """A layer of more than 1024 base tiles takes a larger tile (fewer partial sums); indexing of
+    the neighbours and the exact-integer sums must be unaffected."""
+    sizes = [7, 20_000_003, 5, 4096]
+    off = np.concatenate([[0], np.cumsum(sizes)])
+    rng = np.random.default_rng(8)
+    g = [rng.integers(-2, 3, size=off[-1]).astype(np.float32) for _ in range(2)]
+    p = [rng.normal(size=off[-1]).astype(np.float32) for _ in range(2)]
+    res = gpu_step(grawa, "lgrawa", p, g, 0.5, off)
+    assert np.array_equal(res["S"], oracle.sumsq(g, off))
+    compare_with_oracle(res, "lgrawa", p, g, 0.5, off)
