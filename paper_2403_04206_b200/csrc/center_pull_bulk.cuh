@@ -84,7 +84,8 @@ __device__ __forceinline__ void bulk_edge_element(const MutPtrs& x, float* cente
 template <int MT, bool PER_LAYER>
 __global__ void __launch_bounds__(kThreads, 1)
 center_pull_bulk_kernel(MutPtrs x, float* __restrict__ center, const float* __restrict__ beta,
-                        const Segment* __restrict__ segs, int items, long long n, int tile, int stages, int M_rt,
+                        const Segment* __restrict__ segs, int item_begin, int item_end, long long n, int tile, int stages,
+                        int M_rt,
                         float lambda, unsigned* __restrict__ work_counter, int* __restrict__ status)
 {
     grid_dependency_sync();
@@ -111,8 +112,8 @@ center_pull_bulk_kernel(MutPtrs x, float* __restrict__ center, const float* __re
     int nxt_len = -1, nxt_layer = 0;
     auto claim_next = [&]() {
         nxt_begin = 0; nxt_len = -1; nxt_layer = 0;
-        const unsigned item = atomicAdd(work_counter, 1u);
-        if (item < static_cast<unsigned>(items)) {
+        const unsigned item = static_cast<unsigned>(item_begin) + atomicAdd(work_counter, 1u);
+        if (item < static_cast<unsigned>(item_end)) {
             if (PER_LAYER) {
                 const Segment sg = segs[item];
                 nxt_begin = sg.begin; nxt_len = sg.len; nxt_layer = sg.layer;

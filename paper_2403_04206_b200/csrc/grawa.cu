@@ -147,11 +147,16 @@ struct Plan {
     WorkspaceLayout ws{};
     float* d_stage = nullptr;        // owned staging for the host-buffer entry point
     int sm_count = 148;
+    std::vector<Segment> h_segs2;    // host copy of the centre+pull items (chunking of the host-buffer path)
+    cudaStream_t d2h_stream = nullptr;   // downloads of the host-buffer path
+    std::vector<cudaEvent_t> events;     // chunk-done events of the host-buffer path
     bool bulk = false;               // centre+pull items are cut for the bulk-copy kernel
     ~Plan()
     {
         cudaFree(d_segs1); cudaFree(d_segs2); cudaFree(d_layer_first); cudaFree(d_ws); cudaFree(d_stage);
         cudaFree(d_tickets); cudaFree(d_layer_flag);
+        if (d2h_stream) cudaStreamDestroy(d2h_stream);
+        for (cudaEvent_t ev : events) cudaEventDestroy(ev);
     }
 };
 
@@ -197,6 +202,7 @@ static grawa_status get_plan(int64_t n, int M, const std::vector<int64_t>& off, 
     build_segments(off, p->tile2, 0, &s2, nullptr);
     if (s1.size() * static_cast<size_t>(M) > 0x7fffffffull || s2.size() > 0x7fffffffull) return GRAWA_ERR_INVALID_ARG;
     p->C1 = static_cast<int>(s1.size()); p->C2 = static_cast<int>(s2.size());
+    p->h_segs2 = s2;
     p->ws = workspace_layout(p->C1, p->K, M);
     GRAWA_CUDA_TRY(cudaMalloc(&p->d_segs1, sizeof(Segment) * std::max<size_t>(1, s1.size())));
     GRAWA_CUDA_TRY(cudaMalloc(&p->d_segs2, sizeof(Segment) * std::max<size_t>(1, s2.size())));
@@ -289,15 +295,15 @@ static cudaError_t launch_kernel(void (*kernel)(KArgs...), int grid, int block, 
 // Bulk-copy centre+pull: MT = M for 2..16 (register column), MT = 0 for larger M.
 
 template <int MT>
-static cudaError_t launch_center_pull_bulk(bool per_layer, int grid, int items, size_t smem, cudaStream_t stream, bool pdl,
-                                           const MutPtrs& x, float* center, const float* beta, const Segment* segs, long long n,
-                                           int tile, int stages, int M, float pull, unsigned* counter, int* status)
+static cudaError_t launch_center_pull_bulk(bool per_layer, int grid, int item_begin, int item_end, size_t smem, cudaStream_t stream,
+                                           bool pdl, const MutPtrs& x, float* center, const float* beta, const Segment* segs,
+                                           long long n, int tile, int stages, int M, float pull, unsigned* counter, int* status)
 {
     auto kernel = per_layer ? center_pull_bulk_kernel<MT, true> : center_pull_bulk_kernel<MT, false>;
     cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(kBulkSmemBudget));
     if (err != cudaSuccess) return err;
-    return launch_kernel_smem(kernel, grid, kThreads, smem, stream, pdl, x, center, beta, segs, items, n, tile, stages, M, pull,
-                              counter, status);
+    return launch_kernel_smem(kernel, grid, kThreads, smem, stream, pdl, x, center, beta, segs, item_begin, item_end, n, tile, stages,
+                              M, pull, counter, status);
 }
 
 template <int MT>
@@ -319,37 +325,57 @@ struct CenterPullBulkDispatch<1> {
 };
 
 template <int M>
-static cudaError_t launch_center_pull(bool per_layer, int grid, int items, cudaStream_t stream, bool pdl, const MutPtrs& x,
-                                      float* center, const float* beta, const Segment* segs, long long n, int tile, float pull)
+static cudaError_t launch_center_pull(bool per_layer, int grid, int item_begin, int item_end, cudaStream_t stream, bool pdl,
+                                      const MutPtrs& x, float* center, const float* beta, const Segment* segs, long long n, int tile,
+                                      float pull)
 {
-    if (per_layer) return launch_kernel(center_pull_kernel<M, true>, grid, kThreads, stream, pdl, x, center, beta, segs, items, n, tile, pull, 1);
-    return launch_kernel(center_pull_kernel<M, false>, grid, kThreads, stream, pdl, x, center, beta, segs, items, n, tile, pull, 1);
+    if (per_layer)
+        return launch_kernel(center_pull_kernel<M, true>, grid, kThreads, stream, pdl, x, center, beta, segs, item_begin, item_end, n,
+                             tile, pull, 1);
+    return launch_kernel(center_pull_kernel<M, false>, grid, kThreads, stream, pdl, x, center, beta, segs, item_begin, item_end, n, tile,
+                         pull, 1);
 }
 
 template <int M>
 struct CenterPullDispatch {
-    static cudaError_t run(int m, bool per_layer, int grid, int items, cudaStream_t stream, bool pdl, const MutPtrs& x,
-                           float* center, const float* beta, const Segment* segs, long long n, int tile, float pull)
+    template <typename... A>
+    static cudaError_t run(int m, A&&... a)
     {
-        if (m == M) return launch_center_pull<M>(per_layer, grid, items, stream, pdl, x, center, beta, segs, n, tile, pull);
-        return CenterPullDispatch<M - 1>::run(m, per_layer, grid, items, stream, pdl, x, center, beta, segs, n, tile, pull);
+        if (m == M) return launch_center_pull<M>(static_cast<A&&>(a)...);
+        return CenterPullDispatch<M - 1>::run(m, static_cast<A&&>(a)...);
     }
 };
 template <>
 struct CenterPullDispatch<1> {
-    static cudaError_t run(int, bool, int, int, cudaStream_t, bool, const MutPtrs&, float*, const float*, const Segment*,
-                           long long, int, float)
+    template <typename... A>
+    static cudaError_t run(int, A&&...)
     {
         return cudaErrorInvalidValue;
     }
 };
 
-static grawa_status enqueue_step(int variant, float* const* params, const float* const* grads, int64_t n, int M,
-                                 float pull, const std::vector<int64_t>& off, float* center_out,
-                                 const grawa_options* opt, cudaStream_t stream, Plan* plan)
+// Device pointers and launch facts of one step, resolved once from the plan and the options.
+struct StepContext {
+    Plan* plan = nullptr;
+    int variant = 0, M = 0;
+    int64_t n = 0;
+    float pull = 0.f;
+    cudaStream_t stream = nullptr;
+    ConstPtrs gp{};
+    MutPtrs xp{};
+    float* center = nullptr;
+    bool vec_g = true, vec_x = true, pdl = false;
+    StepScratch sc{};
+    int* status = nullptr;
+    unsigned* counter = nullptr;
+    TimedStep* ts = nullptr;
+    int pull_items = 0;            // centre+pull work items of the whole vector
+};
+
+static grawa_status make_context(int variant, float* const* params, const float* const* grads, int64_t n, int M, float pull,
+                                 float* center_out, const grawa_options* opt, cudaStream_t stream, Plan* plan, StepContext* ctx)
 {
     const int K = plan->K;
-    // scratch
     char* ws = static_cast<char*>(opt ? opt->workspace : nullptr);
     if (ws) {
         if ((reinterpret_cast<uintptr_t>(ws) & 255u) || opt->workspace_bytes < plan->ws.total) return GRAWA_ERR_WORKSPACE;
@@ -358,86 +384,113 @@ static grawa_status enqueue_step(int variant, float* const* params, const float*
         if (!plan->d_ws) GRAWA_CUDA_TRY(cudaMalloc(&plan->d_ws, plan->ws.total));
         ws = static_cast<char*>(plan->d_ws);
     }
-    double* partials = reinterpret_cast<double*>(ws + plan->ws.partials);
-    double* S = reinterpret_cast<double*>(ws + plan->ws.S);
-    double* A = reinterpret_cast<double*>(ws + plan->ws.A);
-    float* beta = reinterpret_cast<float*>(ws + plan->ws.beta);
-    int* status = reinterpret_cast<int*>(ws + plan->ws.words) + 1;
-    unsigned* counter = reinterpret_cast<unsigned*>(ws + plan->ws.words) + 2;
-    g_last_status[{plan->device, stream}] = status;
-
-    ConstPtrs gp{};
-    MutPtrs xp{};
-    bool vec_g = true, vec_x = center_out == nullptr || aligned16(center_out);
+    ctx->plan = plan; ctx->variant = variant; ctx->M = M; ctx->n = n; ctx->pull = pull; ctx->stream = stream;
+    ctx->center = center_out;
+    ctx->status = reinterpret_cast<int*>(ws + plan->ws.words) + 1;
+    ctx->counter = reinterpret_cast<unsigned*>(ws + plan->ws.words) + 2;
+    g_last_status[{plan->device, stream}] = ctx->status;
+    ctx->vec_g = true;
+    ctx->vec_x = center_out == nullptr || aligned16(center_out);
     for (int m = 0; m < M; ++m) {
-        gp.p[m] = grads[m]; xp.p[m] = params[m];
-        vec_g = vec_g && aligned16(grads[m]);
-        vec_x = vec_x && aligned16(params[m]);
+        ctx->gp.p[m] = grads[m]; ctx->xp.p[m] = params[m];
+        ctx->vec_g = ctx->vec_g && aligned16(grads[m]);
+        ctx->vec_x = ctx->vec_x && aligned16(params[m]);
     }
+    StepScratch& sc = ctx->sc;
+    sc.segs = plan->d_segs1; sc.layer_seg_first = plan->d_layer_first;
+    sc.C = plan->C1; sc.K = K; sc.M = M; sc.variant = variant;
+    sc.partials = reinterpret_cast<double*>(ws + plan->ws.partials);
+    sc.S = reinterpret_cast<double*>(ws + plan->ws.S);
+    sc.A = reinterpret_cast<double*>(ws + plan->ws.A);
+    sc.beta = reinterpret_cast<float*>(ws + plan->ws.beta);
+    sc.layer_flag = plan->d_layer_flag;
+    sc.global_ticket = plan->d_tickets;
+    sc.global_target = static_cast<unsigned>(K);
+    sc.status = ctx->status; sc.work_counter = ctx->counter;
+    sc.weights_out = opt ? opt->weights_out : nullptr;
+    sc.scores_out = opt ? opt->scores_out : nullptr;
+    sc.sumsq_out = opt ? opt->sumsq_out : nullptr;
+    const int64_t tiles = variant == kLgrawa ? plan->C2 : (n + plan->tile2 - 1) / plan->tile2;
+    if (tiles > 0x7fffffffll) return GRAWA_ERR_INVALID_ARG;
+    ctx->pull_items = static_cast<int>(tiles);
+    ctx->ts = nullptr;
+    ctx->pdl = g_pdl != 0;
+    return GRAWA_OK;
+}
 
-    TimedStep* ts = nullptr;
+// Steps 1-3: sums of squares, scores, weights (two launches).
+static grawa_status enqueue_weights(StepContext& c)
+{
+    Plan* plan = c.plan;
+    const int items1 = plan->C1 * c.M;
+    const int grid1 = g_sumsq_ctas_per_sm > 0
+                          ? static_cast<int>(std::min<int64_t>(items1, g_sumsq_ctas_per_sm * plan->sm_count)) : items1;
+    GRAWA_CUDA_TRY(launch_kernel(sumsq_kernel<8>, grid1, kThreads, c.stream, c.pdl, c.gp, c.sc, items1, c.vec_g ? 1 : 0));
+    if (c.ts) GRAWA_CUDA_TRY(cudaEventRecord(c.ts->e[1], c.stream));
+    GRAWA_CUDA_TRY(launch_kernel(finalize_kernel, plan->K, kThreads, c.stream, c.pdl, c.sc));
+    if (c.ts) GRAWA_CUDA_TRY(cudaEventRecord(c.ts->e[2], c.stream));
+    return GRAWA_OK;
+}
+
+// Steps 4-5 on the work items [item_begin, item_end) (one launch).  M >= 2.
+static grawa_status enqueue_center_pull(StepContext& c, int item_begin, int item_end)
+{
+    Plan* plan = c.plan;
+    const int M = c.M;
+    const bool per_layer = c.variant == kLgrawa;
+    const int grid = item_end - item_begin;
+    if (grid <= 0) return GRAWA_OK;
+    const int tile = static_cast<int>(plan->tile2);
+    const float* beta = c.sc.beta;
+    // bulk-copy variant: asked for explicitly, or the only vector path for M > 16
+    const size_t stage_bytes = sizeof(float) * static_cast<size_t>(plan->tile2) * (M + 1);
+    const int stages = static_cast<int>(std::min<size_t>(kBulkMaxStages, kBulkSmemBudget / stage_bytes));
+    if (c.vec_x && plan->bulk && stages >= 2) {
+        const int gridb = std::min(grid, plan->sm_count);
+        GRAWA_CUDA_TRY(CenterPullBulkDispatch<kMaxRegWorkers>::run(M <= kMaxRegWorkers ? M : 1, per_layer, gridb, item_begin, item_end,
+                                                                   stage_bytes * stages, c.stream, c.pdl, c.xp, c.center, beta,
+                                                                   plan->d_segs2, c.n, tile, stages, M, c.pull, c.counter, c.status));
+    } else if (c.vec_x && M <= kMaxRegWorkers) {
+        const int grid2 = g_pull_ctas_per_sm > 0
+                              ? static_cast<int>(std::min<int64_t>(grid, g_pull_ctas_per_sm * plan->sm_count)) : grid;
+        GRAWA_CUDA_TRY(CenterPullDispatch<kMaxRegWorkers>::run(M, per_layer, grid2, item_begin, item_end, c.stream, c.pdl, c.xp,
+                                                               c.center, beta, plan->d_segs2, c.n, tile, c.pull));
+    } else {
+        GRAWA_CUDA_TRY(launch_kernel(center_pull_generic_kernel, grid, kThreads, c.stream, c.pdl, c.xp, c.center, beta, plan->d_segs2,
+                                     per_layer ? 1 : 0, item_begin, c.n, tile, c.pull, M));
+    }
+    return GRAWA_OK;
+}
+
+static grawa_status enqueue_step(int variant, float* const* params, const float* const* grads, int64_t n, int M,
+                                 float pull, float* center_out, const grawa_options* opt, cudaStream_t stream, Plan* plan)
+{
+    StepContext c;
+    grawa_status st = make_context(variant, params, grads, n, M, pull, center_out, opt, stream, plan, &c);
+    if (st != GRAWA_OK) return st;
     if (g_kernel_timing) {
         if (g_timed_used == g_timed_pool.size()) {
             TimedStep fresh{};
             for (auto& ev : fresh.e) GRAWA_CUDA_TRY(cudaEventCreate(&ev));
             g_timed_pool.push_back(fresh);
         }
-        ts = &g_timed_pool[g_timed_used++];
-        GRAWA_CUDA_TRY(cudaEventRecord(ts->e[0], stream));
+        c.ts = &g_timed_pool[g_timed_used++];
+        c.pdl = false;                               // event records between the kernels need plain ordering
+        GRAWA_CUDA_TRY(cudaEventRecord(c.ts->e[0], stream));
     }
-    const bool pdl = g_pdl != 0 && ts == nullptr;   // event records between the kernels need plain ordering
-    StepScratch sc{};
-    sc.segs = plan->d_segs1; sc.layer_seg_first = plan->d_layer_first;
-    sc.C = plan->C1; sc.K = K; sc.M = M; sc.variant = variant;
-    sc.partials = partials; sc.S = S; sc.A = A; sc.beta = beta; sc.layer_flag = plan->d_layer_flag;
-    sc.global_ticket = plan->d_tickets;
-    sc.global_target = static_cast<unsigned>(K);
-    sc.status = status; sc.work_counter = counter;
-    sc.weights_out = opt ? opt->weights_out : nullptr;
-    sc.scores_out = opt ? opt->scores_out : nullptr;
-    sc.sumsq_out = opt ? opt->sumsq_out : nullptr;
-    // step 1: partial sums of squares, one CTA per (worker, item)
-    const int items1 = plan->C1 * M;
-    const int grid1 = g_sumsq_ctas_per_sm > 0
-                          ? static_cast<int>(std::min<int64_t>(items1, g_sumsq_ctas_per_sm * plan->sm_count)) : items1;
-    GRAWA_CUDA_TRY(launch_kernel(sumsq_kernel<8>, grid1, kThreads, stream, pdl, gp, sc, items1, vec_g ? 1 : 0));
-    if (ts) GRAWA_CUDA_TRY(cudaEventRecord(ts->e[1], stream));
-    // steps 1b-3: S, scores, weights
-    GRAWA_CUDA_TRY(launch_kernel(finalize_kernel, K, kThreads, stream, pdl, sc));
-    if (ts) GRAWA_CUDA_TRY(cudaEventRecord(ts->e[2], stream));
-    // steps 4-5
+    st = enqueue_weights(c);
+    if (st != GRAWA_OK) return st;
     if (M == 1) {
         if (center_out) {
             const bool v = aligned16(center_out) && aligned16(params[0]);
             const int grid = static_cast<int>(std::min<int64_t>((n + kThreads * 4 - 1) / (kThreads * 4), 148 * 16));
-            GRAWA_CUDA_TRY(launch_kernel(copy_kernel, grid, kThreads, stream, pdl, params[0], center_out, n, v ? 1 : 0));
+            GRAWA_CUDA_TRY(launch_kernel(copy_kernel, grid, kThreads, stream, c.pdl, params[0], center_out, n, v ? 1 : 0));
         }
-        if (ts) GRAWA_CUDA_TRY(cudaEventRecord(ts->e[3], stream));
-        return GRAWA_OK;
-    }
-    const bool per_layer = variant == kLgrawa;
-    const int64_t tiles = per_layer ? plan->C2 : (n + plan->tile2 - 1) / plan->tile2;
-    if (tiles > 0x7fffffffll) return GRAWA_ERR_INVALID_ARG;
-    const int grid = static_cast<int>(tiles);
-    // bulk-copy variant: asked for explicitly, or the only vector path for M > 16
-    const size_t stage_bytes = sizeof(float) * static_cast<size_t>(plan->tile2) * (M + 1);
-    const int stages = static_cast<int>(std::min<size_t>(kBulkMaxStages, kBulkSmemBudget / stage_bytes));
-    if (vec_x && plan->bulk && stages >= 2) {
-        const int gridb = static_cast<int>(std::min<int64_t>(grid, plan->sm_count));
-        GRAWA_CUDA_TRY(CenterPullBulkDispatch<kMaxRegWorkers>::run(M <= kMaxRegWorkers ? M : 1, per_layer, gridb, grid,
-                                                                   stage_bytes * stages, stream, pdl, xp, center_out, beta,
-                                                                   plan->d_segs2, n, static_cast<int>(plan->tile2), stages, M, pull,
-                                                                   counter, status));
-    } else if (vec_x && M <= kMaxRegWorkers) {
-        const int grid2 = g_pull_ctas_per_sm > 0
-                              ? static_cast<int>(std::min<int64_t>(grid, g_pull_ctas_per_sm * plan->sm_count)) : grid;
-        GRAWA_CUDA_TRY(CenterPullDispatch<kMaxRegWorkers>::run(M, per_layer, grid2, grid, stream, pdl, xp, center_out, beta,
-                                                               plan->d_segs2, n, static_cast<int>(plan->tile2), pull));
     } else {
-        GRAWA_CUDA_TRY(launch_kernel(center_pull_generic_kernel, grid, kThreads, stream, pdl, xp, center_out, beta, plan->d_segs2,
-                                     per_layer ? 1 : 0, n, static_cast<int>(plan->tile2), pull, M));
+        st = enqueue_center_pull(c, 0, c.pull_items);
+        if (st != GRAWA_OK) return st;
     }
-    if (ts) GRAWA_CUDA_TRY(cudaEventRecord(ts->e[3], stream));
+    if (c.ts) GRAWA_CUDA_TRY(cudaEventRecord(c.ts->e[3], stream));
     return GRAWA_OK;
 }
 
@@ -453,7 +506,7 @@ static grawa_status step_entry(int variant, float* const* params, const float* c
     Plan* plan = nullptr;
     st = get_plan(n, M, off, stream, &plan);
     if (st != GRAWA_OK) return st;
-    return enqueue_step(variant, params, grads, n, M, pull, off, center_out, opt, stream, plan);
+    return enqueue_step(variant, params, grads, n, M, pull, center_out, opt, stream, plan);
 }
 
 // ------------------------------------------------------------------ allocation-free sum of squares
@@ -602,24 +655,64 @@ grawa_status grawa_step_host(grawa_variant variant, float* const* params, const 
     if (st != GRAWA_OK) return st;
     const size_t nn = align_up(static_cast<size_t>(n), 64);      // keeps every staged vector 256-byte aligned
     if (!plan->d_stage) GRAWA_CUDA_TRY(cudaMalloc(&plan->d_stage, sizeof(float) * nn * (2 * static_cast<size_t>(M) + 1)));
+    if (!plan->d2h_stream) GRAWA_CUDA_TRY(cudaStreamCreateWithFlags(&plan->d2h_stream, cudaStreamNonBlocking));
     std::vector<float*> dx(M);
     std::vector<const float*> dg(M);
     float* dc = plan->d_stage + nn * 2 * M;
     const size_t bytes = sizeof(float) * static_cast<size_t>(n);
     for (int m = 0; m < M; ++m) {
         dg[m] = plan->d_stage + nn * m;
+        dx[m] = plan->d_stage + nn * (M + m);
         GRAWA_CUDA_TRY(cudaMemcpyAsync(plan->d_stage + nn * m, grads[m], bytes, cudaMemcpyHostToDevice, stream));
     }
-    for (int m = 0; m < M; ++m) {
-        dx[m] = plan->d_stage + nn * (M + m);
-        GRAWA_CUDA_TRY(cudaMemcpyAsync(dx[m], params[m], bytes, cudaMemcpyHostToDevice, stream));
-    }
-    st = enqueue_step(variant, dx.data(), dg.data(), n, M, pull, off, center_out ? dc : nullptr, nullptr, stream, plan);
+    StepContext c;
+    st = make_context(variant, dx.data(), dg.data(), n, M, pull, center_out ? dc : nullptr, nullptr, stream, plan, &c);
     if (st != GRAWA_OK) return st;
-    if (M > 1)
+    st = enqueue_weights(c);                          // runs while the parameters are still arriving
+    if (st != GRAWA_OK) return st;
+    if (M == 1) {
+        // identity: the worker is untouched; the centre is the worker itself
+        if (center_out) std::memcpy(center_out, params[0], bytes);
+        GRAWA_CUDA_TRY(cudaStreamSynchronize(stream));
+        return GRAWA_OK;
+    }
+    // Centre+pull in chunks of work items: upload the chunk of all M workers, run it, and download
+    // its results on a second stream while the next chunk is being uploaded (the two directions of
+    // the host link work at the same time).
+    const bool per_layer = variant == kLgrawa;
+    const int items = c.pull_items;
+    const int64_t chunk_elems = std::max<int64_t>(int64_t{1} << 20, (n + 15) / 16);
+    auto item_begin_elem = [&](int i) -> int64_t {
+        if (i >= items) return n;
+        return per_layer ? plan->h_segs2[i].begin : static_cast<int64_t>(i) * plan->tile2;
+    };
+    size_t ev_used = 0;
+    int i0 = 0;
+    while (i0 < items) {
+        int i1 = i0 + 1;
+        const int64_t e0 = item_begin_elem(i0);
+        while (i1 < items && item_begin_elem(i1) - e0 < chunk_elems) ++i1;
+        const int64_t e1 = item_begin_elem(i1);
+        const size_t cb = sizeof(float) * static_cast<size_t>(e1 - e0);
         for (int m = 0; m < M; ++m)
-            GRAWA_CUDA_TRY(cudaMemcpyAsync(params[m], dx[m], bytes, cudaMemcpyDeviceToHost, stream));
-    if (center_out) GRAWA_CUDA_TRY(cudaMemcpyAsync(center_out, dc, bytes, cudaMemcpyDeviceToHost, stream));
+            GRAWA_CUDA_TRY(cudaMemcpyAsync(dx[m] + e0, params[m] + e0, cb, cudaMemcpyHostToDevice, stream));
+        if (plan->bulk) GRAWA_CUDA_TRY(cudaMemsetAsync(c.counter, 0, sizeof(unsigned), stream));
+        st = enqueue_center_pull(c, i0, i1);
+        if (st != GRAWA_OK) return st;
+        if (ev_used == plan->events.size()) {
+            cudaEvent_t ev;
+            GRAWA_CUDA_TRY(cudaEventCreateWithFlags(&ev, cudaEventDisableTiming));
+            plan->events.push_back(ev);
+        }
+        cudaEvent_t ev = plan->events[ev_used++];
+        GRAWA_CUDA_TRY(cudaEventRecord(ev, stream));
+        GRAWA_CUDA_TRY(cudaStreamWaitEvent(plan->d2h_stream, ev, 0));
+        for (int m = 0; m < M; ++m)
+            GRAWA_CUDA_TRY(cudaMemcpyAsync(params[m] + e0, dx[m] + e0, cb, cudaMemcpyDeviceToHost, plan->d2h_stream));
+        if (center_out) GRAWA_CUDA_TRY(cudaMemcpyAsync(center_out + e0, dc + e0, cb, cudaMemcpyDeviceToHost, plan->d2h_stream));
+        i0 = i1;
+    }
+    GRAWA_CUDA_TRY(cudaStreamSynchronize(plan->d2h_stream));
     GRAWA_CUDA_TRY(cudaStreamSynchronize(stream));
     return GRAWA_OK;
 }

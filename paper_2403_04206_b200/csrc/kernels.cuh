@@ -350,8 +350,8 @@ finalize_kernel(StepScratch sc)
 // parameter is read once and M independent vector loads are in flight per column.
 //   x_C = sum_m beta_m x_m   (fp32 FMA chain, m = 0..M-1)      x_m <- fmaf(pull, x_C, (1-pull) x_m)
 // PER_LAYER: the items are the Segments, weights of the segment's layer (Eq. 7); otherwise flat
-// tiles of `tile` elements and one weight per worker (Eq. 2 / Eq. 4).  CTA b takes items b,
-// b + gridDim.x, ...
+// tiles of `tile` elements and one weight per worker (Eq. 2 / Eq. 4).  The launch covers items
+// [item_begin, item_end); CTA b takes items item_begin + b, + gridDim.x, ...
 // ---------------------------------------------------------------------------------------------
 template <int M>
 __device__ __forceinline__ void pull_scalar(const MutPtrs& x, float* center, const float (&w)[M],
@@ -389,7 +389,8 @@ template <> struct VecIO<2> {
 template <int M, bool PER_LAYER>
 __global__ void __launch_bounds__(kThreads, 2)
 center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restrict__ beta,
-                   const Segment* __restrict__ segs, int items, long long n, int tile, float lambda, int vec_ok)
+                   const Segment* __restrict__ segs, int item_begin, int item_end, long long n, int tile, float lambda,
+                   int vec_ok)
 {
     grid_dependency_sync();
     constexpr int COLS = pull_cols(M);
@@ -401,7 +402,7 @@ center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restric
 #pragma unroll
         for (int m = 0; m < M; ++m) w[m] = beta[m];
     }
-    for (int item = blockIdx.x; item < items; item += gridDim.x) {
+    for (int item = item_begin + blockIdx.x; item < item_end; item += gridDim.x) {
         long long b, e;
         if (PER_LAYER) {
             const Segment sg = segs[item];
@@ -459,19 +460,19 @@ center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restric
 // (the second pass re-reads the elements the same thread has just read, from cache).
 __global__ void __launch_bounds__(kThreads)
 center_pull_generic_kernel(MutPtrs x, float* __restrict__ center, const float* __restrict__ beta,
-                           const Segment* __restrict__ segs, int per_layer, long long n, int tile,
-                           float lambda, int M)
+                           const Segment* __restrict__ segs, int per_layer, int item_begin, long long n,
+                           int tile, float lambda, int M)
 {
     grid_dependency_sync();
     long long b, e;
     const float* __restrict__ bt = beta;
     if (per_layer) {
-        const Segment sg = segs[blockIdx.x];
+        const Segment sg = segs[item_begin + blockIdx.x];
         b = sg.begin;
         e = b + sg.len;
         bt = beta + static_cast<size_t>(sg.layer) * M;
     } else {
-        b = static_cast<long long>(blockIdx.x) * tile;
+        b = static_cast<long long>(item_begin + blockIdx.x) * tile;
         e = min(n, b + tile);
     }
     __shared__ float w[kMaxWorkers];
