@@ -109,6 +109,18 @@ def pinned_inputs(cfg):
     return hp, hg
 
 
+def workload_config(args):
+    """The named workload, or (for small profiling captures) only its first --layers-limit layers
+    with the same value recipe."""
+    cfg = gen.CONFIGS[args.workload]
+    if args.layers_limit and args.layers_limit < cfg.K:
+        sizes = np.diff(cfg.offsets()[:args.layers_limit + 1])
+        cfg = gen.custom_config(sizes, cfg.M, seed=cfg.seed, pull=cfg.pull, grad_recipe=cfg.grad_recipe,
+                                log10_sigma=cfg.log10_sigma, loud_worker_factor=cfg.loud_worker_factor,
+                                name=f"{cfg.name}[first {args.layers_limit} layers]")
+    return cfg
+
+
 def step_fn(grawa, variant):
     return {"lgrawa": grawa.grawa_lgrawa_step, "mgrawa": grawa.grawa_mgrawa_step, "grawa": grawa.grawa_grawa_step}[variant]
 
@@ -188,6 +200,41 @@ def _oracle_sample(oracle, variant, p, g, pull, off):
         oracle.center_pull(p, beta, pull, off, j0, min(n, j0 + chunk), out=bufs)
 
 
+def max_over_ranks(values, world, device):
+    """Element-wise maximum of per-rank timings (the slowest rank defines the step time)."""
+    import torch
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_steps_per_s(world, ms_per_step_max):
+    """Replicas only: every rank runs the same workload, so the job does `world` steps per step time."""
+    return world * 1e3 / ms_per_step_max
+
+
+# DRAM traffic of one centre+pull launch, from the ncu capture summarised in
+# profiles/center_pull_kernel_vit_b16_28layers.md (M = 16; 1916.09 MB for 14 918 400 elements),
+# scaled to a full launch by the number of elements.  Only valid for the kernel source it was taken
+# from: the hash below is that of csrc/kernels.cuh at capture time, anything else reports null.
+TRAFFIC_CAPTURE = {"M": 16, "dram_bytes_per_element": 1916.086016e6 / 14918400,
+                   "kernels_sha256": "62cdcc12ea80c91ff8b853adb65108d333fe0d27591baaabcae7cdb5f62864a5"}
+
+
+def center_pull_traffic(cfg):
+    import hashlib
+    path = os.path.join(ROOT, "paper_2403_04206_b200", "csrc", "kernels.cuh")
+    try:
+        digest = hashlib.sha256(open(path, "rb").read()).hexdigest()
+    except OSError:
+        return None
+    if digest != TRAFFIC_CAPTURE["kernels_sha256"] or cfg.M != TRAFFIC_CAPTURE["M"]:
+        return None
+    return TRAFFIC_CAPTURE["dram_bytes_per_element"] * cfg.n
+
+
 def run_cuda(args):
     import torch
     import torch.distributed as dist
@@ -202,8 +249,11 @@ def run_cuda(args):
     import paper_2403_04206_b200 as grawa
     grawa.library()
 
-    cfg = gen.CONFIGS[args.workload]
+    cfg = workload_config(args)
     variant = args.variant
+    for kv in args.option:
+        name, value = kv.split("=")
+        grawa.grawa_set_option(name, int(value))
     hp, hg = pinned_inputs(cfg)
     x = [t.cuda(non_blocking=True) for t in hp]
     g = [t.cuda(non_blocking=True) for t in hg]
@@ -231,10 +281,7 @@ def run_cuda(args):
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
     e2e_ms = time_e2e_steps(grawa, cfg, variant, hp, hg, hc, e2e_steps, 1)
 
-    t = torch.tensor([ms, e2e_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_max, e2e_ms_max = float(t[0]), float(t[1])
+    ms_max, e2e_ms_max = max_over_ranks([ms, e2e_ms], world, "cuda")
 
     if rank == 0:
         peak, peak_src = measured_peak_gbs()
@@ -247,7 +294,7 @@ def run_cuda(args):
         achieved = pull_bytes / (pull_ms * 1e-3) / 1e9
         step_gbs = alg_bytes / (ms_max * 1e-3) / 1e9
         line = {
-            "metric": METRIC, "value": world * 1e3 / ms_max, "unit": "steps/s", "n_gpus": world,
+            "metric": METRIC, "value": whole_job_steps_per_s(world, ms_max), "unit": "steps/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_max, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
             "config": {"workload": f"{cfg.name} layer table, M={cfg.M} workers, n={cfg.n}, K={cfg.K} layers, "
@@ -260,7 +307,8 @@ def run_cuda(args):
                          "frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS},
             "roofline": {"bound": "hbm", "kernel": "center_pull", "achieved": achieved, "peak": peak,
                          "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
-                         "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "traffic": None,
+                         "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "traffic": center_pull_traffic(cfg),
+                         "traffic_source": "ncu dram bytes of a 14.9M-element capture at the same M, scaled by elements",
                          "algorithmic_bytes_per_launch": pull_bytes, "kernel_ms": pull_ms,
                          "timed_with": "library CUDA events around each kernel in a second K-step region",
                          "other_kernels": {
@@ -269,7 +317,7 @@ def run_cuda(args):
                                        "frac": sumsq_bytes / (sumsq_ms * 1e-3) / 1e9 / peak},
                              "finalize": {"kernel_ms": fin_ms}},
                          "ms_per_step_with_events": ms_k},
-            "e2e": {"value": world * 1e3 / e2e_ms_max, "unit": "steps/s", "steps": e2e_steps,
+            "e2e": {"value": whole_job_steps_per_s(world, e2e_ms_max), "unit": "steps/s", "steps": e2e_steps,
                     "h2d_bytes_per_step": 2 * cfg.M * 4 * cfg.n, "d2h_bytes_per_step": (cfg.M + 1) * 4 * cfg.n,
                     "entry_point": "grawa_step_host (pinned host buffers)"},
             "gpu_launches": launches, "clocks": clocks, "last_step_status": status,
@@ -317,7 +365,7 @@ def run_reference(args):
     if rank != 0:
         return
     import oracle
-    cfg = gen.CONFIGS[args.workload]
+    cfg = workload_config(args)
     variant = args.variant
     off = cfg.offsets()
     total = args.steps + args.warmup
@@ -371,6 +419,8 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--also", action="store_true", help="add short runs of the other large workloads/variants")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--layers-limit", type=int, default=0, help="use only the first L layers (small profiling captures)")
+    ap.add_argument("--option", action="append", default=[], help="library tuning knob, name=value (repeatable)")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
     if args.impl == "reference":

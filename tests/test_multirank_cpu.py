@@ -1,0 +1,55 @@
+"""The N > 1 path of bench.py on CPU: two gloo ranks.  The update itself does not shard
+("replicas only"), so what has to work across ranks is the timing reduction (max over ranks), the
+whole-job aggregate, and the reference arm's rule that only rank 0 works."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+import torch
+import torch.distributed as dist
+import torch.multiprocessing as mp
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+sys.path.insert(0, ROOT)
+
+
+def _worker(rank, world, port, out):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import bench
+    local = [2.0 + rank, 300.0 - 10 * rank]           # rank 1 is slower on the first, faster on the second
+    got = bench.max_over_ranks(local, world, "cpu")
+    dist.barrier()
+    out[rank] = got
+    dist.destroy_process_group()
+
+
+def test_timing_is_the_max_over_two_gloo_ranks():
+    with mp.Manager() as manager:
+        out = manager.dict()
+        mp.spawn(_worker, args=(2, 29533, out), nprocs=2, join=True)
+        assert out[0] == out[1] == [3.0, 300.0]
+    import bench
+    assert bench.whole_job_steps_per_s(2, 4.0) == 500.0      # two replicas, 4 ms per step
+    assert bench.max_over_ranks([1.5], 1, "cpu") == [1.5]
+
+
+def test_reference_arm_only_rank_zero_prints():
+    env = dict(os.environ, RANK="1", WORLD_SIZE="2", LOCAL_RANK="1")
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--gpus", "2",
+                          "--steps", "1", "--warmup", "0"], env=env, capture_output=True, text=True, timeout=120)
+    assert res.returncode == 0 and res.stdout.strip() == ""
+
+
+def test_reference_arm_line_has_the_contract_keys():
+    env = dict(os.environ, RANK="0", WORLD_SIZE="1")
+    res = subprocess.run([sys.executable, os.path.join(ROOT, "bench.py"), "--impl", "reference", "--workload", "toy10",
+                          "--steps", "2", "--warmup", "1"], env=env, capture_output=True, text=True, timeout=300)
+    assert res.returncode == 0, res.stderr
+    line = json.loads(res.stdout.strip().splitlines()[-1])
+    assert line["impl"] == "reference" and line["unit"] == "steps/s" and line["value"] > 0
+    assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] == 1
+    assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
+    assert line["higher_is_better"] is True and line["config"]["workload"].startswith("toy10")
