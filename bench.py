@@ -218,17 +218,20 @@ def whole_job_steps_per_s(world, ms_per_step_max):
 # DRAM traffic of one centre+pull launch, from the ncu capture summarised in
 # profiles/center_pull_kernel_vit_b16_28layers.md (M = 16; 1916.09 MB for 14 918 400 elements),
 # scaled to a full launch by the number of elements.  Only valid for the kernel source it was taken
-# from: the hash below is that of csrc/kernels.cuh at capture time, anything else reports null.
+# from: the hash below is that of the centre+pull kernel's text in csrc/kernels.cuh (from its
+# heading comment to the next kernel's) at capture time; anything else reports null.
 TRAFFIC_CAPTURE = {"M": 16, "dram_bytes_per_element": 1916.086016e6 / 14918400,
-                   "kernels_sha256": "62cdcc12ea80c91ff8b853adb65108d333fe0d27591baaabcae7cdb5f62864a5"}
+                   "kernels_sha256": "dfe4c7fc8a7a1661c74c90bc473b55c2492cfc82aca6445c50cd3cb601430930"}
 
 
 def center_pull_traffic(cfg):
     import hashlib
     path = os.path.join(ROOT, "paper_2403_04206_b200", "csrc", "kernels.cuh")
     try:
-        digest = hashlib.sha256(open(path, "rb").read()).hexdigest()
-    except OSError:
+        text = open(path).read()
+        region = text[text.index("// Steps 4-5, register variant"):text.index("// Steps 4-5 for any M up to")]
+        digest = hashlib.sha256(region.encode()).hexdigest()
+    except (OSError, ValueError):
         return None
     if digest != TRAFFIC_CAPTURE["kernels_sha256"] or cfg.M != TRAFFIC_CAPTURE["M"]:
         return None

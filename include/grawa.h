@@ -132,6 +132,34 @@ grawa_status grawa_last_step_status(grawa_stream_t stream);
 grawa_status grawa_prox_step(float *const *params, const float *center, int64_t n, int M,
                              float mu_over_tau, grawa_stream_t stream);
 
+/* The "Local" variants of the paper's appendix (Local MGRAWA / Local LGRAWA) take the norms from
+ * the local optimizer's own gradients instead of a dedicated batch.  Three calls cover them:
+ *
+ * grawa_layer_norms: norms_out[k] = ||grad[layer k]||_2 for ONE worker's gradient (the vector
+ * g_cur of that algorithm).  grad: DEVICE, n fp32, read only.  norms_out: DEVICE, n_layers doubles
+ * (1 when there is no layer table); empty layers give 0. */
+grawa_status grawa_layer_norms(const float *grad, int64_t n, const int64_t *layer_offsets, int n_layers,
+                               double *norms_out, grawa_stream_t stream);
+
+/* grawa_norm_ema: the running estimate, exactly as the appendix algorithm prints it:
+ *   g_mvg <- gamma g_mvg + (1 - gamma) g_cur ;  g_est <- gamma g_mvg / (1 - gamma^t)
+ * on DEVICE vectors of n_layers doubles (g_mvg in place; g_est may alias g_cur).  t >= 1 is the
+ * local iteration count since the last reset, gamma in [0, 1).  (The leading gamma of g_est is
+ * the paper's; it cancels in the weights when all workers share t.) */
+grawa_status grawa_norm_ema(double *g_mvg, const double *g_cur, int n_layers, double gamma, int64_t t,
+                            double *g_est, grawa_stream_t stream);
+
+/* grawa_step_from_layer_norms: the averaging step with the scores taken from given per-layer norms
+ * instead of gradients ("form x_C using the running gradient norm estimate"): layer_norms is
+ * DEVICE, [n_layers][M] doubles (row k holds the M workers' norm estimates of layer k).
+ * LGRAWA: A^k_m = layer_norms[k][m]; MGRAWA: A_m = sum_k layer_norms[k][m]; GRAWA:
+ * A_m = sqrt(sum_k layer_norms[k][m]^2).  Everything else as in the step entry points; no
+ * gradient is read (the step moves (2M+1)*4n bytes instead of (3M+1)*4n). */
+grawa_status grawa_step_from_layer_norms(grawa_variant variant, float *const *params, const double *layer_norms,
+                                         int64_t n, int M, float pull, const int64_t *layer_offsets,
+                                         int n_layers, float *center_out, const grawa_options *options,
+                                         grawa_stream_t stream);
+
 /* Largest number of partial sums grawa_sumsq_static can hold: M * ceil(n / 16384) must not
  * exceed it (for example M = 16 workers of up to 134 million elements each). */
 #define GRAWA_STATIC_MAX_PARTIALS 131072

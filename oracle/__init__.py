@@ -43,6 +43,8 @@ def _load():
         lib.grawa_oracle_sumsq.restype = None
         lib.grawa_oracle_scores.argtypes = [vp, ci, ci, ci, vp]
         lib.grawa_oracle_scores.restype = None
+        lib.grawa_oracle_scores_from_norms.argtypes = [vp, ci, ci, ci, vp]
+        lib.grawa_oracle_scores_from_norms.restype = None
         lib.grawa_oracle_weights.argtypes = [vp, ci, ci, vp]
         lib.grawa_oracle_weights.restype = ci
         lib.grawa_oracle_center_pull.argtypes = [vp, ci, vp, ci, vp, ci, i64, i64, dbl, vp, vp]
@@ -94,6 +96,16 @@ def scores(S, variant) -> np.ndarray:
     K, M = S.shape
     A = np.zeros((K, M) if v == LGRAWA else (M,), dtype=np.float64)
     _load().grawa_oracle_scores(S.ctypes.data, K, M, v, A.ctypes.data)
+    return A
+
+
+def scores_from_norms(norms, variant) -> np.ndarray:
+    """Step 2 from given per-layer norms [K, M] (the running estimates of the Local variants)."""
+    v = VARIANTS[variant] if isinstance(variant, str) else variant
+    N = np.ascontiguousarray(norms, dtype=np.float64)
+    K, M = N.shape
+    A = np.zeros((K, M) if v == LGRAWA else (M,), dtype=np.float64)
+    _load().grawa_oracle_scores_from_norms(N.ctypes.data, K, M, v, A.ctypes.data)
     return A
 
 

@@ -72,6 +72,29 @@ void grawa_oracle_scores(const double *S, int K, int M, int variant, double *A)
     }
 }
 
+/* Step 2 when the per-layer norms are given instead of gradients (the running estimates g_est of
+ * the Local variants, appendix algorithm: "form x_C using the running gradient norm estimate based
+ * on MGRAWA/LGRAWA policy").  N is [K][M].  LGRAWA: A^k_m = N[k][m]; MGRAWA: A_m = sum_k N[k][m]
+ * (Eq. 3 with the estimate in place of ||G_k||_F); GRAWA: A_m = sqrt(sum_k N[k][m]^2). */
+void grawa_oracle_scores_from_norms(const double *N, int K, int M, int variant, double *A)
+{
+    if (variant == ORACLE_LGRAWA) {
+        for (int i = 0; i < K * M; ++i) A[i] = N[i];
+    } else if (variant == ORACLE_MGRAWA) {
+        for (int m = 0; m < M; ++m) {
+            double a = 0.0;
+            for (int k = 0; k < K; ++k) a += N[(size_t)k * M + m];
+            A[m] = a;
+        }
+    } else {
+        for (int m = 0; m < M; ++m) {
+            double s = 0.0;
+            for (int k = 0; k < K; ++k) s += N[(size_t)k * M + m] * N[(size_t)k * M + m];
+            A[m] = sqrt(s);
+        }
+    }
+}
+
 /* Step 3 for one normalisation group of M scores.  Returns 1 when a non-finite
  * score was met (the fallback above was applied), else 0. */
 int grawa_oracle_weights_group(const double *A, int M, double *beta)

@@ -14,6 +14,9 @@ from .binding import (  # noqa: F401
     grawa_last_cuda_error,
     grawa_last_step_status,
     grawa_launch_count,
+    grawa_layer_norms,
+    grawa_norm_ema,
+    grawa_step_from_layer_norms,
     grawa_lgrawa_step,
     grawa_mgrawa_step,
     grawa_prox_step,

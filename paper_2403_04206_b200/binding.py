@@ -67,6 +67,12 @@ def library() -> ctypes.CDLL:
     lib.grawa_get_option.restype = i64
     lib.grawa_launch_count.restype = i64
     lib.grawa_clear_plans.restype = None
+    lib.grawa_layer_norms.argtypes = [vp, i64, vp, ci, vp, vp]
+    lib.grawa_layer_norms.restype = ci
+    lib.grawa_norm_ema.argtypes = [vp, vp, ci, ctypes.c_double, i64, vp, vp]
+    lib.grawa_norm_ema.restype = ci
+    lib.grawa_step_from_layer_norms.argtypes = [ci, vp, vp, i64, ci, cf, vp, ci, vp, vp, vp]
+    lib.grawa_step_from_layer_norms.restype = ci
     lib.grawa_sumsq_static.argtypes = [vp, i64, ci, vp, vp]
     lib.grawa_sumsq_static.restype = ci
     lib.grawa_collect_kernel_times.argtypes = [vp, vp, vp, vp]
@@ -199,6 +205,43 @@ def grawa_prox_step(params, center, mu_over_tau, *, stream=None, n=None) -> None
         n = _numel(center)
     _raise(lib.grawa_prox_step(_ptr_array(params), _addr(center), n, M, float(mu_over_tau), _stream(stream)),
            "grawa_prox_step")
+
+
+def grawa_layer_norms(grad, layer_offsets, norms_out, *, stream=None, n=None) -> None:
+    """Per-layer L2 norms of one worker's gradient into ``norms_out`` (device, K float64)."""
+    _check_f32([grad])
+    if n is None:
+        n = _numel(grad)
+    off, K = _offsets(layer_offsets)
+    _raise(library().grawa_layer_norms(_addr(grad), n, off.ctypes.data if off is not None else None, K,
+                                       _addr(norms_out), _stream(stream)), "grawa_layer_norms")
+
+
+def grawa_norm_ema(g_mvg, g_cur, gamma, t, g_est, *, stream=None) -> None:
+    """Running norm estimate of the Local variants on device float64 vectors (g_mvg updated in place)."""
+    _raise(library().grawa_norm_ema(_addr(g_mvg), _addr(g_cur), _numel(g_mvg), float(gamma), int(t), _addr(g_est),
+                                    _stream(stream)), "grawa_norm_ema")
+
+
+def grawa_step_from_layer_norms(variant, params, layer_norms, pull, layer_offsets=None, center_out=None, *,
+                                weights_out=None, scores_out=None, sumsq_out=None, workspace=None, stream=None,
+                                n=None) -> None:
+    """Averaging step with scores from given per-layer norms ([K, M] device float64) instead of gradients."""
+    lib = library()
+    v = _VARIANTS[variant] if isinstance(variant, str) else int(variant)
+    _check_f32(list(params) + ([center_out] if center_out is not None else []))
+    M = len(params)
+    if n is None:
+        n = _numel(params[0]) if M else 0
+    off, K = _offsets(layer_offsets)
+    opt = None
+    if any(b is not None for b in (weights_out, scores_out, sumsq_out, workspace)):
+        ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+        opt = _Options(_addr(weights_out), _addr(scores_out), _addr(sumsq_out), _addr(workspace), ws_bytes)
+    _raise(lib.grawa_step_from_layer_norms(v, _ptr_array(params), _addr(layer_norms), n, M, float(pull),
+                                           off.ctypes.data if off is not None else None, K, _addr(center_out),
+                                           ctypes.byref(opt) if opt is not None else None, _stream(stream)),
+           "grawa_step_from_layer_norms")
 
 
 def grawa_sumsq_static(grads, sumsq_out, *, stream=None, n=None) -> None:

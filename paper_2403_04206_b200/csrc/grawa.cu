@@ -392,8 +392,8 @@ static grawa_status make_context(int variant, float* const* params, const float*
     ctx->vec_g = true;
     ctx->vec_x = center_out == nullptr || aligned16(center_out);
     for (int m = 0; m < M; ++m) {
-        ctx->gp.p[m] = grads[m]; ctx->xp.p[m] = params[m];
-        ctx->vec_g = ctx->vec_g && aligned16(grads[m]);
+        ctx->gp.p[m] = grads ? grads[m] : nullptr; ctx->xp.p[m] = params[m];
+        ctx->vec_g = ctx->vec_g && grads && aligned16(grads[m]);
         ctx->vec_x = ctx->vec_x && aligned16(params[m]);
     }
     StepScratch& sc = ctx->sc;
@@ -410,6 +410,7 @@ static grawa_status make_context(int variant, float* const* params, const float*
     sc.weights_out = opt ? opt->weights_out : nullptr;
     sc.scores_out = opt ? opt->scores_out : nullptr;
     sc.sumsq_out = opt ? opt->sumsq_out : nullptr;
+    sc.layer_norms = nullptr;
     const int64_t tiles = variant == kLgrawa ? plan->C2 : (n + plan->tile2 - 1) / plan->tile2;
     if (tiles > 0x7fffffffll) return GRAWA_ERR_INVALID_ARG;
     ctx->pull_items = static_cast<int>(tiles);
@@ -422,6 +423,12 @@ static grawa_status make_context(int variant, float* const* params, const float*
 static grawa_status enqueue_weights(StepContext& c)
 {
     Plan* plan = c.plan;
+    if (c.sc.layer_norms != nullptr) {               // scores are given: no pass over gradients
+        if (c.ts) GRAWA_CUDA_TRY(cudaEventRecord(c.ts->e[1], c.stream));
+        GRAWA_CUDA_TRY(launch_kernel(finalize_kernel, plan->K, kThreads, c.stream, c.pdl, c.sc));
+        if (c.ts) GRAWA_CUDA_TRY(cudaEventRecord(c.ts->e[2], c.stream));
+        return GRAWA_OK;
+    }
     const int items1 = plan->C1 * c.M;
     const int grid1 = g_sumsq_ctas_per_sm > 0
                           ? static_cast<int>(std::min<int64_t>(items1, g_sumsq_ctas_per_sm * plan->sm_count)) : items1;
@@ -462,12 +469,14 @@ static grawa_status enqueue_center_pull(StepContext& c, int item_begin, int item
     return GRAWA_OK;
 }
 
-static grawa_status enqueue_step(int variant, float* const* params, const float* const* grads, int64_t n, int M,
-                                 float pull, float* center_out, const grawa_options* opt, cudaStream_t stream, Plan* plan)
+static grawa_status enqueue_step(int variant, float* const* params, const float* const* grads, const double* layer_norms,
+                                 int64_t n, int M, float pull, float* center_out, const grawa_options* opt,
+                                 cudaStream_t stream, Plan* plan)
 {
     StepContext c;
     grawa_status st = make_context(variant, params, grads, n, M, pull, center_out, opt, stream, plan, &c);
     if (st != GRAWA_OK) return st;
+    c.sc.layer_norms = layer_norms;
     if (g_kernel_timing) {
         if (g_timed_used == g_timed_pool.size()) {
             TimedStep fresh{};
@@ -494,11 +503,11 @@ static grawa_status enqueue_step(int variant, float* const* params, const float*
     return GRAWA_OK;
 }
 
-static grawa_status step_entry(int variant, float* const* params, const float* const* grads, int64_t n, int M, float pull,
-                               const int64_t* layer_offsets, int n_layers, float* center_out, const grawa_options* opt,
-                               cudaStream_t stream)
+static grawa_status step_entry(int variant, float* const* params, const float* const* grads, const double* layer_norms,
+                               int64_t n, int M, float pull, const int64_t* layer_offsets, int n_layers, float* center_out,
+                               const grawa_options* opt, cudaStream_t stream)
 {
-    if (grads == nullptr) return GRAWA_ERR_INVALID_ARG;
+    if ((grads == nullptr) == (layer_norms == nullptr)) return GRAWA_ERR_INVALID_ARG;   // exactly one source of scores
     std::vector<int64_t> off;
     grawa_status st = validate(params, grads, n, M, pull, layer_offsets, n_layers, center_out, &off);
     if (st != GRAWA_OK || n == 0) return st;
@@ -506,7 +515,7 @@ static grawa_status step_entry(int variant, float* const* params, const float* c
     Plan* plan = nullptr;
     st = get_plan(n, M, off, stream, &plan);
     if (st != GRAWA_OK) return st;
-    return enqueue_step(variant, params, grads, n, M, pull, center_out, opt, stream, plan);
+    return enqueue_step(variant, params, grads, layer_norms, n, M, pull, center_out, opt, stream, plan);
 }
 
 // ------------------------------------------------------------------ allocation-free sum of squares
@@ -622,21 +631,65 @@ grawa_status grawa_mgrawa_step(float* const* params, const float* const* grads, 
                                const int64_t* layer_offsets, int n_layers, float* center_out,
                                const grawa_options* options, grawa_stream_t stream)
 {
-    return step_entry(kMgrawa, params, grads, n, M, pull, layer_offsets, n_layers, center_out, options, stream);
+    return step_entry(kMgrawa, params, grads, nullptr, n, M, pull, layer_offsets, n_layers, center_out, options, stream);
 }
 
 grawa_status grawa_grawa_step(float* const* params, const float* const* grads, int64_t n, int M, float pull,
                               const int64_t* layer_offsets, int n_layers, float* center_out,
                               const grawa_options* options, grawa_stream_t stream)
 {
-    return step_entry(kGrawa, params, grads, n, M, pull, layer_offsets, n_layers, center_out, options, stream);
+    return step_entry(kGrawa, params, grads, nullptr, n, M, pull, layer_offsets, n_layers, center_out, options, stream);
 }
 
 grawa_status grawa_lgrawa_step(float* const* params, const float* const* grads, int64_t n, int M, float pull,
                                const int64_t* layer_offsets, int n_layers, float* center_out,
                                const grawa_options* options, grawa_stream_t stream)
 {
-    return step_entry(kLgrawa, params, grads, n, M, pull, layer_offsets, n_layers, center_out, options, stream);
+    return step_entry(kLgrawa, params, grads, nullptr, n, M, pull, layer_offsets, n_layers, center_out, options, stream);
+}
+
+grawa_status grawa_step_from_layer_norms(grawa_variant variant, float* const* params, const double* layer_norms, int64_t n,
+                                         int M, float pull, const int64_t* layer_offsets, int n_layers, float* center_out,
+                                         const grawa_options* options, grawa_stream_t stream)
+{
+    if (variant != GRAWA_VARIANT_GRAWA && variant != GRAWA_VARIANT_MGRAWA && variant != GRAWA_VARIANT_LGRAWA)
+        return GRAWA_ERR_INVALID_ARG;
+    return step_entry(static_cast<int>(variant), params, nullptr, layer_norms, n, M, pull, layer_offsets, n_layers, center_out,
+                      options, stream);
+}
+
+grawa_status grawa_layer_norms(const float* grad, int64_t n, const int64_t* layer_offsets, int n_layers, double* norms_out,
+                               grawa_stream_t stream)
+{
+    if (grad == nullptr || norms_out == nullptr || n < 0 || (reinterpret_cast<uintptr_t>(grad) & 3u)) return GRAWA_ERR_INVALID_ARG;
+    // validate() wants a parameter vector; the gradient stands in (nothing is written through it)
+    float* fake_params[1] = {const_cast<float*>(grad)};
+    std::vector<int64_t> off;
+    grawa_status st = validate(fake_params, nullptr, n, 1, 0.0f, layer_offsets, n_layers, nullptr, &off);
+    if (st != GRAWA_OK || n == 0) return st;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    Plan* plan = nullptr;
+    st = get_plan(n, 1, off, stream, &plan);
+    if (st != GRAWA_OK) return st;
+    grawa_options opt{};
+    opt.scores_out = norms_out;
+    const float* grads[1] = {grad};
+    StepContext c;
+    st = make_context(kLgrawa, fake_params, grads, n, 1, 0.0f, nullptr, &opt, stream, plan, &c);
+    if (st != GRAWA_OK) return st;
+    return enqueue_weights(c);
+}
+
+grawa_status grawa_norm_ema(double* g_mvg, const double* g_cur, int n_layers, double gamma, int64_t t, double* g_est,
+                            grawa_stream_t stream)
+{
+    if (g_mvg == nullptr || g_cur == nullptr || g_est == nullptr || n_layers < 0 || t < 1) return GRAWA_ERR_INVALID_ARG;
+    if (!(gamma >= 0.0 && gamma < 1.0)) return GRAWA_ERR_INVALID_ARG;
+    if (n_layers == 0) return GRAWA_OK;
+    const double corr = 1.0 - std::pow(gamma, static_cast<double>(t));
+    GRAWA_CUDA_TRY(launch_kernel(norm_ema_kernel, (n_layers + kThreads - 1) / kThreads, kThreads, stream, false, g_mvg, g_cur,
+                                 n_layers, gamma, corr, g_est));
+    return GRAWA_OK;
 }
 
 grawa_status grawa_step_host(grawa_variant variant, float* const* params, const float* const* grads, int64_t n, int M,

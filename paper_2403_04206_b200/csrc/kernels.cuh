@@ -92,6 +92,7 @@ struct StepScratch {
     unsigned global_target;        // arrivals that complete the step's finalisation
     int* status;                   // written (not or-ed) when the finalisation completes
     unsigned* work_counter;        // cleared for the bulk-copy centre+pull kernel
+    const double* layer_norms;     // [K][M] given per-layer norms (steps from scores), else NULL
     float* weights_out;            // optional copies
     double* scores_out;
     double* sumsq_out;
@@ -142,35 +143,46 @@ struct FinalizeSmem {
 // Steps 1b-3 for one non-empty layer, by a whole CTA of kThreads threads.  Warp w adds the partials
 // of workers w, w+8, ... of layer k in a fixed order into S[k][m]; the layer's terms sqrt(S) (S
 // itself for the flat norm) go to row k of A; LGRAWA turns them into the layer's weights (Eq. 7).
+// With layer_norms set the sums are not needed: the given norm of (layer, worker) takes the place
+// of sqrt(S) (the running estimates of the Local variants).
 __device__ __forceinline__ void finalize_layer(const StepScratch& sc, int k, FinalizeSmem& sm)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int M = sc.M;
-    const int s0 = sc.layer_seg_first[k], s1 = sc.layer_seg_first[k + 1];
-    for (int m = warp; m < M; m += kThreads / 32) {
-        const double* row = sc.partials + static_cast<size_t>(m) * sc.C;
-        // eight independent running sums per lane keep eight loads in flight; the order in which
-        // they are combined is fixed, so the sum is the same on every run
-        double part[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
-        int s = s0 + lane;
-        for (; s + 7 * 32 < s1; s += 8 * 32) {
+    if (sc.layer_norms == nullptr) {
+        const int s0 = sc.layer_seg_first[k], s1 = sc.layer_seg_first[k + 1];
+        for (int m = warp; m < M; m += kThreads / 32) {
+            const double* row = sc.partials + static_cast<size_t>(m) * sc.C;
+            // eight independent running sums per lane keep eight loads in flight; the order in which
+            // they are combined is fixed, so the sum is the same on every run
+            double part[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
+            int s = s0 + lane;
+            for (; s + 7 * 32 < s1; s += 8 * 32) {
 #pragma unroll
-            for (int u = 0; u < 8; ++u) part[u] += __ldcg(row + s + u * 32);
+                for (int u = 0; u < 8; ++u) part[u] += __ldcg(row + s + u * 32);
+            }
+            for (int u = 0; s < s1; s += 32, ++u) part[u] += __ldcg(row + s);
+            double acc = ((part[0] + part[1]) + (part[2] + part[3])) + ((part[4] + part[5]) + (part[6] + part[7]));
+#pragma unroll
+            for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, d);
+            if (lane == 0) sm.layer_sum[m] = acc;
         }
-        for (int u = 0; s < s1; s += 32, ++u) part[u] += __ldcg(row + s);
-        double acc = ((part[0] + part[1]) + (part[2] + part[3])) + ((part[4] + part[5]) + (part[6] + part[7]));
-#pragma unroll
-        for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, d);
-        if (lane == 0) sm.layer_sum[m] = acc;
     }
     __syncthreads();
     double term = 0.0;
     const size_t idx = static_cast<size_t>(k) * M + tid;
     if (tid < M) {
-        const double s = sm.layer_sum[tid];
+        double s;
+        if (sc.layer_norms == nullptr) {
+            s = sm.layer_sum[tid];
+            term = (sc.variant == kGrawa) ? s : sqrt(s);
+        } else {                                   // the caller's norm estimate stands in for sqrt(S)
+            const double a = sc.layer_norms[idx];
+            s = a * a;
+            term = (sc.variant == kGrawa) ? s : a;
+        }
         sc.S[idx] = s;
         if (sc.sumsq_out) sc.sumsq_out[idx] = s;
-        term = (sc.variant == kGrawa) ? s : sqrt(s);
         sc.A[idx] = term;
     }
     if (sc.variant == kLgrawa) {
@@ -484,6 +496,21 @@ center_pull_generic_kernel(MutPtrs x, float* __restrict__ center, const float* _
         for (int m = 1; m < M; ++m) c = fmaf(w[m], x.p[m][i], c);
         if (center) center[i] = c;
         for (int m = 0; m < M; ++m) x.p[m][i] = fmaf(lambda, c, oml * x.p[m][i]);
+    }
+}
+
+// Running gradient-norm estimate of the Local variants (appendix algorithm, taken literally):
+// g_mvg <- gamma g_mvg + (1-gamma) g_cur ; g_est <- gamma g_mvg / corr, corr = 1 - gamma^t.
+__global__ void __launch_bounds__(kThreads)
+norm_ema_kernel(double* __restrict__ g_mvg, const double* __restrict__ g_cur, int K, double gamma, double corr,
+                double* __restrict__ g_est)
+{
+    grid_dependency_sync();
+    const int k = blockIdx.x * kThreads + threadIdx.x;
+    if (k < K) {
+        const double v = gamma * g_mvg[k] + (1.0 - gamma) * g_cur[k];
+        g_mvg[k] = v;
+        g_est[k] = gamma * v / corr;
     }
 }
 

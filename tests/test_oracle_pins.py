@@ -335,3 +335,33 @@ def test_norm_ema_constant_input_closed_form():
         est = oracle.norm_ema(mvg, c, gamma, t)
         assert np.allclose(mvg, (1 - gamma ** t) * c, rtol=1e-13)
         assert np.allclose(est, gamma * c, rtol=1e-13)
+
+
+def test_scores_from_norms_match_scores_from_sums():
+    """Given the exact layer norms, the from-norms scores are the from-gradients scores."""
+    sizes = [5, 17, 1, 300]
+    off = np.concatenate([[0], np.cumsum(sizes)])
+    g = [f32(rng.normal(size=off[-1]) * s) for s in (0.1, 1.0, 7.0)]
+    S = oracle.sumsq(g, off)
+    N = np.sqrt(S)
+    assert np.array_equal(oracle.scores_from_norms(N, "lgrawa"), oracle.scores(S, "lgrawa"))
+    assert np.array_equal(oracle.scores_from_norms(N, "mgrawa"), oracle.scores(S, "mgrawa"))
+    assert np.allclose(oracle.scores_from_norms(N, "grawa"), oracle.scores(S, "grawa"), rtol=1e-14)
+    # hand case: norms (3, 4) and (6, 8) over two layers -> MGRAWA (7, 14), GRAWA (5, 10), LGRAWA as given
+    N = np.array([[3.0, 6.0], [4.0, 8.0]])
+    assert np.array_equal(oracle.scores_from_norms(N, "mgrawa"), [7, 14])
+    assert np.array_equal(oracle.scores_from_norms(N, "grawa"), [5, 10])
+    assert np.array_equal(oracle.scores_from_norms(N, "lgrawa"), N)
+
+
+def test_norm_ema_bias_correction_cancels_in_the_weights():
+    """All workers share t, so the literal estimate (with its leading gamma) gives the same weights
+    as the plain moving value: beta only sees ratios."""
+    gamma = 0.8
+    cur = rng.uniform(0.5, 2.0, size=(4, 3))            # 4 steps, 3 workers, one layer
+    mvg = np.zeros((3, 1))
+    for t in range(1, 5):
+        est = np.stack([oracle.norm_ema(mvg[m], cur[t - 1, m:m + 1], gamma, t) for m in range(3)])
+    beta_est = oracle.weights(est[:, 0])[0]
+    beta_mvg = oracle.weights(mvg[:, 0])[0]
+    assert np.allclose(beta_est, beta_mvg, rtol=1e-13)
