@@ -160,6 +160,25 @@ grawa_status grawa_step_from_layer_norms(grawa_variant variant, float *const *pa
                                          int n_layers, float *center_out, const grawa_options *options,
                                          grawa_stream_t stream);
 
+/* Element-range sharding over several GPUs (each GPU holds the same index range of all M
+ * replicas; derived from Eq. 3-7: sums of squares add over disjoint index ranges).  Two calls, with
+ * one all-gather of a [n_layers][M] table of doubles between them (the caller's, e.g. NCCL):
+ *
+ * grawa_layer_sumsq: sumsq_out[k][m] = sum over the LOCAL elements of layer k of grads[m][j]^2.
+ * grads: HOST array of M DEVICE pointers (n local elements each); layer_offsets: the local layer
+ * table (layers without local elements are empty layers); sumsq_out: DEVICE, [n_layers][M]. */
+grawa_status grawa_layer_sumsq(const float *const *grads, int64_t n, int M, const int64_t *layer_offsets,
+                               int n_layers, double *sumsq_out, grawa_stream_t stream);
+
+/* grawa_step_from_layer_sums: the averaging step on the local elements with S[k][m] = the sum, in
+ * part order (so every GPU gets the same bits), of layer_sums[r][k][m], r = 0..parts-1.
+ * layer_sums: DEVICE, [parts][n_layers][M] doubles, e.g. the all-gathered tables of all ranks.
+ * Scores, weights, centre and pull follow as in the step entry points; no gradient is read. */
+grawa_status grawa_step_from_layer_sums(grawa_variant variant, float *const *params, const double *layer_sums,
+                                        int parts, int64_t n, int M, float pull, const int64_t *layer_offsets,
+                                        int n_layers, float *center_out, const grawa_options *options,
+                                        grawa_stream_t stream);
+
 /* Largest number of partial sums grawa_sumsq_static can hold: M * ceil(n / 16384) must not
  * exceed it (for example M = 16 workers of up to 134 million elements each). */
 #define GRAWA_STATIC_MAX_PARTIALS 131072

@@ -15,6 +15,8 @@ from .binding import (  # noqa: F401
     grawa_last_step_status,
     grawa_launch_count,
     grawa_layer_norms,
+    grawa_layer_sumsq,
+    grawa_step_from_layer_sums,
     grawa_norm_ema,
     grawa_step_from_layer_norms,
     grawa_lgrawa_step,

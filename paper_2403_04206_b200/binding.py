@@ -73,6 +73,10 @@ def library() -> ctypes.CDLL:
     lib.grawa_norm_ema.restype = ci
     lib.grawa_step_from_layer_norms.argtypes = [ci, vp, vp, i64, ci, cf, vp, ci, vp, vp, vp]
     lib.grawa_step_from_layer_norms.restype = ci
+    lib.grawa_layer_sumsq.argtypes = [vp, i64, ci, vp, ci, vp, vp]
+    lib.grawa_layer_sumsq.restype = ci
+    lib.grawa_step_from_layer_sums.argtypes = [ci, vp, vp, ci, i64, ci, cf, vp, ci, vp, vp, vp]
+    lib.grawa_step_from_layer_sums.restype = ci
     lib.grawa_sumsq_static.argtypes = [vp, i64, ci, vp, vp]
     lib.grawa_sumsq_static.restype = ci
     lib.grawa_collect_kernel_times.argtypes = [vp, vp, vp, vp]
@@ -242,6 +246,38 @@ def grawa_step_from_layer_norms(variant, params, layer_norms, pull, layer_offset
                                            off.ctypes.data if off is not None else None, K, _addr(center_out),
                                            ctypes.byref(opt) if opt is not None else None, _stream(stream)),
            "grawa_step_from_layer_norms")
+
+
+def grawa_layer_sumsq(grads, layer_offsets, sumsq_out, *, stream=None, n=None) -> None:
+    """Per-layer sums of squares of the M workers' local gradients into ``sumsq_out`` ([K, M] device float64)."""
+    _check_f32(list(grads))
+    M = len(grads)
+    if n is None:
+        n = _numel(grads[0]) if M else 0
+    off, K = _offsets(layer_offsets)
+    _raise(library().grawa_layer_sumsq(_ptr_array(grads), n, M, off.ctypes.data if off is not None else None, K,
+                                       _addr(sumsq_out), _stream(stream)), "grawa_layer_sumsq")
+
+
+def grawa_step_from_layer_sums(variant, params, layer_sums, parts, pull, layer_offsets=None, center_out=None, *,
+                               weights_out=None, scores_out=None, sumsq_out=None, workspace=None, stream=None,
+                               n=None) -> None:
+    """Averaging step on local elements with S = sum over ``parts`` tables of ``layer_sums`` ([parts, K, M])."""
+    lib = library()
+    v = _VARIANTS[variant] if isinstance(variant, str) else int(variant)
+    _check_f32(list(params) + ([center_out] if center_out is not None else []))
+    M = len(params)
+    if n is None:
+        n = _numel(params[0]) if M else 0
+    off, K = _offsets(layer_offsets)
+    opt = None
+    if any(b is not None for b in (weights_out, scores_out, sumsq_out, workspace)):
+        ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+        opt = _Options(_addr(weights_out), _addr(scores_out), _addr(sumsq_out), _addr(workspace), ws_bytes)
+    _raise(lib.grawa_step_from_layer_sums(v, _ptr_array(params), _addr(layer_sums), int(parts), n, M, float(pull),
+                                          off.ctypes.data if off is not None else None, K, _addr(center_out),
+                                          ctypes.byref(opt) if opt is not None else None, _stream(stream)),
+           "grawa_step_from_layer_sums")
 
 
 def grawa_sumsq_static(grads, sumsq_out, *, stream=None, n=None) -> None:

@@ -410,7 +410,7 @@ static grawa_status make_context(int variant, float* const* params, const float*
     sc.weights_out = opt ? opt->weights_out : nullptr;
     sc.scores_out = opt ? opt->scores_out : nullptr;
     sc.sumsq_out = opt ? opt->sumsq_out : nullptr;
-    sc.layer_norms = nullptr;
+    sc.given = nullptr; sc.given_parts = 1; sc.given_sums = 0;
     const int64_t tiles = variant == kLgrawa ? plan->C2 : (n + plan->tile2 - 1) / plan->tile2;
     if (tiles > 0x7fffffffll) return GRAWA_ERR_INVALID_ARG;
     ctx->pull_items = static_cast<int>(tiles);
@@ -423,7 +423,7 @@ static grawa_status make_context(int variant, float* const* params, const float*
 static grawa_status enqueue_weights(StepContext& c)
 {
     Plan* plan = c.plan;
-    if (c.sc.layer_norms != nullptr) {               // scores are given: no pass over gradients
+    if (c.sc.given != nullptr) {                     // scores are given: no pass over gradients
         if (c.ts) GRAWA_CUDA_TRY(cudaEventRecord(c.ts->e[1], c.stream));
         GRAWA_CUDA_TRY(launch_kernel(finalize_kernel, plan->K, kThreads, c.stream, c.pdl, c.sc));
         if (c.ts) GRAWA_CUDA_TRY(cudaEventRecord(c.ts->e[2], c.stream));
@@ -469,14 +469,21 @@ static grawa_status enqueue_center_pull(StepContext& c, int item_begin, int item
     return GRAWA_OK;
 }
 
-static grawa_status enqueue_step(int variant, float* const* params, const float* const* grads, const double* layer_norms,
+// Given scores of a step that reads no gradients: per-layer norms, or `parts` sets of per-layer sums.
+struct GivenScores {
+    const double* data = nullptr;
+    int parts = 1;
+    int sums = 0;
+};
+
+static grawa_status enqueue_step(int variant, float* const* params, const float* const* grads, const GivenScores& given,
                                  int64_t n, int M, float pull, float* center_out, const grawa_options* opt,
                                  cudaStream_t stream, Plan* plan)
 {
     StepContext c;
     grawa_status st = make_context(variant, params, grads, n, M, pull, center_out, opt, stream, plan, &c);
     if (st != GRAWA_OK) return st;
-    c.sc.layer_norms = layer_norms;
+    c.sc.given = given.data; c.sc.given_parts = given.parts; c.sc.given_sums = given.sums;
     if (g_kernel_timing) {
         if (g_timed_used == g_timed_pool.size()) {
             TimedStep fresh{};
@@ -503,11 +510,12 @@ static grawa_status enqueue_step(int variant, float* const* params, const float*
     return GRAWA_OK;
 }
 
-static grawa_status step_entry(int variant, float* const* params, const float* const* grads, const double* layer_norms,
+static grawa_status step_entry(int variant, float* const* params, const float* const* grads, const GivenScores& given,
                                int64_t n, int M, float pull, const int64_t* layer_offsets, int n_layers, float* center_out,
                                const grawa_options* opt, cudaStream_t stream)
 {
-    if ((grads == nullptr) == (layer_norms == nullptr)) return GRAWA_ERR_INVALID_ARG;   // exactly one source of scores
+    if ((grads == nullptr) == (given.data == nullptr)) return GRAWA_ERR_INVALID_ARG;   // exactly one source of scores
+    if (given.parts < 1) return GRAWA_ERR_INVALID_ARG;
     std::vector<int64_t> off;
     grawa_status st = validate(params, grads, n, M, pull, layer_offsets, n_layers, center_out, &off);
     if (st != GRAWA_OK || n == 0) return st;
@@ -515,7 +523,7 @@ static grawa_status step_entry(int variant, float* const* params, const float* c
     Plan* plan = nullptr;
     st = get_plan(n, M, off, stream, &plan);
     if (st != GRAWA_OK) return st;
-    return enqueue_step(variant, params, grads, layer_norms, n, M, pull, center_out, opt, stream, plan);
+    return enqueue_step(variant, params, grads, given, n, M, pull, center_out, opt, stream, plan);
 }
 
 // ------------------------------------------------------------------ allocation-free sum of squares
@@ -631,21 +639,21 @@ grawa_status grawa_mgrawa_step(float* const* params, const float* const* grads, 
                                const int64_t* layer_offsets, int n_layers, float* center_out,
                                const grawa_options* options, grawa_stream_t stream)
 {
-    return step_entry(kMgrawa, params, grads, nullptr, n, M, pull, layer_offsets, n_layers, center_out, options, stream);
+    return step_entry(kMgrawa, params, grads, GivenScores{}, n, M, pull, layer_offsets, n_layers, center_out, options, stream);
 }
 
 grawa_status grawa_grawa_step(float* const* params, const float* const* grads, int64_t n, int M, float pull,
                               const int64_t* layer_offsets, int n_layers, float* center_out,
                               const grawa_options* options, grawa_stream_t stream)
 {
-    return step_entry(kGrawa, params, grads, nullptr, n, M, pull, layer_offsets, n_layers, center_out, options, stream);
+    return step_entry(kGrawa, params, grads, GivenScores{}, n, M, pull, layer_offsets, n_layers, center_out, options, stream);
 }
 
 grawa_status grawa_lgrawa_step(float* const* params, const float* const* grads, int64_t n, int M, float pull,
                                const int64_t* layer_offsets, int n_layers, float* center_out,
                                const grawa_options* options, grawa_stream_t stream)
 {
-    return step_entry(kLgrawa, params, grads, nullptr, n, M, pull, layer_offsets, n_layers, center_out, options, stream);
+    return step_entry(kLgrawa, params, grads, GivenScores{}, n, M, pull, layer_offsets, n_layers, center_out, options, stream);
 }
 
 grawa_status grawa_step_from_layer_norms(grawa_variant variant, float* const* params, const double* layer_norms, int64_t n,
@@ -654,8 +662,48 @@ grawa_status grawa_step_from_layer_norms(grawa_variant variant, float* const* pa
 {
     if (variant != GRAWA_VARIANT_GRAWA && variant != GRAWA_VARIANT_MGRAWA && variant != GRAWA_VARIANT_LGRAWA)
         return GRAWA_ERR_INVALID_ARG;
-    return step_entry(static_cast<int>(variant), params, nullptr, layer_norms, n, M, pull, layer_offsets, n_layers, center_out,
+    GivenScores given;
+    given.data = layer_norms;
+    return step_entry(static_cast<int>(variant), params, nullptr, given, n, M, pull, layer_offsets, n_layers, center_out,
                       options, stream);
+}
+
+grawa_status grawa_step_from_layer_sums(grawa_variant variant, float* const* params, const double* layer_sums, int parts,
+                                        int64_t n, int M, float pull, const int64_t* layer_offsets, int n_layers,
+                                        float* center_out, const grawa_options* options, grawa_stream_t stream)
+{
+    if (variant != GRAWA_VARIANT_GRAWA && variant != GRAWA_VARIANT_MGRAWA && variant != GRAWA_VARIANT_LGRAWA)
+        return GRAWA_ERR_INVALID_ARG;
+    GivenScores given;
+    given.data = layer_sums; given.parts = parts; given.sums = 1;
+    return step_entry(static_cast<int>(variant), params, nullptr, given, n, M, pull, layer_offsets, n_layers, center_out,
+                      options, stream);
+}
+
+grawa_status grawa_layer_sumsq(const float* const* grads, int64_t n, int M, const int64_t* layer_offsets, int n_layers,
+                               double* sumsq_out, grawa_stream_t stream)
+{
+    if (grads == nullptr || sumsq_out == nullptr || M < 1 || M > GRAWA_MAX_WORKERS) return GRAWA_ERR_INVALID_ARG;
+    // validate() wants parameter vectors; the gradients stand in (nothing is written through them)
+    std::vector<float*> fake(M);
+    for (int m = 0; m < M; ++m) fake[m] = const_cast<float*>(grads[m]);
+    std::vector<int64_t> off;
+    grawa_status st = validate(fake.data(), nullptr, n, M, 0.0f, layer_offsets, n_layers, nullptr, &off);
+    if (st != GRAWA_OK) return st;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    if (n == 0) {                                    // nothing to add up: every sum is zero
+        GRAWA_CUDA_TRY(cudaMemsetAsync(sumsq_out, 0, sizeof(double) * (off.size() - 1) * M, stream));
+        return GRAWA_OK;
+    }
+    Plan* plan = nullptr;
+    st = get_plan(n, M, off, stream, &plan);
+    if (st != GRAWA_OK) return st;
+    grawa_options opt{};
+    opt.sumsq_out = sumsq_out;
+    StepContext c;
+    st = make_context(kLgrawa, fake.data(), grads, n, M, 0.0f, nullptr, &opt, stream, plan, &c);
+    if (st != GRAWA_OK) return st;
+    return enqueue_weights(c);
 }
 
 grawa_status grawa_layer_norms(const float* grad, int64_t n, const int64_t* layer_offsets, int n_layers, double* norms_out,

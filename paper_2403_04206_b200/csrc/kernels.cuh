@@ -92,7 +92,9 @@ struct StepScratch {
     unsigned global_target;        // arrivals that complete the step's finalisation
     int* status;                   // written (not or-ed) when the finalisation completes
     unsigned* work_counter;        // cleared for the bulk-copy centre+pull kernel
-    const double* layer_norms;     // [K][M] given per-layer norms (steps from scores), else NULL
+    const double* given;           // [given_parts][K][M] given per-layer norms or sums of squares, else NULL
+    int given_parts;               // parts (e.g. ranks) whose sums are added in part order; 1 for norms
+    int given_sums;                // 1: `given` holds sums of squares, 0: norms
     float* weights_out;            // optional copies
     double* scores_out;
     double* sumsq_out;
@@ -143,13 +145,14 @@ struct FinalizeSmem {
 // Steps 1b-3 for one non-empty layer, by a whole CTA of kThreads threads.  Warp w adds the partials
 // of workers w, w+8, ... of layer k in a fixed order into S[k][m]; the layer's terms sqrt(S) (S
 // itself for the flat norm) go to row k of A; LGRAWA turns them into the layer's weights (Eq. 7).
-// With layer_norms set the sums are not needed: the given norm of (layer, worker) takes the place
-// of sqrt(S) (the running estimates of the Local variants).
+// With `given` set no partials are read: either the given norm of (layer, worker) takes the place
+// of sqrt(S) (the running estimates of the Local variants), or S is the sum, in part order, of
+// given partial sums of squares (element-range shards of the vector on several GPUs).
 __device__ __forceinline__ void finalize_layer(const StepScratch& sc, int k, FinalizeSmem& sm)
 {
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int M = sc.M;
-    if (sc.layer_norms == nullptr) {
+    if (sc.given == nullptr) {
         const int s0 = sc.layer_seg_first[k], s1 = sc.layer_seg_first[k + 1];
         for (int m = warp; m < M; m += kThreads / 32) {
             const double* row = sc.partials + static_cast<size_t>(m) * sc.C;
@@ -173,11 +176,15 @@ __device__ __forceinline__ void finalize_layer(const StepScratch& sc, int k, Fin
     const size_t idx = static_cast<size_t>(k) * M + tid;
     if (tid < M) {
         double s;
-        if (sc.layer_norms == nullptr) {
+        if (sc.given == nullptr) {
             s = sm.layer_sum[tid];
             term = (sc.variant == kGrawa) ? s : sqrt(s);
+        } else if (sc.given_sums) {                // sums of squares of the parts, added in part order
+            s = 0.0;
+            for (int r = 0; r < sc.given_parts; ++r) s += sc.given[static_cast<size_t>(r) * sc.K * M + idx];
+            term = (sc.variant == kGrawa) ? s : sqrt(s);
         } else {                                   // the caller's norm estimate stands in for sqrt(S)
-            const double a = sc.layer_norms[idx];
+            const double a = sc.given[idx];
             s = a * a;
             term = (sc.variant == kGrawa) ? s : a;
         }
@@ -216,9 +223,11 @@ __device__ __forceinline__ void finalize_arrive(const StepScratch& sc, FinalizeS
     if (!sm.flag) return;
     __threadfence();
 
-    // empty layers: zero sums and terms, uniform weights (they are never applied)
+    // empty layers: zero sums and terms, uniform weights (they are never applied).  With given
+    // norms or sums every layer has been processed, whether it has local elements or not.
+    const bool all_layers = sc.given != nullptr;
     for (int k = tid; k < K; k += kThreads) {
-        if (sc.layer_seg_first[k] != sc.layer_seg_first[k + 1]) continue;
+        if (all_layers || sc.layer_seg_first[k] != sc.layer_seg_first[k + 1]) continue;
         for (int m = 0; m < M; ++m) {
             const size_t idx = static_cast<size_t>(k) * M + m;
             sc.S[idx] = 0.0;
@@ -236,7 +245,7 @@ __device__ __forceinline__ void finalize_arrive(const StepScratch& sc, FinalizeS
     if (sc.variant == kLgrawa) {
         int f = 0;
         for (int k = tid; k < K; k += kThreads)
-            if (sc.layer_seg_first[k] != sc.layer_seg_first[k + 1]) f |= __ldcg(sc.layer_flag + k);
+            if (all_layers || sc.layer_seg_first[k] != sc.layer_seg_first[k + 1]) f |= __ldcg(sc.layer_flag + k);
         flagged = __syncthreads_or(f);
     } else {
         // Rows of A are staged through shared memory in blocks (parallel loads); thread m then adds
@@ -247,7 +256,7 @@ __device__ __forceinline__ void finalize_arrive(const StepScratch& sc, FinalizeS
             const int rows = min(rows_per_block, K - k0);
             for (int i = tid; i < rows * M; i += kThreads) {
                 const int k = k0 + i / M;
-                const bool empty = sc.layer_seg_first[k] == sc.layer_seg_first[k + 1];
+                const bool empty = !all_layers && sc.layer_seg_first[k] == sc.layer_seg_first[k + 1];
                 sm.stage[i] = empty ? 0.0 : __ldcg(sc.A + static_cast<size_t>(k0) * M + i);
             }
             __syncthreads();
@@ -353,7 +362,7 @@ finalize_kernel(StepScratch sc)
     grid_dependency_sync();
     __shared__ FinalizeSmem fsm;
     const int k = blockIdx.x;
-    if (sc.layer_seg_first[k] != sc.layer_seg_first[k + 1]) finalize_layer(sc, k, fsm);
+    if (sc.given != nullptr || sc.layer_seg_first[k] != sc.layer_seg_first[k + 1]) finalize_layer(sc, k, fsm);
     finalize_arrive(sc, fsm);
 }
 
