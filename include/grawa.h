@@ -110,6 +110,23 @@ grawa_status grawa_lgrawa_step(float *const *params, const float *const *grads, 
                                float pull, const int64_t *layer_offsets, int n_layers,
                                float *center_out, const grawa_options *options, grawa_stream_t stream);
 
+/* Element type of params / grads / center_out in grawa_step_typed. */
+typedef enum grawa_dtype { GRAWA_F32 = 0, GRAWA_BF16 = 1, GRAWA_F16 = 2 } grawa_dtype;
+
+/* The same step (Eq. 2-7, centre, pull) with parameters, gradients and centre STORED in `dtype`:
+ * fp32, bfloat16 or IEEE half.  16-bit storage halves the bytes the step moves.  The arithmetic is
+ * unchanged: every element is widened exactly to fp32 on load, sums of squares, scores and weights
+ * are computed as for fp32, the centre is the fp32 FMA chain, the pull uses the unrounded fp32
+ * centre, and each result is rounded to nearest-even once, on its store (pull = 1 still makes
+ * every worker bit-equal to center_out, pull = 0 leaves them untouched).
+ * params, grads: HOST arrays of M DEVICE pointers to n elements of `dtype`, aligned to the element
+ * size (16-byte aligned bases take the vector kernels); center_out: DEVICE, n elements, or NULL.
+ * GRAWA_F32 is exactly the three step entry points above. */
+grawa_status grawa_step_typed(grawa_dtype dtype, grawa_variant variant, void *const *params,
+                              const void *const *grads, int64_t n, int M, float pull,
+                              const int64_t *layer_offsets, int n_layers, void *center_out,
+                              const grawa_options *options, grawa_stream_t stream);
+
 /* Same update with HOST buffers: params[m], grads[m] and center_out are HOST pointers (pinned
  * memory gives asynchronous copies; pageable memory works and is slower).  The call uploads the
  * M gradient and parameter vectors to device staging buffers owned by the cached plan, runs the

@@ -25,6 +25,7 @@ from .binding import (  # noqa: F401
     grawa_set_option,
     grawa_status_string,
     grawa_step_host,
+    grawa_step_typed,
     grawa_sumsq_static,
     grawa_version,
     grawa_workspace_bytes,

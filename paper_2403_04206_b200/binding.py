@@ -48,6 +48,8 @@ def library() -> ctypes.CDLL:
     for name in ("grawa_mgrawa_step", "grawa_grawa_step", "grawa_lgrawa_step"):
         getattr(lib, name).argtypes = step_args
         getattr(lib, name).restype = ci
+    lib.grawa_step_typed.argtypes = [ci, ci, vp, vp, i64, ci, cf, vp, ci, vp, vp, vp]
+    lib.grawa_step_typed.restype = ci
     lib.grawa_step_host.argtypes = [ci, vp, vp, i64, ci, cf, vp, ci, vp, vp]
     lib.grawa_step_host.restype = ci
     lib.grawa_prox_step.argtypes = [vp, vp, i64, ci, cf, vp]
@@ -184,6 +186,36 @@ def grawa_lgrawa_step(params, grads, pull, layer_offsets, center_out=None, *, we
     """LGRAWA step (Eq. 5-7: per-layer weights); see grawa_lgrawa_step in grawa.h."""
     _step("grawa_lgrawa_step", params, grads, pull, layer_offsets, center_out, weights_out, scores_out,
           sumsq_out, workspace, stream, n)
+
+
+_DTYPES = {"torch.float32": 0, "torch.bfloat16": 1, "torch.float16": 2}
+
+
+def grawa_step_typed(variant, params, grads, pull, layer_offsets=None, center_out=None, *, weights_out=None,
+                     scores_out=None, sumsq_out=None, workspace=None, stream=None, n=None) -> None:
+    """The step on parameters / gradients / centre stored as float32, bfloat16 or float16 device tensors
+    (all of one dtype, taken from ``params[0]``); arithmetic in fp32/fp64, one rounding per stored value."""
+    lib = library()
+    M = len(params)
+    if len(grads) != M or M == 0:
+        raise ValueError("params and grads must have one entry per worker")
+    key = str(params[0].dtype)
+    if key not in _DTYPES:
+        raise TypeError(f"unsupported storage dtype {key}")
+    for b in list(params) + list(grads) + ([center_out] if center_out is not None else []):
+        if str(b.dtype) != key:
+            raise TypeError(f"all buffers must be {key}, got {b.dtype}")
+    v = _VARIANTS[variant] if isinstance(variant, str) else int(variant)
+    if n is None:
+        n = _numel(params[0])
+    off, K = _offsets(layer_offsets)
+    opt = None
+    if any(b is not None for b in (weights_out, scores_out, sumsq_out, workspace)):
+        ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+        opt = _Options(_addr(weights_out), _addr(scores_out), _addr(sumsq_out), _addr(workspace), ws_bytes)
+    _raise(lib.grawa_step_typed(_DTYPES[key], v, _ptr_array(params), _ptr_array(grads), n, M, float(pull),
+                                off.ctypes.data if off is not None else None, K, _addr(center_out),
+                                ctypes.byref(opt) if opt is not None else None, _stream(stream)), "grawa_step_typed")
 
 
 def grawa_step_host(variant, params, grads, pull, layer_offsets=None, center_out=None, *, stream=None, n=None) -> None:

@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "libgrawa.so")
 SOURCES = [os.path.join(CSRC, "grawa.cu")]
-HEADERS = [os.path.join(CSRC, "kernels.cuh"), os.path.join(CSRC, "center_pull_bulk.cuh"),
+HEADERS = [os.path.join(CSRC, "kernels.cuh"), os.path.join(CSRC, "center_pull_bulk.cuh"), os.path.join(CSRC, "kernels_16bit.cuh"),
            os.path.join(_ROOT, "include", "grawa.h")]
 
 # IEEE arithmetic throughout: no fast-math.

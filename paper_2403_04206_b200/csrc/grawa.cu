@@ -16,6 +16,7 @@
 
 #include "kernels.cuh"
 #include "center_pull_bulk.cuh"
+#include "kernels_16bit.cuh"
 
 namespace grawa {
 
@@ -228,7 +229,7 @@ static bool ranges_overlap(const void* a, const void* b, size_t bytes)
 
 static grawa_status validate(float* const* params, const float* const* grads, int64_t n, int M, float pull,
                              const int64_t* layer_offsets, int n_layers, const float* center_out,
-                             std::vector<int64_t>* off)
+                             std::vector<int64_t>* off, size_t elem_size = sizeof(float))
 {
     if (M < 1 || M > GRAWA_MAX_WORKERS || n < 0 || n_layers < 0) return GRAWA_ERR_INVALID_ARG;
     if (!(pull >= 0.0f && pull <= 1.0f)) return GRAWA_ERR_INVALID_ARG;   // also rejects NaN
@@ -243,13 +244,14 @@ static grawa_status validate(float* const* params, const float* const* grads, in
         off->assign({0, n});
     }
     if (n == 0) return GRAWA_OK;
-    const size_t bytes = static_cast<size_t>(n) * sizeof(float);
+    const size_t bytes = static_cast<size_t>(n) * elem_size;
+    const uintptr_t amask = elem_size - 1;          // buffers must be aligned to their element size
     for (int m = 0; m < M; ++m) {
         if (params[m] == nullptr || (grads && grads[m] == nullptr)) return GRAWA_ERR_INVALID_ARG;
-        if ((reinterpret_cast<uintptr_t>(params[m]) & 3u) || (grads && (reinterpret_cast<uintptr_t>(grads[m]) & 3u)))
+        if ((reinterpret_cast<uintptr_t>(params[m]) & amask) || (grads && (reinterpret_cast<uintptr_t>(grads[m]) & amask)))
             return GRAWA_ERR_INVALID_ARG;
     }
-    if (reinterpret_cast<uintptr_t>(center_out) & 3u) return GRAWA_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(center_out) & amask) return GRAWA_ERR_INVALID_ARG;
     for (int a = 0; a < M; ++a) {
         for (int b = a + 1; b < M; ++b)
             if (ranges_overlap(params[a], params[b], bytes)) return GRAWA_ERR_INVALID_ARG;
@@ -354,6 +356,37 @@ struct CenterPullDispatch<1> {
     }
 };
 
+// 16-bit storage: register kernel for 2..16 aligned workers.
+template <typename T, int M>
+static cudaError_t launch_center_pull16(bool per_layer, int grid, int item_begin, int item_end, cudaStream_t stream, bool pdl,
+                                        const MutPtrs& x, T* center, const float* beta, const Segment* segs, long long n,
+                                        int tile, float pull)
+{
+    if (per_layer)
+        return launch_kernel(center_pull16_kernel<T, M, true>, grid, kThreads, stream, pdl, x, center, beta, segs, item_begin,
+                             item_end, n, tile, pull, 1);
+    return launch_kernel(center_pull16_kernel<T, M, false>, grid, kThreads, stream, pdl, x, center, beta, segs, item_begin, item_end,
+                         n, tile, pull, 1);
+}
+
+template <typename T, int M>
+struct CenterPull16Dispatch {
+    template <typename... A>
+    static cudaError_t run(int m, A&&... a)
+    {
+        if (m == M) return launch_center_pull16<T, M>(static_cast<A&&>(a)...);
+        return CenterPull16Dispatch<T, M - 1>::run(m, static_cast<A&&>(a)...);
+    }
+};
+template <typename T>
+struct CenterPull16Dispatch<T, 1> {
+    template <typename... A>
+    static cudaError_t run(int, A&&...)
+    {
+        return cudaErrorInvalidValue;
+    }
+};
+
 // Device pointers and launch facts of one step, resolved once from the plan and the options.
 struct StepContext {
     Plan* plan = nullptr;
@@ -370,6 +403,7 @@ struct StepContext {
     unsigned* counter = nullptr;
     TimedStep* ts = nullptr;
     int pull_items = 0;            // centre+pull work items of the whole vector
+    int dtype = 0;                 // storage of params / grads / centre: 0 fp32, 1 bfloat16, 2 half
 };
 
 static grawa_status make_context(int variant, float* const* params, const float* const* grads, int64_t n, int M, float pull,
@@ -432,11 +466,43 @@ static grawa_status enqueue_weights(StepContext& c)
     const int items1 = plan->C1 * c.M;
     const int grid1 = g_sumsq_ctas_per_sm > 0
                           ? static_cast<int>(std::min<int64_t>(items1, g_sumsq_ctas_per_sm * plan->sm_count)) : items1;
-    GRAWA_CUDA_TRY(launch_kernel(sumsq_kernel<8>, grid1, kThreads, c.stream, c.pdl, c.gp, c.sc, items1, c.vec_g ? 1 : 0));
+    const int vg = c.vec_g ? 1 : 0;
+    if (c.dtype == 1)
+        GRAWA_CUDA_TRY(launch_kernel(sumsq16_kernel<__nv_bfloat16, 4>, grid1, kThreads, c.stream, c.pdl, c.gp, c.sc, items1, vg));
+    else if (c.dtype == 2)
+        GRAWA_CUDA_TRY(launch_kernel(sumsq16_kernel<__half, 4>, grid1, kThreads, c.stream, c.pdl, c.gp, c.sc, items1, vg));
+    else
+        GRAWA_CUDA_TRY(launch_kernel(sumsq_kernel<8>, grid1, kThreads, c.stream, c.pdl, c.gp, c.sc, items1, vg));
     if (c.ts) GRAWA_CUDA_TRY(cudaEventRecord(c.ts->e[1], c.stream));
     GRAWA_CUDA_TRY(launch_kernel(finalize_kernel, plan->K, kThreads, c.stream, c.pdl, c.sc));
     if (c.ts) GRAWA_CUDA_TRY(cudaEventRecord(c.ts->e[2], c.stream));
     return GRAWA_OK;
+}
+
+// Steps 4-5 on 16-bit storage: register kernel for 2..16 aligned workers, scalar kernel otherwise.
+template <typename T>
+static grawa_status enqueue_center_pull16_t(StepContext& c, int item_begin, int item_end)
+{
+    Plan* plan = c.plan;
+    const int M = c.M;
+    const bool per_layer = c.variant == kLgrawa;
+    const int grid = item_end - item_begin;
+    const int tile = static_cast<int>(plan->tile2);
+    T* center = reinterpret_cast<T*>(c.center);
+    if (c.vec_x && M <= kMaxRegWorkers) {
+        GRAWA_CUDA_TRY((CenterPull16Dispatch<T, kMaxRegWorkers>::run(M, per_layer, grid, item_begin, item_end, c.stream, c.pdl, c.xp,
+                                                                     center, c.sc.beta, plan->d_segs2, c.n, tile, c.pull)));
+    } else {
+        GRAWA_CUDA_TRY(launch_kernel(center_pull16_generic_kernel<T>, grid, kThreads, c.stream, c.pdl, c.xp, center, c.sc.beta,
+                                     plan->d_segs2, per_layer ? 1 : 0, item_begin, c.n, tile, c.pull, M));
+    }
+    return GRAWA_OK;
+}
+
+static grawa_status enqueue_center_pull16(StepContext& c, int item_begin, int item_end)
+{
+    if (c.dtype == 1) return enqueue_center_pull16_t<__nv_bfloat16>(c, item_begin, item_end);
+    return enqueue_center_pull16_t<__half>(c, item_begin, item_end);
 }
 
 // Steps 4-5 on the work items [item_begin, item_end) (one launch).  M >= 2.
@@ -449,6 +515,7 @@ static grawa_status enqueue_center_pull(StepContext& c, int item_begin, int item
     if (grid <= 0) return GRAWA_OK;
     const int tile = static_cast<int>(plan->tile2);
     const float* beta = c.sc.beta;
+    if (c.dtype != 0) return enqueue_center_pull16(c, item_begin, item_end);
     // bulk-copy variant: asked for explicitly, or the only vector path for M > 16
     const size_t stage_bytes = sizeof(float) * static_cast<size_t>(plan->tile2) * (M + 1);
     const int stages = static_cast<int>(std::min<size_t>(kBulkMaxStages, kBulkSmemBudget / stage_bytes));
@@ -478,11 +545,12 @@ struct GivenScores {
 
 static grawa_status enqueue_step(int variant, float* const* params, const float* const* grads, const GivenScores& given,
                                  int64_t n, int M, float pull, float* center_out, const grawa_options* opt,
-                                 cudaStream_t stream, Plan* plan)
+                                 cudaStream_t stream, Plan* plan, int dtype = 0)
 {
     StepContext c;
     grawa_status st = make_context(variant, params, grads, n, M, pull, center_out, opt, stream, plan, &c);
     if (st != GRAWA_OK) return st;
+    c.dtype = dtype;
     c.sc.given = given.data; c.sc.given_parts = given.parts; c.sc.given_sums = given.sums;
     if (g_kernel_timing) {
         if (g_timed_used == g_timed_pool.size()) {
@@ -500,7 +568,15 @@ static grawa_status enqueue_step(int variant, float* const* params, const float*
         if (center_out) {
             const bool v = aligned16(center_out) && aligned16(params[0]);
             const int grid = static_cast<int>(std::min<int64_t>((n + kThreads * 4 - 1) / (kThreads * 4), 148 * 16));
-            GRAWA_CUDA_TRY(launch_kernel(copy_kernel, grid, kThreads, stream, c.pdl, params[0], center_out, n, v ? 1 : 0));
+            if (dtype == 1)
+                GRAWA_CUDA_TRY(launch_kernel(copy16_kernel<__nv_bfloat16>, grid, kThreads, stream, c.pdl,
+                                             reinterpret_cast<const __nv_bfloat16*>(params[0]),
+                                             reinterpret_cast<__nv_bfloat16*>(center_out), n));
+            else if (dtype == 2)
+                GRAWA_CUDA_TRY(launch_kernel(copy16_kernel<__half>, grid, kThreads, stream, c.pdl,
+                                             reinterpret_cast<const __half*>(params[0]), reinterpret_cast<__half*>(center_out), n));
+            else
+                GRAWA_CUDA_TRY(launch_kernel(copy_kernel, grid, kThreads, stream, c.pdl, params[0], center_out, n, v ? 1 : 0));
         }
     } else {
         st = enqueue_center_pull(c, 0, c.pull_items);
@@ -512,18 +588,19 @@ static grawa_status enqueue_step(int variant, float* const* params, const float*
 
 static grawa_status step_entry(int variant, float* const* params, const float* const* grads, const GivenScores& given,
                                int64_t n, int M, float pull, const int64_t* layer_offsets, int n_layers, float* center_out,
-                               const grawa_options* opt, cudaStream_t stream)
+                               const grawa_options* opt, cudaStream_t stream, int dtype = 0)
 {
     if ((grads == nullptr) == (given.data == nullptr)) return GRAWA_ERR_INVALID_ARG;   // exactly one source of scores
     if (given.parts < 1) return GRAWA_ERR_INVALID_ARG;
     std::vector<int64_t> off;
-    grawa_status st = validate(params, grads, n, M, pull, layer_offsets, n_layers, center_out, &off);
+    grawa_status st = validate(params, grads, n, M, pull, layer_offsets, n_layers, center_out, &off,
+                               dtype == 0 ? sizeof(float) : size_t{2});
     if (st != GRAWA_OK || n == 0) return st;
     std::lock_guard<std::mutex> lock(g_mutex);
     Plan* plan = nullptr;
     st = get_plan(n, M, off, stream, &plan);
     if (st != GRAWA_OK) return st;
-    return enqueue_step(variant, params, grads, given, n, M, pull, center_out, opt, stream, plan);
+    return enqueue_step(variant, params, grads, given, n, M, pull, center_out, opt, stream, plan, dtype);
 }
 
 // ------------------------------------------------------------------ allocation-free sum of squares
@@ -654,6 +731,19 @@ grawa_status grawa_lgrawa_step(float* const* params, const float* const* grads, 
                                const grawa_options* options, grawa_stream_t stream)
 {
     return step_entry(kLgrawa, params, grads, GivenScores{}, n, M, pull, layer_offsets, n_layers, center_out, options, stream);
+}
+
+grawa_status grawa_step_typed(grawa_dtype dtype, grawa_variant variant, void* const* params, const void* const* grads, int64_t n,
+                              int M, float pull, const int64_t* layer_offsets, int n_layers, void* center_out,
+                              const grawa_options* options, grawa_stream_t stream)
+{
+    if (variant != GRAWA_VARIANT_GRAWA && variant != GRAWA_VARIANT_MGRAWA && variant != GRAWA_VARIANT_LGRAWA)
+        return GRAWA_ERR_INVALID_ARG;
+    if (dtype != GRAWA_F32 && dtype != GRAWA_BF16 && dtype != GRAWA_F16) return GRAWA_ERR_INVALID_ARG;
+    // the pointer tables carry untyped addresses; the kernels of `dtype` give them their element type
+    return step_entry(static_cast<int>(variant), reinterpret_cast<float* const*>(params),
+                      reinterpret_cast<const float* const*>(grads), GivenScores{}, n, M, pull, layer_offsets, n_layers,
+                      static_cast<float*>(center_out), options, stream, static_cast<int>(dtype));
 }
 
 grawa_status grawa_step_from_layer_norms(grawa_variant variant, float* const* params, const double* layer_norms, int64_t n,

@@ -1,0 +1,295 @@
+// 16-bit storage (bfloat16 / half) variants of the two streaming kernels: parameters, gradients
+// and centre are stored in T, all arithmetic is the fp32 / fp64 arithmetic of the fp32 kernels, and
+// results are rounded to nearest-even once, on the store.  Half the bytes per element.
+#pragma once
+#include <cuda_bf16.h>
+#include <cuda_fp16.h>
+
+#include "kernels.cuh"
+
+namespace grawa {
+
+// Conversions between a 32-bit word holding two T and two floats.
+template <typename T> struct Pair16;
+template <> struct Pair16<__nv_bfloat16> {
+    static __device__ __forceinline__ void unpack(unsigned w, float& lo, float& hi)
+    {
+        lo = __uint_as_float(w << 16);              // a bfloat16 is the upper half of a float
+        hi = __uint_as_float(w & 0xffff0000u);
+    }
+    static __device__ __forceinline__ unsigned pack(float lo, float hi)
+    {
+        const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+        return *reinterpret_cast<const unsigned*>(&v);
+    }
+    static __device__ __forceinline__ float load1(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+    static __device__ __forceinline__ void store1(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+};
+template <> struct Pair16<__half> {
+    static __device__ __forceinline__ void unpack(unsigned w, float& lo, float& hi)
+    {
+        const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&w));
+        lo = f.x;
+        hi = f.y;
+    }
+    static __device__ __forceinline__ unsigned pack(float lo, float hi)
+    {
+        const __half2 v = __floats2half2_rn(lo, hi);
+        return *reinterpret_cast<const unsigned*>(&v);
+    }
+    static __device__ __forceinline__ float load1(const __half* p) { return __half2float(*p); }
+    static __device__ __forceinline__ void store1(__half* p, float v) { *p = __float2half_rn(v); }
+};
+
+// VEC consecutive elements (16 bytes for VEC = 8, 8 bytes for VEC = 4), aligned, streaming.
+template <typename T, int VEC> struct Vec16IO;
+template <typename T> struct Vec16IO<T, 8> {
+    static __device__ __forceinline__ void ld(const T* p, float (&o)[8])
+    {
+        const uint4 r = __ldcs(reinterpret_cast<const uint4*>(p));
+        Pair16<T>::unpack(r.x, o[0], o[1]); Pair16<T>::unpack(r.y, o[2], o[3]);
+        Pair16<T>::unpack(r.z, o[4], o[5]); Pair16<T>::unpack(r.w, o[6], o[7]);
+    }
+    static __device__ __forceinline__ void st(T* p, const float (&o)[8])
+    {
+        uint4 r;
+        r.x = Pair16<T>::pack(o[0], o[1]); r.y = Pair16<T>::pack(o[2], o[3]);
+        r.z = Pair16<T>::pack(o[4], o[5]); r.w = Pair16<T>::pack(o[6], o[7]);
+        __stcs(reinterpret_cast<uint4*>(p), r);
+    }
+};
+template <typename T> struct Vec16IO<T, 4> {
+    static __device__ __forceinline__ void ld(const T* p, float (&o)[4])
+    {
+        const uint2 r = __ldcs(reinterpret_cast<const uint2*>(p));
+        Pair16<T>::unpack(r.x, o[0], o[1]); Pair16<T>::unpack(r.y, o[2], o[3]);
+    }
+    static __device__ __forceinline__ void st(T* p, const float (&o)[4])
+    {
+        uint2 r;
+        r.x = Pair16<T>::pack(o[0], o[1]); r.y = Pair16<T>::pack(o[2], o[3]);
+        __stcs(reinterpret_cast<uint2*>(p), r);
+    }
+};
+
+// [b, e) -> scalar head, body aligned to 8 elements (16 bytes), scalar tail.
+__device__ __forceinline__ void split_range16(long long b, long long e, int vec_ok, long long& hb, long long& te)
+{
+    if (vec_ok) {
+        hb = min((b + 7) & ~7LL, e);
+        te = max(e & ~7LL, hb);
+    } else {
+        hb = e;
+        te = e;
+    }
+}
+
+// Step 1 on 16-bit gradients: same work list, same fp32-run / fp64-combine scheme as sumsq_kernel;
+// a thread's 16-byte load carries 8 elements, each with its own fp32 accumulator.
+template <typename T, int UNROLL>
+__global__ void __launch_bounds__(kThreads, 5)
+sumsq16_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
+{
+    grid_dependency_sync();
+    __shared__ double warp_part[2][kThreads / 32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int C = sc.C;
+
+    int parity = 0;
+    for (int item = blockIdx.x; item < items; item += gridDim.x, parity ^= 1) {
+        const int m = item / C;
+        const int s = item - m * C;
+        const Segment sg = sc.segs[s];
+        const T* __restrict__ g = reinterpret_cast<const T*>(grads.p[m]);
+        const long long b = sg.begin, e = b + sg.len;
+        long long hb, te;
+        split_range16(b, e, vec_ok, hb, te);
+        double dacc = 0.0;
+
+        const int ncol = static_cast<int>((te - hb) >> 3);
+        for (int c0 = 0; c0 < ncol; c0 += kThreads * UNROLL) {
+            float v[UNROLL][8];
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+                const int c = c0 + u * kThreads + tid;
+                if (c < ncol) {
+                    Vec16IO<T, 8>::ld(g + hb + static_cast<long long>(c) * 8, v[u]);
+                } else {
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) v[u][t] = 0.f;
+                }
+            }
+            float a[8];
+#pragma unroll
+            for (int t = 0; t < 8; ++t) a[t] = 0.f;
+#pragma unroll
+            for (int u = 0; u < UNROLL; ++u) {
+#pragma unroll
+                for (int t = 0; t < 8; ++t) a[t] = fmaf(v[u][t], v[u][t], a[t]);
+            }
+            dacc += ((static_cast<double>(a[0]) + static_cast<double>(a[1])) + (static_cast<double>(a[2]) + static_cast<double>(a[3]))) +
+                    ((static_cast<double>(a[4]) + static_cast<double>(a[5])) + (static_cast<double>(a[6]) + static_cast<double>(a[7])));
+        }
+        for (long long i = b + tid; i < hb; i += kThreads) {
+            const double v = static_cast<double>(Pair16<T>::load1(g + i));
+            dacc += v * v;
+        }
+        for (long long i = te + tid; i < e; i += kThreads) {
+            const double v = static_cast<double>(Pair16<T>::load1(g + i));
+            dacc += v * v;
+        }
+#pragma unroll
+        for (int d = 16; d > 0; d >>= 1) dacc += __shfl_down_sync(0xffffffffu, dacc, d);
+        if (lane == 0) warp_part[parity][warp] = dacc;
+        __syncthreads();
+        if (tid == 0) {
+            double total = 0.0;
+#pragma unroll
+            for (int w = 0; w < kThreads / 32; ++w) total += warp_part[parity][w];
+            sc.partials[static_cast<size_t>(m) * C + s] = total;
+        }
+    }
+}
+
+// Shape of the 16-bit centre+pull kernel: 16-byte columns (8 elements) up to 8 workers, 8-byte
+// columns (4 elements) above, so that a thread never holds more than 64 values; the elements one
+// CTA covers per pass come out the same as for fp32 (pull_pass_elems).
+__host__ __device__ constexpr int pull16_vec(int M) { return (M <= 8) ? 8 : 4; }
+__host__ __device__ constexpr int pull16_cols(int M) { return (M <= 2) ? 4 : (M <= 4) ? 2 : 1; }
+static_assert(kThreads * pull16_cols(2) * pull16_vec(2) == pull_pass_elems(2), "pass size differs from fp32");
+static_assert(kThreads * pull16_cols(4) * pull16_vec(4) == pull_pass_elems(4), "pass size differs from fp32");
+static_assert(kThreads * pull16_cols(8) * pull16_vec(8) == pull_pass_elems(8), "pass size differs from fp32");
+static_assert(kThreads * pull16_cols(16) * pull16_vec(16) == pull_pass_elems(16), "pass size differs from fp32");
+
+template <typename T, int M>
+__device__ __forceinline__ void pull16_scalar(const MutPtrs& x, T* center, const float (&w)[M], float lambda, float oml,
+                                              long long i)
+{
+    float v[M];
+#pragma unroll
+    for (int m = 0; m < M; ++m) v[m] = Pair16<T>::load1(reinterpret_cast<const T*>(x.p[m]) + i);
+    float c = w[0] * v[0];
+#pragma unroll
+    for (int m = 1; m < M; ++m) c = fmaf(w[m], v[m], c);
+    if (center) Pair16<T>::store1(center + i, c);
+#pragma unroll
+    for (int m = 0; m < M; ++m) Pair16<T>::store1(reinterpret_cast<T*>(x.p[m]) + i, fmaf(lambda, c, oml * v[m]));
+}
+
+// Steps 4-5 on 16-bit parameters: same arithmetic as center_pull_kernel (fp32 FMA chain over
+// m = 0..M-1, pull from the unrounded fp32 centre), one rounding on each store.
+template <typename T, int M, bool PER_LAYER>
+__global__ void __launch_bounds__(kThreads, 2)
+center_pull16_kernel(MutPtrs x, T* __restrict__ center, const float* __restrict__ beta, const Segment* __restrict__ segs,
+                     int item_begin, int item_end, long long n, int tile, float lambda, int vec_ok)
+{
+    grid_dependency_sync();
+    constexpr int COLS = pull16_cols(M);
+    constexpr int VEC = pull16_vec(M);
+    const float oml = 1.0f - lambda;
+    const int tid = threadIdx.x;
+    float w[M];
+    if (!PER_LAYER) {
+#pragma unroll
+        for (int m = 0; m < M; ++m) w[m] = beta[m];
+    }
+    for (int item = item_begin + blockIdx.x; item < item_end; item += gridDim.x) {
+        long long b, e;
+        if (PER_LAYER) {
+            const Segment sg = segs[item];
+            b = sg.begin;
+            e = b + sg.len;
+            const float* __restrict__ bt = beta + static_cast<size_t>(sg.layer) * M;
+#pragma unroll
+            for (int m = 0; m < M; ++m) w[m] = bt[m];
+        } else {
+            b = static_cast<long long>(item) * tile;
+            e = min(n, b + tile);
+        }
+        long long hb, te;
+        split_range16(b, e, vec_ok, hb, te);
+        const int ncol = static_cast<int>((te - hb) / VEC);      // te - hb is a multiple of 8
+        for (int c0 = 0; c0 < ncol; c0 += kThreads * COLS) {
+            float v[COLS][M][VEC];
+#pragma unroll
+            for (int q = 0; q < COLS; ++q) {
+                const int c = c0 + q * kThreads + tid;
+                if (c < ncol) {
+#pragma unroll
+                    for (int m = 0; m < M; ++m)
+                        Vec16IO<T, VEC>::ld(reinterpret_cast<const T*>(x.p[m]) + hb + static_cast<long long>(c) * VEC, v[q][m]);
+                }
+            }
+#pragma unroll
+            for (int q = 0; q < COLS; ++q) {
+                const int c = c0 + q * kThreads + tid;
+                if (c < ncol) {
+                    float cc[VEC];
+#pragma unroll
+                    for (int t = 0; t < VEC; ++t) cc[t] = w[0] * v[q][0][t];
+#pragma unroll
+                    for (int m = 1; m < M; ++m) {
+#pragma unroll
+                        for (int t = 0; t < VEC; ++t) cc[t] = fmaf(w[m], v[q][m][t], cc[t]);
+                    }
+                    if (center) Vec16IO<T, VEC>::st(center + hb + static_cast<long long>(c) * VEC, cc);
+#pragma unroll
+                    for (int m = 0; m < M; ++m) {
+                        float o[VEC];
+#pragma unroll
+                        for (int t = 0; t < VEC; ++t) o[t] = fmaf(lambda, cc[t], oml * v[q][m][t]);
+                        Vec16IO<T, VEC>::st(reinterpret_cast<T*>(x.p[m]) + hb + static_cast<long long>(c) * VEC, o);
+                    }
+                }
+            }
+        }
+        for (long long i = b + tid; i < hb; i += kThreads) pull16_scalar<T, M>(x, center, w, lambda, oml, i);
+        for (long long i = te + tid; i < e; i += kThreads) pull16_scalar<T, M>(x, center, w, lambda, oml, i);
+    }
+}
+
+// Steps 4-5 on 16-bit parameters for any M and any alignment (scalar).
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+center_pull16_generic_kernel(MutPtrs x, T* __restrict__ center, const float* __restrict__ beta,
+                             const Segment* __restrict__ segs, int per_layer, int item_begin, long long n, int tile,
+                             float lambda, int M)
+{
+    grid_dependency_sync();
+    long long b, e;
+    const float* __restrict__ bt = beta;
+    if (per_layer) {
+        const Segment sg = segs[item_begin + blockIdx.x];
+        b = sg.begin;
+        e = b + sg.len;
+        bt = beta + static_cast<size_t>(sg.layer) * M;
+    } else {
+        b = static_cast<long long>(item_begin + blockIdx.x) * tile;
+        e = min(n, b + tile);
+    }
+    __shared__ float w[kMaxWorkers];
+    if (threadIdx.x < M) w[threadIdx.x] = bt[threadIdx.x];
+    __syncthreads();
+    const float oml = 1.0f - lambda;
+    for (long long i = b + threadIdx.x; i < e; i += kThreads) {
+        float c = w[0] * Pair16<T>::load1(reinterpret_cast<const T*>(x.p[0]) + i);
+        for (int m = 1; m < M; ++m) c = fmaf(w[m], Pair16<T>::load1(reinterpret_cast<const T*>(x.p[m]) + i), c);
+        if (center) Pair16<T>::store1(center + i, c);
+        for (int m = 0; m < M; ++m) {
+            T* p = reinterpret_cast<T*>(x.p[m]) + i;
+            Pair16<T>::store1(p, fmaf(lambda, c, oml * Pair16<T>::load1(p)));
+        }
+    }
+}
+
+// M = 1 on 16-bit parameters: the centre is a copy of the single worker.
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+copy16_kernel(const T* __restrict__ src, T* __restrict__ dst, long long n)
+{
+    grid_dependency_sync();
+    const long long stride = static_cast<long long>(gridDim.x) * kThreads;
+    for (long long i = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x; i < n; i += stride) dst[i] = src[i];
+}
+
+}  // namespace grawa

@@ -1,0 +1,140 @@
+"""GPU parity of the step on 16-bit storage (bfloat16 / float16 parameters, gradients, centre).
+
+The inputs are exactly representable in fp32, so the oracle runs on their fp32 images.  The GPU
+rounds each result to the storage type once, so the bound is the fp32 bound of the parity contract
+plus half a unit in the last place of the storage type at the oracle's value."""
+import numpy as np
+import pytest
+
+import gen
+import oracle
+from gpu_util import TOL_BETA_REL, TOL_S_REL, TOL_X_ABS_FACTOR
+
+pytestmark = pytest.mark.gpu
+
+HALF_ULP = {"bfloat16": 2.0 ** -8, "float16": 2.0 ** -11}      # relative, normal range
+TINY = {"bfloat16": 0.0, "float16": 2.0 ** -25}                # half the smallest fp16 subnormal step
+
+
+@pytest.fixture(scope="module")
+def grawa():
+    import paper_2403_04206_b200 as g
+    g.library()
+    return g
+
+
+def run_typed(grawa, dtype_name, variant, p32, g32, pull, off, want_center=True, offset_elems=0):
+    """p32/g32: fp32 numpy inputs; they are rounded to the storage type first (that is the problem
+    both sides then solve).  Returns GPU results as fp32 numpy plus the fp32 images of the inputs."""
+    import torch
+    dt = getattr(torch, dtype_name)
+
+    def dev(a):
+        t = torch.zeros(a.size + offset_elems, dtype=dt, device="cuda")
+        t[offset_elems:] = torch.from_numpy(a).cuda().to(dt)
+        return t[offset_elems:]
+    x = [dev(a) for a in p32]
+    g = [dev(a) for a in g32]
+    p_img = [t.float().cpu().numpy() for t in x]
+    g_img = [t.float().cpu().numpy() for t in g]
+    M, n = len(x), p32[0].size
+    K = len(off) - 1
+    G = K if variant == "lgrawa" else 1
+    beta = torch.empty(G * M, device="cuda")
+    sumsq = torch.empty(K * M, dtype=torch.float64, device="cuda")
+    center = torch.zeros(n, dtype=dt, device="cuda") if want_center else None
+    grawa.grawa_step_typed(variant, x, g, pull, off, center, weights_out=beta, sumsq_out=sumsq)
+    assert grawa.grawa_last_step_status() == 0
+    return {"workers": [t.float().cpu().numpy() for t in x], "center": center.float().cpu().numpy() if want_center else None,
+            "beta": beta.cpu().numpy(), "S": sumsq.cpu().numpy().reshape(K, M), "p_img": p_img, "g_img": g_img}
+
+
+def check(res, dtype_name, variant, pull, off, check_workers=True):
+    p, g = res["p_img"], res["g_img"]
+    ref = oracle.step(p, g, pull, variant, off)
+    assert np.allclose(res["S"], ref["S"], rtol=TOL_S_REL, atol=0)
+    rb = ref["beta"].ravel()
+    nz = rb != 0
+    assert np.abs(res["beta"][nz] / rb[nz] - 1).max() <= TOL_BETA_REL
+    base = TOL_X_ABS_FACTOR * max(float(np.abs(a).max()) for a in p)
+    hu, tiny = HALF_ULP[dtype_name], TINY[dtype_name]
+    if res["center"] is not None:
+        assert np.all(np.abs(res["center"] - ref["center"]) <= base + hu * np.abs(ref["center"]) + tiny)
+    if check_workers:
+        for m in range(len(p)):
+            assert np.all(np.abs(res["workers"][m] - ref["workers"][m]) <= base + hu * np.abs(ref["workers"][m]) + tiny)
+
+
+@pytest.mark.parametrize("dtype_name", ["bfloat16", "float16"])
+@pytest.mark.parametrize("variant", ["mgrawa", "lgrawa", "grawa"])
+@pytest.mark.parametrize("name", ["toy10", "resnet20_cifar", "resnet18_imagenet"])
+def test_16bit_parity_on_workloads(grawa, name, variant, dtype_name):
+    cfg = gen.CONFIGS[name]
+    p, g = gen.make_inputs(cfg)
+    res = run_typed(grawa, dtype_name, variant, p, g, cfg.pull, cfg.offsets())
+    check(res, dtype_name, variant, cfg.pull, cfg.offsets())
+
+
+@pytest.mark.parametrize("dtype_name", ["bfloat16", "float16"])
+@pytest.mark.parametrize("M", [1, 2, 3, 4, 5, 8, 9, 16, 17, 33])
+def test_16bit_parity_on_worker_counts_and_ragged_tables(grawa, M, dtype_name):
+    cfg = gen.custom_config([7, 5001, 0, 3, 12001, 777, 8, 9, 8192, 8193], M, seed=200 + M, log10_sigma=(-2.0, 0.0))
+    p, g = gen.make_inputs(cfg)
+    for variant in ("mgrawa", "lgrawa"):
+        res = run_typed(grawa, dtype_name, variant, p, g, 0.3, cfg.offsets())
+        check(res, dtype_name, variant, 0.3, cfg.offsets(), check_workers=(M > 1))
+        if M == 1:
+            assert np.array_equal(res["workers"][0], res["p_img"][0]) and np.array_equal(res["center"], res["p_img"][0])
+
+
+@pytest.mark.parametrize("dtype_name", ["bfloat16", "float16"])
+def test_16bit_unaligned_bases_and_no_centre(grawa, dtype_name):
+    cfg = gen.custom_config([10, 5000, 3, 9000], 4, seed=21)
+    p, g = gen.make_inputs(cfg)
+    res = run_typed(grawa, dtype_name, "lgrawa", p, g, 0.5, cfg.offsets(), offset_elems=1)     # bases 2 bytes off
+    check(res, dtype_name, "lgrawa", 0.5, cfg.offsets())
+    res = run_typed(grawa, dtype_name, "mgrawa", p, g, 0.5, cfg.offsets(), want_center=False)
+    check(res, dtype_name, "mgrawa", 0.5, cfg.offsets())
+
+
+@pytest.mark.parametrize("dtype_name", ["bfloat16", "float16"])
+def test_16bit_pull_extremes_are_bit_exact(grawa, dtype_name):
+    cfg = gen.CONFIGS["toy10"]
+    p, g = gen.make_inputs(cfg)
+    r1 = run_typed(grawa, dtype_name, "lgrawa", p, g, 1.0, cfg.offsets())
+    for w in r1["workers"]:
+        assert np.array_equal(w, r1["center"])                   # full pull: every worker is the stored centre
+    r0 = run_typed(grawa, dtype_name, "lgrawa", p, g, 0.0, cfg.offsets())
+    for w, a in zip(r0["workers"], r0["p_img"]):
+        assert np.array_equal(w, a)                              # no pull: untouched
+    assert np.array_equal(r0["center"], r1["center"])
+
+
+def test_16bit_sumsq_bit_exact_on_integer_gradients(grawa):
+    sizes = [10, 1000, 8192, 3, 20000, 1, 4097, 70000]
+    rng = np.random.default_rng(3)
+    off = np.concatenate([[0], np.cumsum(sizes)])
+    g = [rng.integers(-3, 4, size=off[-1]).astype(np.float32) for _ in range(3)]
+    p = [rng.normal(size=off[-1]).astype(np.float32) for _ in range(3)]
+    for dtype_name in ("bfloat16", "float16"):
+        res = run_typed(grawa, dtype_name, "lgrawa", p, g, 0.5, off)
+        assert np.array_equal(res["S"], oracle.sumsq(g, off))
+
+
+def test_typed_entry_with_float32_equals_the_plain_entry(grawa):
+    import torch
+    cfg = gen.CONFIGS["resnet20_cifar"]
+    p, g = gen.make_inputs(cfg)
+    off = cfg.offsets()
+    xa = [torch.from_numpy(a).cuda() for a in p]
+    xb = [torch.from_numpy(a).cuda() for a in p]
+    gr = [torch.from_numpy(a).cuda() for a in g]
+    ca, cb = torch.empty(cfg.n, device="cuda"), torch.empty(cfg.n, device="cuda")
+    grawa.grawa_lgrawa_step(xa, gr, 0.5, off, ca)
+    grawa.grawa_step_typed("lgrawa", xb, gr, 0.5, off, cb)
+    torch.cuda.synchronize()
+    assert bool((ca == cb).all()) and all(bool((u == v).all()) for u, v in zip(xa, xb))
+    with pytest.raises(TypeError):
+        grawa.grawa_step_typed("lgrawa", [t.double() for t in xa], gr, 0.5, off, ca)
+    with pytest.raises(TypeError):
+        grawa.grawa_step_typed("lgrawa", [t.half() for t in xa], gr, 0.5, off, ca)      # mixed dtypes
