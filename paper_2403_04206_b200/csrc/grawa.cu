@@ -940,7 +940,7 @@ grawa_status grawa_prox_step(float* const* params, const float* center, int64_t 
     int64_t tile;
     {
         std::lock_guard<std::mutex> lock(g_mutex);
-        tile = g_pull_tile > 0 ? g_pull_tile : 4096;
+        tile = g_pull_tile > 0 ? g_pull_tile : 1024;   // one vector column per thread: measured best (6.6-6.9 TB/s)
     }
     const int64_t tiles = (n + tile - 1) / tile;
     if (tiles > 0x7fffffffll) return GRAWA_ERR_INVALID_ARG;
