@@ -162,10 +162,11 @@ struct Plan {
 };
 
 struct PlanKey {
-    int device; cudaStream_t stream; int64_t n; int M; std::vector<int64_t> off;
+    int device; cudaStream_t stream; int64_t n; int M; int elem; std::vector<int64_t> off;
     bool operator<(const PlanKey& o) const
     {
         if (device != o.device) return device < o.device;
+        if (elem != o.elem) return elem < o.elem;
         if (stream != o.stream) return stream < o.stream;
         if (n != o.n) return n < o.n;
         if (M != o.M) return M < o.M;
@@ -182,19 +183,21 @@ static size_t g_timed_used = 0;
 static auto& g_plans = *new std::map<PlanKey, std::unique_ptr<Plan>>;
 static auto& g_last_status = *new std::map<std::pair<int, cudaStream_t>, int*>;   // (device, stream) -> status word
 
-static grawa_status get_plan(int64_t n, int M, const std::vector<int64_t>& off, cudaStream_t stream, Plan** out)
+// `elem`: bytes per stored element (4, or 2 for 16-bit storage, whose kernels cover twice the
+// elements per pass and therefore cut the work lists with twice the tile).
+static grawa_status get_plan(int64_t n, int M, const std::vector<int64_t>& off, cudaStream_t stream, Plan** out, int elem = 4)
 {
     int device = 0;
     GRAWA_CUDA_TRY(cudaGetDevice(&device));
-    PlanKey key{device, stream, n, M, off};
+    PlanKey key{device, stream, n, M, elem, off};
     auto it = g_plans.find(key);
     if (it != g_plans.end()) { *out = it->second.get(); return GRAWA_OK; }
 
     std::unique_ptr<Plan> p(new Plan);
     p->device = device; p->stream = stream; p->n = n; p->M = M; p->off = off;
     p->K = static_cast<int>(off.size()) - 1;
-    p->bulk = wants_bulk(M);
-    p->tile1 = g_sumsq_tile;
+    p->bulk = elem == 4 && wants_bulk(M);
+    p->tile1 = g_sumsq_tile * (4 / elem);
     p->tile2 = p->bulk ? bulk_tile_for(M) : (g_pull_tile > 0 ? g_pull_tile : pull_pass_elems(std::min(M, kMaxRegWorkers)));
     GRAWA_CUDA_TRY(cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, device));
     std::vector<Segment> s1, s2;
@@ -468,9 +471,9 @@ static grawa_status enqueue_weights(StepContext& c)
                           ? static_cast<int>(std::min<int64_t>(items1, g_sumsq_ctas_per_sm * plan->sm_count)) : items1;
     const int vg = c.vec_g ? 1 : 0;
     if (c.dtype == 1)
-        GRAWA_CUDA_TRY(launch_kernel(sumsq16_kernel<__nv_bfloat16, 4>, grid1, kThreads, c.stream, c.pdl, c.gp, c.sc, items1, vg));
+        GRAWA_CUDA_TRY(launch_kernel(sumsq16_kernel<__nv_bfloat16, 8>, grid1, kThreads, c.stream, c.pdl, c.gp, c.sc, items1, vg));
     else if (c.dtype == 2)
-        GRAWA_CUDA_TRY(launch_kernel(sumsq16_kernel<__half, 4>, grid1, kThreads, c.stream, c.pdl, c.gp, c.sc, items1, vg));
+        GRAWA_CUDA_TRY(launch_kernel(sumsq16_kernel<__half, 8>, grid1, kThreads, c.stream, c.pdl, c.gp, c.sc, items1, vg));
     else
         GRAWA_CUDA_TRY(launch_kernel(sumsq_kernel<8>, grid1, kThreads, c.stream, c.pdl, c.gp, c.sc, items1, vg));
     if (c.ts) GRAWA_CUDA_TRY(cudaEventRecord(c.ts->e[1], c.stream));
@@ -598,7 +601,7 @@ static grawa_status step_entry(int variant, float* const* params, const float* c
     if (st != GRAWA_OK || n == 0) return st;
     std::lock_guard<std::mutex> lock(g_mutex);
     Plan* plan = nullptr;
-    st = get_plan(n, M, off, stream, &plan);
+    st = get_plan(n, M, off, stream, &plan, dtype == 0 ? 4 : 2);
     if (st != GRAWA_OK) return st;
     return enqueue_step(variant, params, grads, given, n, M, pull, center_out, opt, stream, plan, dtype);
 }

@@ -41,36 +41,22 @@ template <> struct Pair16<__half> {
     static __device__ __forceinline__ void store1(__half* p, float v) { *p = __float2half_rn(v); }
 };
 
-// VEC consecutive elements (16 bytes for VEC = 8, 8 bytes for VEC = 4), aligned, streaming.
-template <typename T, int VEC> struct Vec16IO;
-template <typename T> struct Vec16IO<T, 8> {
-    static __device__ __forceinline__ void ld(const T* p, float (&o)[8])
-    {
-        const uint4 r = __ldcs(reinterpret_cast<const uint4*>(p));
-        Pair16<T>::unpack(r.x, o[0], o[1]); Pair16<T>::unpack(r.y, o[2], o[3]);
-        Pair16<T>::unpack(r.z, o[4], o[5]); Pair16<T>::unpack(r.w, o[6], o[7]);
-    }
-    static __device__ __forceinline__ void st(T* p, const float (&o)[8])
-    {
-        uint4 r;
-        r.x = Pair16<T>::pack(o[0], o[1]); r.y = Pair16<T>::pack(o[2], o[3]);
-        r.z = Pair16<T>::pack(o[4], o[5]); r.w = Pair16<T>::pack(o[6], o[7]);
-        __stcs(reinterpret_cast<uint4*>(p), r);
-    }
-};
-template <typename T> struct Vec16IO<T, 4> {
-    static __device__ __forceinline__ void ld(const T* p, float (&o)[4])
-    {
-        const uint2 r = __ldcs(reinterpret_cast<const uint2*>(p));
-        Pair16<T>::unpack(r.x, o[0], o[1]); Pair16<T>::unpack(r.y, o[2], o[3]);
-    }
-    static __device__ __forceinline__ void st(T* p, const float (&o)[4])
-    {
-        uint2 r;
-        r.x = Pair16<T>::pack(o[0], o[1]); r.y = Pair16<T>::pack(o[2], o[3]);
-        __stcs(reinterpret_cast<uint2*>(p), r);
-    }
-};
+// Eight consecutive elements travel as one 16-byte word and stay packed in registers (four
+// registers instead of eight) until the arithmetic needs them.
+template <typename T>
+__device__ __forceinline__ void unpack8(const uint4& r, float (&o)[8])
+{
+    Pair16<T>::unpack(r.x, o[0], o[1]); Pair16<T>::unpack(r.y, o[2], o[3]);
+    Pair16<T>::unpack(r.z, o[4], o[5]); Pair16<T>::unpack(r.w, o[6], o[7]);
+}
+template <typename T>
+__device__ __forceinline__ uint4 pack8(const float (&o)[8])
+{
+    uint4 r;
+    r.x = Pair16<T>::pack(o[0], o[1]); r.y = Pair16<T>::pack(o[2], o[3]);
+    r.z = Pair16<T>::pack(o[4], o[5]); r.w = Pair16<T>::pack(o[6], o[7]);
+    return r;
+}
 
 // [b, e) -> scalar head, body aligned to 8 elements (16 bytes), scalar tail.
 __device__ __forceinline__ void split_range16(long long b, long long e, int vec_ok, long long& hb, long long& te)
@@ -107,25 +93,23 @@ sumsq16_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
         double dacc = 0.0;
 
         const int ncol = static_cast<int>((te - hb) >> 3);
+        const uint4* __restrict__ g8 = reinterpret_cast<const uint4*>(g + hb);
         for (int c0 = 0; c0 < ncol; c0 += kThreads * UNROLL) {
-            float v[UNROLL][8];
+            uint4 raw[UNROLL];
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const int c = c0 + u * kThreads + tid;
-                if (c < ncol) {
-                    Vec16IO<T, 8>::ld(g + hb + static_cast<long long>(c) * 8, v[u]);
-                } else {
-#pragma unroll
-                    for (int t = 0; t < 8; ++t) v[u][t] = 0.f;
-                }
+                raw[u] = (c < ncol) ? __ldcs(g8 + c) : make_uint4(0u, 0u, 0u, 0u);      // all-zero bits are 0.0 in both types
             }
             float a[8];
 #pragma unroll
             for (int t = 0; t < 8; ++t) a[t] = 0.f;
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
+                float v[8];
+                unpack8<T>(raw[u], v);
 #pragma unroll
-                for (int t = 0; t < 8; ++t) a[t] = fmaf(v[u][t], v[u][t], a[t]);
+                for (int t = 0; t < 8; ++t) a[t] = fmaf(v[t], v[t], a[t]);
             }
             dacc += ((static_cast<double>(a[0]) + static_cast<double>(a[1])) + (static_cast<double>(a[2]) + static_cast<double>(a[3]))) +
                     ((static_cast<double>(a[4]) + static_cast<double>(a[5])) + (static_cast<double>(a[6]) + static_cast<double>(a[7])));
@@ -151,15 +135,34 @@ sumsq16_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
     }
 }
 
-// Shape of the 16-bit centre+pull kernel: 16-byte columns (8 elements) up to 8 workers, 8-byte
-// columns (4 elements) above, so that a thread never holds more than 64 values; the elements one
-// CTA covers per pass come out the same as for fp32 (pull_pass_elems).
-__host__ __device__ constexpr int pull16_vec(int M) { return (M <= 8) ? 8 : 4; }
+// Shape of the 16-bit centre+pull kernel: columns of WORDS 32-bit words (two elements each) kept
+// packed in registers: 16-byte columns up to 8 workers, 8-byte columns above, and half the fp32
+// kernel's columns per thread, so that a thread holds at most 32 packed registers and a CTA covers
+// the same number of elements per pass as the fp32 kernel (the work lists are shared).
+__host__ __device__ constexpr int pull16_words(int M) { return (M <= 8) ? 4 : 2; }
 __host__ __device__ constexpr int pull16_cols(int M) { return (M <= 2) ? 4 : (M <= 4) ? 2 : 1; }
-static_assert(kThreads * pull16_cols(2) * pull16_vec(2) == pull_pass_elems(2), "pass size differs from fp32");
-static_assert(kThreads * pull16_cols(4) * pull16_vec(4) == pull_pass_elems(4), "pass size differs from fp32");
-static_assert(kThreads * pull16_cols(8) * pull16_vec(8) == pull_pass_elems(8), "pass size differs from fp32");
-static_assert(kThreads * pull16_cols(16) * pull16_vec(16) == pull_pass_elems(16), "pass size differs from fp32");
+static_assert(kThreads * pull16_cols(2) * pull16_words(2) * 2 == pull_pass_elems(2), "pass size differs from fp32");
+static_assert(kThreads * pull16_cols(4) * pull16_words(4) * 2 == pull_pass_elems(4), "pass size differs from fp32");
+static_assert(kThreads * pull16_cols(8) * pull16_words(8) * 2 == pull_pass_elems(8), "pass size differs from fp32");
+static_assert(kThreads * pull16_cols(16) * pull16_words(16) * 2 == pull_pass_elems(16), "pass size differs from fp32");
+
+template <int WORDS> struct Words;
+template <> struct Words<4> {
+    static __device__ __forceinline__ void ld(const void* p, unsigned (&o)[4])
+    {
+        const uint4 r = __ldcs(reinterpret_cast<const uint4*>(p));
+        o[0] = r.x; o[1] = r.y; o[2] = r.z; o[3] = r.w;
+    }
+    static __device__ __forceinline__ void st(void* p, const unsigned (&o)[4]) { __stcs(reinterpret_cast<uint4*>(p), make_uint4(o[0], o[1], o[2], o[3])); }
+};
+template <> struct Words<2> {
+    static __device__ __forceinline__ void ld(const void* p, unsigned (&o)[2])
+    {
+        const uint2 r = __ldcs(reinterpret_cast<const uint2*>(p));
+        o[0] = r.x; o[1] = r.y;
+    }
+    static __device__ __forceinline__ void st(void* p, const unsigned (&o)[2]) { __stcs(reinterpret_cast<uint2*>(p), make_uint2(o[0], o[1])); }
+};
 
 template <typename T, int M>
 __device__ __forceinline__ void pull16_scalar(const MutPtrs& x, T* center, const float (&w)[M], float lambda, float oml,
@@ -185,7 +188,8 @@ center_pull16_kernel(MutPtrs x, T* __restrict__ center, const float* __restrict_
 {
     grid_dependency_sync();
     constexpr int COLS = pull16_cols(M);
-    constexpr int VEC = pull16_vec(M);
+    constexpr int WORDS = pull16_words(M);
+    constexpr int VEC = 2 * WORDS;                 // elements per column
     const float oml = 1.0f - lambda;
     const int tid = threadIdx.x;
     float w[M];
@@ -210,35 +214,55 @@ center_pull16_kernel(MutPtrs x, T* __restrict__ center, const float* __restrict_
         split_range16(b, e, vec_ok, hb, te);
         const int ncol = static_cast<int>((te - hb) / VEC);      // te - hb is a multiple of 8
         for (int c0 = 0; c0 < ncol; c0 += kThreads * COLS) {
-            float v[COLS][M][VEC];
+            unsigned raw[COLS][M][WORDS];
 #pragma unroll
             for (int q = 0; q < COLS; ++q) {
                 const int c = c0 + q * kThreads + tid;
                 if (c < ncol) {
 #pragma unroll
                     for (int m = 0; m < M; ++m)
-                        Vec16IO<T, VEC>::ld(reinterpret_cast<const T*>(x.p[m]) + hb + static_cast<long long>(c) * VEC, v[q][m]);
+                        Words<WORDS>::ld(reinterpret_cast<const T*>(x.p[m]) + hb + static_cast<long long>(c) * VEC, raw[q][m]);
                 }
             }
 #pragma unroll
             for (int q = 0; q < COLS; ++q) {
                 const int c = c0 + q * kThreads + tid;
                 if (c < ncol) {
+                    // centre of the column's elements (fp32 FMA chain over the workers)
                     float cc[VEC];
 #pragma unroll
-                    for (int t = 0; t < VEC; ++t) cc[t] = w[0] * v[q][0][t];
+                    for (int k = 0; k < WORDS; ++k) {
+                        float lo, hi;
+                        Pair16<T>::unpack(raw[q][0][k], lo, hi);
+                        cc[2 * k] = w[0] * lo;
+                        cc[2 * k + 1] = w[0] * hi;
+                    }
 #pragma unroll
                     for (int m = 1; m < M; ++m) {
 #pragma unroll
-                        for (int t = 0; t < VEC; ++t) cc[t] = fmaf(w[m], v[q][m][t], cc[t]);
+                        for (int k = 0; k < WORDS; ++k) {
+                            float lo, hi;
+                            Pair16<T>::unpack(raw[q][m][k], lo, hi);
+                            cc[2 * k] = fmaf(w[m], lo, cc[2 * k]);
+                            cc[2 * k + 1] = fmaf(w[m], hi, cc[2 * k + 1]);
+                        }
                     }
-                    if (center) Vec16IO<T, VEC>::st(center + hb + static_cast<long long>(c) * VEC, cc);
+                    if (center) {
+                        unsigned o[WORDS];
+#pragma unroll
+                        for (int k = 0; k < WORDS; ++k) o[k] = Pair16<T>::pack(cc[2 * k], cc[2 * k + 1]);
+                        Words<WORDS>::st(center + hb + static_cast<long long>(c) * VEC, o);
+                    }
 #pragma unroll
                     for (int m = 0; m < M; ++m) {
-                        float o[VEC];
+                        unsigned o[WORDS];
 #pragma unroll
-                        for (int t = 0; t < VEC; ++t) o[t] = fmaf(lambda, cc[t], oml * v[q][m][t]);
-                        Vec16IO<T, VEC>::st(reinterpret_cast<T*>(x.p[m]) + hb + static_cast<long long>(c) * VEC, o);
+                        for (int k = 0; k < WORDS; ++k) {
+                            float lo, hi;
+                            Pair16<T>::unpack(raw[q][m][k], lo, hi);
+                            o[k] = Pair16<T>::pack(fmaf(lambda, cc[2 * k], oml * lo), fmaf(lambda, cc[2 * k + 1], oml * hi));
+                        }
+                        Words<WORDS>::st(reinterpret_cast<T*>(x.p[m]) + hb + static_cast<long long>(c) * VEC, o);
                     }
                 }
             }
