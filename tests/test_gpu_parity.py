@@ -474,3 +474,23 @@ def test_parity_one_huge_layer_among_small_ones(grawa):
     res = gpu_step(grawa, "lgrawa", p, g, 0.5, off)
     assert np.array_equal(res["S"], oracle.sumsq(g, off))
     compare_with_oracle(res, "lgrawa", p, g, 0.5, off)
+
+
+@pytest.mark.parametrize("M,sizes", [(1, [10, 5000, 3]), (3, [7, 5, 3, 1, 2, 6]), (5, [10, 3_000_001, 0, 3, 1_200_001, 777]),
+                                     (20, [100001, 33, 200001])],
+                         ids=["one-worker", "tiny", "chunked", "many-workers"])
+def test_host_buffer_entry_point_on_ragged_problems(grawa, M, sizes):
+    """The host-buffer call runs centre+pull chunk by chunk (several chunks for the large case);
+    chunk cuts, unaligned layer edges and the many-worker kernel must give the device-buffer result."""
+    cfg = gen.custom_config(sizes, M, seed=300 + M, log10_sigma=(-2.0, 0.0))
+    p, g = gen.make_inputs(cfg)
+    off = cfg.offsets()
+    for variant in ("mgrawa", "lgrawa"):
+        hp = [a.copy() for a in p]
+        hc = np.full(cfg.n, np.nan, np.float32)
+        grawa.grawa_step_host(variant, hp, g, 0.5, off, hc)
+        dev = gpu_step(grawa, variant, p, g, 0.5, off)
+        assert np.array_equal(hc, dev["center"].cpu().numpy())
+        for m in range(M):
+            assert np.array_equal(hp[m], dev["workers"][m].cpu().numpy())
+        compare_with_oracle(dev, variant, p, g, 0.5, off, check_workers=(M > 1))
