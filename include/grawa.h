@@ -37,7 +37,11 @@
  *     gradients) gives that worker weight 0, the rest are normalised among themselves (uniform
  *     1/M if none is finite), and the step's status word is set; see grawa_last_step_status.
  *   - Errors detectable on the host return a negative code before anything is enqueued.
- *     Nothing on the device traps or waits.
+ *     Nothing on the device traps.  The only device-side waits are the bulk-copy kernel's waits
+ *     for its own copies; each is bounded and reports GRAWA_ERR_TIMEOUT instead of hanging.
+ *   - A plan (and its device memory) lives until grawa_clear_plans(); a program that meets many
+ *     different shapes or streams should call it now and then.  Steps that share a plan (same
+ *     device, stream, shape) must not overlap on the GPU; the stream order guarantees that.
  *   - There is no CPU implementation behind this interface.
  */
 #ifndef GRAWA_H
@@ -84,8 +88,10 @@ const char *grawa_status_string(grawa_status status);
 /* Text of the last CUDA error seen by the calling thread ("" if none). */
 const char *grawa_last_cuda_error(void);
 
-/* Bytes of device scratch a step needs for this problem (partial sums, S, A, beta, status).
- * layer_offsets may be NULL with n_layers = 0 (one layer).  Returns 0 on invalid arguments. */
+/* Bytes of device scratch a step needs for this problem (partial sums, S, A, beta, status), for
+ * any storage type (16-bit storage needs no more than fp32).  layer_offsets may be NULL with
+ * n_layers = 0 (one layer).  Returns 0 on invalid arguments.  The value depends on the
+ * "sumsq_tile" option in force. */
 size_t grawa_workspace_bytes(int64_t n, int M, const int64_t *layer_offsets, int n_layers);
 
 /* MGRAWA step (Eq. 3-4, then centre and pull): one weight per worker from the sum of its
