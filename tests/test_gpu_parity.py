@@ -494,3 +494,31 @@ def test_host_buffer_entry_point_on_ragged_problems(grawa, M, sizes):
         for m in range(M):
             assert np.array_equal(hp[m], dev["workers"][m].cpu().numpy())
         compare_with_oracle(dev, variant, p, g, 0.5, off, check_workers=(M > 1))
+
+
+def test_more_than_2_to_31_elements_per_worker(grawa):
+    """Index arithmetic beyond 32 bits: 2^31 + 12345 elements per worker (34 GB on the device for two
+    workers), one layer of 2^31 - 5 elements and a short one behind it.  Sums of squares are checked
+    in full against the oracle, centre and workers on ranges at the start, across 2^31 and at the end."""
+    import torch
+    n = (1 << 31) + 12345
+    off = np.array([0, (1 << 31) - 5, n], dtype=np.int64)
+    block = gen.make_inputs(gen.custom_config([1 << 20], 4, seed=404, log10_sigma=(-2.0, 0.0)))
+    reps = n // (1 << 20) + 1
+    p = [np.tile(block[0][m], reps)[:n] for m in range(2)]
+    g = [np.tile(block[1][m + 2], reps)[:n] * np.float32(1 + m) for m in range(2)]
+    g[1][-12345:] *= np.float32(5.0)                       # the short layer gets different weights
+    res = gpu_step(grawa, "lgrawa", p, g, 0.5, off)
+    S = oracle.sumsq(g, off)
+    assert np.allclose(res["S"], S, rtol=1e-6, atol=0)
+    beta, _ = oracle.weights(oracle.scores(S, "lgrawa"))
+    assert np.abs(res["beta"] / beta - 1).max() <= 1e-5
+    assert abs(beta[0, 0] - beta[1, 0]) > 0.1              # the two layers really differ
+    tol = 2e-6 * max(float(np.abs(a).max()) for a in p)
+    centre = res["center"]
+    for j0, j1 in [(0, 1 << 20), ((1 << 31) - (1 << 19), (1 << 31) + 12345), (n - (1 << 18), n)]:
+        c, w = oracle.center_pull(p, beta, 0.5, off, j0, j1)
+        assert np.abs(centre[j0:j1].cpu().numpy() - c).max() <= tol
+        for m in range(2):
+            assert np.abs(res["workers"][m][j0:j1].cpu().numpy() - w[m]).max() <= tol
+    assert grawa.grawa_last_step_status() == 0
