@@ -13,8 +13,8 @@
  *   3. weights  beta_m = (1/A_m) / sum_i (1/A_i), sum_m beta_m = 1 (Eq. 2, Eq. 4); LGRAWA does
  *               this separately in every layer (Eq. 7)
  *   4. centre   x_C[j] = sum_m beta_{m,layer(j)} x_m[j]            (display under Eq. 2; Eq. 7)
- *   5. pull     x_m[j] <- (1-pull) x_m[j] + pull x_C[j]            (same display; last line of
- *               Algorithms 1 and 2), x_C taken from the values before the pull.
+ *   5. pull     x_m[j] <- (1-pull) x_m[j] + pull x_C[j]            (same display; the distributed
+ *               update of Algorithms 1 and 2), x_C taken from the values before the pull.
  *
  * Conventions common to every entry point
  *   - `params`, `grads`: HOST arrays of M DEVICE pointers, each to n contiguous fp32 values.
@@ -148,7 +148,7 @@ grawa_status grawa_step_host(grawa_variant variant, float *const *params, const 
  * synchronisation itself fails, GRAWA_ERR_INVALID_ARG if no step was enqueued on it). */
 grawa_status grawa_last_step_status(grawa_stream_t stream);
 
-/* Proximity-search step of the local phase (the line marked "Prox." in Algorithms 1 and 2):
+/* Proximity-search step of the local phase (the "Prox." update of Algorithms 1 and 2):
  * x_m[j] <- (1 - mu_over_tau) x_m[j] + mu_over_tau * center[j] for all M workers in one pass,
  * with `center` (DEVICE, n fp32, read only) the centre stored by the last averaging step.
  * mu_over_tau must lie in [0, 1]. */

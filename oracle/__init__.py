@@ -159,7 +159,7 @@ def step(params, grads, pull, variant, layer_offsets=None):
 
 
 def prox(params, center, mu_over_tau):
-    """Proximity step of the local phase: x_m <- (1 - mu/tau) x_m + (mu/tau) x_C (Algorithm 1, "Prox." line)."""
+    """Proximity step of the local phase: x_m <- (1 - mu/tau) x_m + (mu/tau) x_C (the "Prox." update of Algorithm 1)."""
     x = _f32_list(params)
     c = _f32_list([center])[0]
     outs = [np.zeros(c.size, dtype=np.float64) for _ in x]

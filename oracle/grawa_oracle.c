@@ -18,7 +18,7 @@
  *   3. weights  beta_m = (1/A_m) / sum_i (1/A_i)         (Eq. 2, Eq. 4; per layer in Eq. 7)
  *   4. centre   x_C[j] = sum_m beta_{m,k(j)} x_m[j]      (display after Eq. 2; Eq. 7 + construct)
  *   5. pull     x_m[j] <- (1-lambda) x_m[j] + lambda x_C[j], every worker, x_C from the
- *               values before the pull (Algorithm 1 / Algorithm 2, last two lines)
+ *               values before the pull (the distributed update of Algorithm 1 / Algorithm 2)
  *
  * Readings where the paper is silent (both sides of the parity tests use them):
  *   - a score that is exactly 0: the limit of 1/A -> infinity.  Within one
@@ -169,7 +169,7 @@ int grawa_oracle_step(const float *const *x, const float *const *grads, int64_t 
     return flagged;
 }
 
-/* Proximity search step of the local phase (Algorithm 1 / 2, the line marked "Prox."):
+/* Proximity search step of the local phase (the "Prox." update of Algorithm 1 / 2):
  * x_m[j] <- (1 - mu/tau) x_m[j] + (mu/tau) x_C[j], with the stored centre. */
 void grawa_oracle_prox(const float *const *x, int M, const float *center, int64_t n,
                        double mu_over_tau, double *const *x_out)

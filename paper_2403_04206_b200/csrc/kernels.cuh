@@ -536,7 +536,7 @@ copy_kernel(const float* __restrict__ src, float* __restrict__ dst, long long n,
     for (long long i = (n4 << 2) + t; i < n; i += stride) dst[i] = src[i];
 }
 
-// Proximity step ("Prox." line of Algorithms 1-2): x_m <- fmaf(a, x_C, (1-a) x_m), a = mu/tau.
+// Proximity step (the "Prox." update of Algorithms 1-2): x_m <- fmaf(a, x_C, (1-a) x_m), a = mu/tau.
 // One CTA per flat tile; the centre column is loaded once and reused for all M workers.
 __global__ void __launch_bounds__(kThreads)
 prox_kernel(MutPtrs x, const float* __restrict__ center, long long n, int tile, float a, int M, int vec_ok)
