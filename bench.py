@@ -204,8 +204,8 @@ def max_over_ranks(values, world, device):
     """Element-wise maximum of per-rank timings (the slowest rank defines the step time)."""
     import torch
     t = torch.tensor(list(values), dtype=torch.float64, device=device)
-    if world > 1:
-        import torch.distributed as dist
+    import torch.distributed as dist
+    if world > 1 or (dist.is_available() and dist.is_initialized()):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return [float(v) for v in t]
 
@@ -246,7 +246,8 @@ def run_cuda(args):
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     torch.cuda.set_device(local_rank)
-    if world > 1:
+    use_dist = "WORLD_SIZE" in os.environ and "MASTER_ADDR" in os.environ    # launched by torchrun, any world size
+    if use_dist:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
     import paper_2403_04206_b200 as grawa
@@ -264,7 +265,7 @@ def run_cuda(args):
     torch.cuda.synchronize()
 
     def barrier():
-        if world > 1:
+        if use_dist:
             dist.barrier()
         torch.cuda.synchronize()
 
@@ -330,7 +331,7 @@ def run_cuda(args):
         if world == 1 and args.also:
             line["also"] = also_runs(grawa, args, exclude=(args.workload, variant))
         print(json.dumps(line), flush=True)
-    if world > 1:
+    if use_dist:
         dist.barrier()
         dist.destroy_process_group()
 
