@@ -237,6 +237,12 @@ grawa_status grawa_step_from_layer_sums(grawa_variant variant, float *const *par
 grawa_status grawa_sumsq_static(const float *const *grads, int64_t n, int M, double *sumsq_out,
                                 grawa_stream_t stream);
 
+/* Self-test of the library's bounded device waits: launches one small kernel that waits on a
+ * barrier nobody signals.  The wait must give up after limit_ns (1 us .. 1 s) of wall time, the
+ * kernel records the timeout and returns, and grawa_last_step_status(stream) then reports
+ * GRAWA_ERR_TIMEOUT with the context still usable.  Touches no caller memory. */
+grawa_status grawa_selftest_bounded_wait(int64_t limit_ns, grawa_stream_t stream);
+
 /* Tuning knobs, process wide; they change speed, never results beyond fp32 summation order
  * of the sums of squares ("sumsq_tile").  Returns GRAWA_ERR_INVALID_ARG for an unknown name
  * or a value out of range.

@@ -22,6 +22,7 @@ from .binding import (  # noqa: F401
     grawa_lgrawa_step,
     grawa_mgrawa_step,
     grawa_prox_step,
+    grawa_selftest_bounded_wait,
     grawa_set_option,
     grawa_status_string,
     grawa_step_host,

@@ -81,6 +81,8 @@ def library() -> ctypes.CDLL:
     lib.grawa_step_from_layer_sums.restype = ci
     lib.grawa_sumsq_static.argtypes = [vp, i64, ci, vp, vp]
     lib.grawa_sumsq_static.restype = ci
+    lib.grawa_selftest_bounded_wait.argtypes = [i64, vp]
+    lib.grawa_selftest_bounded_wait.restype = ci
     lib.grawa_collect_kernel_times.argtypes = [vp, vp, vp, vp]
     lib.grawa_collect_kernel_times.restype = ci
     _lib = lib
@@ -366,6 +368,11 @@ def grawa_collect_kernel_times() -> dict:
     _raise(library().grawa_collect_kernel_times(ctypes.byref(a), ctypes.byref(b), ctypes.byref(c), ctypes.byref(k)),
            "grawa_collect_kernel_times")
     return {"sumsq_ms": a.value, "finalize_ms": b.value, "center_pull_ms": c.value, "steps": k.value}
+
+
+def grawa_selftest_bounded_wait(limit_ns: int, *, stream=None) -> None:
+    """Launches the bounded-wait self-test; read the outcome with grawa_last_step_status (expect -5)."""
+    _raise(library().grawa_selftest_bounded_wait(int(limit_ns), _stream(stream)), "grawa_selftest_bounded_wait")
 
 
 def grawa_clear_plans() -> None:

@@ -4,7 +4,7 @@
 // stores.  One CTA per SM keeps a ring of stages in flight; work items are claimed from an atomic
 // counter so that faster SMs take more of them.
 //
-// Every wait is bounded: when a barrier does not complete within the poll limit the CTA records
+// Every wait is bounded: when a barrier does not complete within the time limit the CTA records
 // kStatusTimeout in the status word, drains what it has in flight (again bounded) and returns.
 #pragma once
 #include "kernels.cuh"
@@ -12,7 +12,7 @@
 namespace grawa {
 
 constexpr int kBulkMaxStages = 8;
-constexpr unsigned kBulkPollLimit = 1u << 22;   // polls of mbarrier.try_wait before giving up
+constexpr unsigned long long kBulkWaitLimitNs = 2000000000ull;   // a wait gives up after 2 s of wall time
 
 struct BulkStageInfo {
     long long begin;   // first element of the item
@@ -42,12 +42,22 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned 
         : "memory");
     return ok != 0;
 }
-// Bounded wait; false when the poll limit ran out.
-__device__ __forceinline__ bool mbar_wait_bounded(unsigned long long* bar, unsigned parity)
+__device__ __forceinline__ unsigned long long global_timer_ns()
 {
-    for (unsigned i = 0; i < kBulkPollLimit; ++i)
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait; false when `limit_ns` of wall time passed without the phase completing.
+__device__ __forceinline__ bool mbar_wait_bounded(unsigned long long* bar, unsigned parity,
+                                                  unsigned long long limit_ns = kBulkWaitLimitNs)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
-    return false;
+        if (global_timer_ns() - t0 > limit_ns) return false;
+    }
 }
 // global -> shared (this CTA's own shared memory), completion counted in bytes on `bar`.
 __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, unsigned bytes, unsigned long long* bar)
@@ -240,9 +250,25 @@ center_pull_bulk_kernel(MutPtrs x, float* __restrict__ center, const float* __re
         // loads that may still be in flight into this CTA's shared memory: wait for them, bounded
         for (int j = 0; j < stages; ++j) {
             const int jt = it + j;
-            (void)mbar_wait_bounded(&full_bar[jt % stages], static_cast<unsigned>(jt / stages) & 1u);
+            (void)mbar_wait_bounded(&full_bar[jt % stages], static_cast<unsigned>(jt / stages) & 1u, 100000000ull);
         }
     }
+}
+
+// Self-test of the bounded wait: a barrier that nobody ever arrives on.  Every thread's wait must
+// give up after `limit_ns` and the kernel must record kStatusTimeout and return.  No memory is
+// touched besides the status word.
+__global__ void __launch_bounds__(kThreads)
+bounded_wait_selftest_kernel(int* __restrict__ status, unsigned long long limit_ns)
+{
+    __shared__ __align__(8) unsigned long long bar;
+    if (threadIdx.x == 0) {
+        mbar_init(&bar, 1u);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncthreads();
+    const bool ok = mbar_wait_bounded(&bar, 0u, limit_ns);
+    if (__syncthreads_or(ok ? 0 : 1) && threadIdx.x == 0) atomicOr(status, kStatusTimeout);
 }
 
 }  // namespace grawa

@@ -993,6 +993,22 @@ grawa_status grawa_sumsq_static(const float* const* grads, int64_t n, int M, dou
     return GRAWA_OK;
 }
 
+grawa_status grawa_selftest_bounded_wait(int64_t limit_ns, grawa_stream_t stream)
+{
+    if (limit_ns < 1000 || limit_ns > 1000000000) return GRAWA_ERR_INVALID_ARG;
+    int device = 0;
+    GRAWA_CUDA_TRY(cudaGetDevice(&device));
+    if (device < 0 || device >= kMaxDevices) return GRAWA_ERR_INVALID_ARG;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    static int* words[kMaxDevices] = {};
+    if (words[device] == nullptr) GRAWA_CUDA_TRY(cudaMalloc(&words[device], sizeof(int)));
+    GRAWA_CUDA_TRY(cudaMemsetAsync(words[device], 0, sizeof(int), stream));
+    g_last_status[{device, stream}] = words[device];
+    GRAWA_CUDA_TRY(launch_kernel(bounded_wait_selftest_kernel, 1, kThreads, stream, false, words[device],
+                                 static_cast<unsigned long long>(limit_ns)));
+    return GRAWA_OK;
+}
+
 static void clear_plans_locked()
 {
     cudaDeviceSynchronize();

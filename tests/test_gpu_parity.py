@@ -522,3 +522,24 @@ def test_more_than_2_to_31_elements_per_worker(grawa):
         for m in range(2):
             assert np.abs(res["workers"][m][j0:j1].cpu().numpy() - w[m]).max() <= tol
     assert grawa.grawa_last_step_status() == 0
+
+
+def test_bounded_device_wait_times_out_and_the_context_stays_usable(grawa):
+    """A wait that nothing will ever satisfy (a barrier nobody signals, inside the library's own
+    self-test kernel) must give up after its time limit, report GRAWA_ERR_TIMEOUT through the status
+    word, and leave the context healthy: the next step runs and is correct."""
+    import time
+    import torch
+    t0 = time.perf_counter()
+    grawa.grawa_selftest_bounded_wait(2_000_000)            # 2 ms limit
+    assert grawa.grawa_last_step_status() == -5
+    assert time.perf_counter() - t0 < 1.0
+    assert "wait" in grawa.grawa_status_string(-5)
+    with pytest.raises(grawa.GrawaError):
+        grawa.grawa_selftest_bounded_wait(10)               # limit out of range: rejected on the host
+    cfg = gen.custom_config([10, 5000, 3, 9000], 4, seed=21)
+    p, g = gen.make_inputs(cfg)
+    res = gpu_step(grawa, "lgrawa", p, g, 0.5, cfg.offsets())
+    compare_with_oracle(res, "lgrawa", p, g, 0.5, cfg.offsets())
+    assert grawa.grawa_last_step_status() == 0
+    torch.cuda.synchronize()
