@@ -224,6 +224,26 @@ TRAFFIC_CAPTURE = {"M": 16, "dram_bytes_per_element": 1916.086016e6 / 14918400,
                    "kernels_sha256": "dfe4c7fc8a7a1661c74c90bc473b55c2492cfc82aca6445c50cd3cb601430930"}
 
 
+# Same for the sum-of-squares kernel (profiles/sumsq_kernel_vit_b16_28layers.md: 954.82 MB read +
+# 4.01 MB written for 14 918 400 elements at M = 16).
+SUMSQ_TRAFFIC_CAPTURE = {"M": 16, "dram_bytes_per_element": (954.823424e6 + 4.00512e6) / 14918400,
+                         "kernels_sha256": "ed96401d750197f1f341cbb1f21abe7a9ec683a46225b06beab3b8644c3b75c2"}
+
+
+def sumsq_traffic(cfg):
+    import hashlib
+    path = os.path.join(ROOT, "paper_2403_04206_b200", "csrc", "kernels.cuh")
+    try:
+        text = open(path).read()
+        region = text[text.index("// Step 1 (Eq. 3 / Eq. 5): partial[m][s]"):text.index("// Steps 1b-3: one CTA per layer reduces")]
+        digest = hashlib.sha256(region.encode()).hexdigest()
+    except (OSError, ValueError):
+        return None
+    if digest != SUMSQ_TRAFFIC_CAPTURE["kernels_sha256"] or cfg.M != SUMSQ_TRAFFIC_CAPTURE["M"]:
+        return None
+    return SUMSQ_TRAFFIC_CAPTURE["dram_bytes_per_element"] * cfg.n
+
+
 def center_pull_traffic(cfg):
     import hashlib
     path = os.path.join(ROOT, "paper_2403_04206_b200", "csrc", "kernels.cuh")
@@ -318,7 +338,8 @@ def run_cuda(args):
                          "other_kernels": {
                              "sumsq": {"algorithmic_bytes_per_launch": sumsq_bytes, "kernel_ms": sumsq_ms,
                                        "achieved": sumsq_bytes / (sumsq_ms * 1e-3) / 1e9,
-                                       "frac": sumsq_bytes / (sumsq_ms * 1e-3) / 1e9 / peak},
+                                       "frac": sumsq_bytes / (sumsq_ms * 1e-3) / 1e9 / peak,
+                                       "traffic": sumsq_traffic(cfg)},
                              "finalize": {"kernel_ms": fin_ms}},
                          "ms_per_step_with_events": ms_k},
             "e2e": {"value": whole_job_steps_per_s(world, e2e_ms_max), "unit": "steps/s", "steps": e2e_steps,
