@@ -27,7 +27,7 @@ def _worker(rank, world, port, out):
 
 
 def test_timing_is_the_max_over_two_gloo_ranks():
-    with mp.Manager() as manager:
+    with mp.get_context("spawn").Manager() as manager:
         out = manager.dict()
         mp.spawn(_worker, args=(2, 29533, out), nprocs=2, join=True)
         assert out[0] == out[1] == [3.0, 300.0]

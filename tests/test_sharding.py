@@ -66,7 +66,7 @@ def _gloo_worker(rank, world, port, out):
 
 
 def test_two_gloo_ranks_reproduce_the_unsharded_result():
-    with mp.Manager() as manager:
+    with mp.get_context("spawn").Manager() as manager:
         out = manager.dict()
         mp.spawn(_gloo_worker, args=(2, 29541, out), nprocs=2, join=True)
         cfg = gen.custom_config([10, 5000, 0, 3, 12001, 777], 3, seed=91, log10_sigma=(-2.0, 0.0))
