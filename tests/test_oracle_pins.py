@@ -365,3 +365,41 @@ def test_norm_ema_bias_correction_cancels_in_the_weights():
     beta_est = oracle.weights(est[:, 0])[0]
     beta_mvg = oracle.weights(mvg[:, 0])[0]
     assert np.allclose(beta_est, beta_mvg, rtol=1e-13)
+
+
+# ---------------------------------------------------------------- property-based checks
+
+from hypothesis import given, settings, strategies as st
+
+
+@settings(max_examples=60, deadline=None)
+@given(st.lists(st.floats(min_value=1e-6, max_value=1e6, allow_nan=False, allow_infinity=False), min_size=1, max_size=16))
+def test_weights_properties_hold_for_any_positive_scores(scores):
+    A = np.array(scores)
+    beta, flagged = oracle.weights(A)
+    assert not flagged
+    assert abs(beta.sum() - 1.0) <= 1e-13 and np.all(beta > 0) and np.all(beta <= 1)
+    assert np.allclose(beta * A, (beta * A)[0], rtol=1e-12)            # beta_m A_m is the same for all m (= Theta)
+    assert (beta * A)[0] <= A.min() * (1 + 1e-12)                      # Theta <= every norm
+
+
+@settings(max_examples=25, deadline=None)
+@given(st.integers(min_value=1, max_value=6), st.lists(st.integers(min_value=0, max_value=9), min_size=1, max_size=5),
+       st.floats(min_value=0.0, max_value=1.0), st.integers(min_value=0, max_value=10_000))
+def test_step_invariants_on_random_small_problems(M, sizes, lam, seed):
+    n = sum(sizes)
+    if n == 0:
+        return
+    r = np.random.default_rng(seed)
+    off = np.concatenate([[0], np.cumsum(sizes)])
+    x = [f32(r.normal(size=n)) for _ in range(M)]
+    g = [f32(r.normal(size=n) * 10.0 ** r.uniform(-2, 1)) for _ in range(M)]
+    for variant in ("grawa", "mgrawa", "lgrawa"):
+        out = oracle.step(x, g, lam, variant, off)
+        X = np.stack(x).astype(np.float64)
+        c = out["center"]
+        assert np.all(c >= X.min(axis=0) - 1e-12) and np.all(c <= X.max(axis=0) + 1e-12)
+        W = np.stack(out["workers"])
+        assert np.allclose(W, (1 - lam) * X + lam * c[None, :], rtol=1e-13, atol=1e-15)
+        b = out["beta"]
+        assert np.allclose(b.sum(axis=-1), 1.0, atol=1e-13)
