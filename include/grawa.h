@@ -243,6 +243,14 @@ grawa_status grawa_sumsq_static(const float *const *grads, int64_t n, int M, dou
  * GRAWA_ERR_TIMEOUT with the context still usable.  Touches no caller memory. */
 grawa_status grawa_selftest_bounded_wait(int64_t limit_ns, grawa_stream_t stream);
 
+/* Debug build only (the library compiled with -DGRAWA_DEBUG_BOUNDS, which checks every global access
+ * of the streaming kernels against the vector length, counts violations and skips them): returns
+ * the number of violations on the current device since the last call and resets it; synchronises
+ * the device.  With selfcheck != 0 it first feeds the checker three out-of-range index triples
+ * (arithmetic only, no memory access), so a healthy debug build returns exactly 3 more.
+ * Returns -1 in the normal build, -2 on a CUDA error. */
+int64_t grawa_debug_bounds_violations(int selfcheck);
+
 /* Tuning knobs, process wide; they change speed, never results beyond fp32 summation order
  * of the sums of squares ("sumsq_tile").  Returns GRAWA_ERR_INVALID_ARG for an unknown name
  * or a value out of range.

@@ -9,6 +9,7 @@ from .binding import (  # noqa: F401
     GRAWA_MAX_WORKERS,
     grawa_clear_plans,
     grawa_collect_kernel_times,
+    grawa_debug_bounds_violations,
     grawa_get_option,
     grawa_grawa_step,
     grawa_last_cuda_error,

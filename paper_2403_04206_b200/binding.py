@@ -41,7 +41,8 @@ def library() -> ctypes.CDLL:
     global _lib
     if _lib is not None:
         return _lib
-    path = _build.build()
+    import os
+    path = _build.build(debug_bounds=os.environ.get("GRAWA_DEBUG_BOUNDS", "0") == "1")
     lib = ctypes.CDLL(path)
     vp, i64, ci, cf = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_float
     step_args = [vp, vp, i64, ci, cf, vp, ci, vp, vp, vp]
@@ -81,6 +82,8 @@ def library() -> ctypes.CDLL:
     lib.grawa_step_from_layer_sums.restype = ci
     lib.grawa_sumsq_static.argtypes = [vp, i64, ci, vp, vp]
     lib.grawa_sumsq_static.restype = ci
+    lib.grawa_debug_bounds_violations.argtypes = [ci]
+    lib.grawa_debug_bounds_violations.restype = i64
     lib.grawa_selftest_bounded_wait.argtypes = [i64, vp]
     lib.grawa_selftest_bounded_wait.restype = ci
     lib.grawa_collect_kernel_times.argtypes = [vp, vp, vp, vp]
@@ -373,6 +376,11 @@ def grawa_collect_kernel_times() -> dict:
 def grawa_selftest_bounded_wait(limit_ns: int, *, stream=None) -> None:
     """Launches the bounded-wait self-test; read the outcome with grawa_last_step_status (expect -5)."""
     _raise(library().grawa_selftest_bounded_wait(int(limit_ns), _stream(stream)), "grawa_selftest_bounded_wait")
+
+
+def grawa_debug_bounds_violations(selfcheck: bool = False) -> int:
+    """Violations counted by a bounds-checking debug build since the last call (-1 in a normal build)."""
+    return int(library().grawa_debug_bounds_violations(1 if selfcheck else 0))
 
 
 def grawa_clear_plans() -> None:

@@ -9,6 +9,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "libgrawa.so")
+DEBUG_LIB_PATH = os.path.join(_HERE, "libgrawa_debug_bounds.so")
 SOURCES = [os.path.join(CSRC, "grawa.cu")]
 HEADERS = [os.path.join(CSRC, "kernels.cuh"), os.path.join(CSRC, "center_pull_bulk.cuh"), os.path.join(CSRC, "kernels_16bit.cuh"),
            os.path.join(_ROOT, "include", "grawa.h")]
@@ -25,15 +26,25 @@ def _nvcc() -> str:
     return exe
 
 
-def is_stale() -> bool:
-    if not os.path.exists(LIB_PATH):
+def is_stale(path: str = LIB_PATH) -> bool:
+    if not os.path.exists(path):
         return True
-    t = os.path.getmtime(LIB_PATH)
+    t = os.path.getmtime(path)
     return any(os.path.getmtime(p) > t for p in SOURCES + HEADERS)
 
 
-def build(force: bool = False, verbose: bool = False) -> str:
-    """Compile the CUDA library when missing or older than its sources; returns its path."""
+def build(force: bool = False, verbose: bool = False, debug_bounds: bool = False) -> str:
+    """Compile the CUDA library when missing or older than its sources; returns its path.
+    debug_bounds: the variant whose kernels check every global access against the vector length."""
+    if debug_bounds:
+        if force or is_stale(DEBUG_LIB_PATH):
+            tmp = DEBUG_LIB_PATH + f".tmp{os.getpid()}"
+            cmd = [_nvcc()] + NVCC_FLAGS + ["-DGRAWA_DEBUG_BOUNDS", "-o", tmp] + SOURCES
+            res = subprocess.run(cmd, capture_output=True, text=True)
+            if res.returncode != 0:
+                raise RuntimeError("nvcc failed:\n" + " ".join(cmd) + "\n" + res.stdout + res.stderr)
+            os.replace(tmp, DEBUG_LIB_PATH)
+        return DEBUG_LIB_PATH
     if force or is_stale():
         tmp = LIB_PATH + f".tmp{os.getpid()}"
         cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + SOURCES

@@ -435,7 +435,7 @@ static grawa_status make_context(int variant, float* const* params, const float*
     }
     StepScratch& sc = ctx->sc;
     sc.segs = plan->d_segs1; sc.layer_seg_first = plan->d_layer_first;
-    sc.C = plan->C1; sc.K = K; sc.M = M; sc.variant = variant;
+    sc.C = plan->C1; sc.K = K; sc.M = M; sc.variant = variant; sc.n = n;
     sc.partials = reinterpret_cast<double*>(ws + plan->ws.partials);
     sc.S = reinterpret_cast<double*>(ws + plan->ws.S);
     sc.A = reinterpret_cast<double*>(ws + plan->ws.A);
@@ -1007,6 +1007,21 @@ grawa_status grawa_selftest_bounded_wait(int64_t limit_ns, grawa_stream_t stream
     GRAWA_CUDA_TRY(launch_kernel(bounded_wait_selftest_kernel, 1, kThreads, stream, false, words[device],
                                  static_cast<unsigned long long>(limit_ns)));
     return GRAWA_OK;
+}
+
+int64_t grawa_debug_bounds_violations(int selfcheck)
+{
+#ifdef GRAWA_DEBUG_BOUNDS
+    if (selfcheck) bounds_selfcheck_kernel<<<1, 32>>>();
+    if (cudaDeviceSynchronize() != cudaSuccess) return -2;
+    int count = 0, zero = 0;
+    if (cudaMemcpyFromSymbol(&count, g_bounds_violations, sizeof count) != cudaSuccess) return -2;
+    if (cudaMemcpyToSymbol(g_bounds_violations, &zero, sizeof zero) != cudaSuccess) return -2;
+    return count;
+#else
+    (void)selfcheck;
+    return -1;
+#endif
 }
 
 static void clear_plans_locked()

@@ -38,6 +38,31 @@ __device__ __forceinline__ void grid_dependency_sync()
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
+// Debug build (-DGRAWA_DEBUG_BOUNDS): every global access of the streaming kernels is first checked
+// against the vector's length; a violation is counted and the access skipped (nothing traps).
+// In the normal build the check is the constant `true` and costs nothing.
+#ifdef GRAWA_DEBUG_BOUNDS
+__device__ int g_bounds_violations = 0;
+__device__ __forceinline__ bool in_bounds(long long first, long long count, long long total)
+{
+    if (first >= 0 && count >= 0 && first + count <= total) return true;
+    atomicAdd(&g_bounds_violations, 1);
+    return false;
+}
+// Arithmetic-only check of the checker itself: three ranges that are out of bounds, one that is not.
+__global__ void bounds_selfcheck_kernel()
+{
+    if (threadIdx.x == 0) {
+        (void)in_bounds(-1, 1, 10);
+        (void)in_bounds(8, 4, 10);
+        (void)in_bounds(10, 1, 10);
+        (void)in_bounds(6, 4, 10);
+    }
+}
+#else
+__device__ __forceinline__ bool in_bounds(long long, long long, long long) { return true; }
+#endif
+
 // Streaming accesses: every byte is touched once per step, so keep it out of the way in L1/L2
 // (ld.global.cs / st.global.cs; measured equal to .nc.L1::no_allocate loads and better than
 // default-cached loads for the sum of squares).
@@ -83,6 +108,7 @@ struct StepScratch {
     const Segment* segs;           // sum-of-squares work items of one worker, C of them
     const int* layer_seg_first;    // first item of each layer, K+1 entries
     int C, K, M, variant;
+    long long n;                   // elements per worker (bounds checks of the debug build)
     double* partials;              // [M][C]
     double* S;                     // [K][M]
     double* A;                     // [K+1][M]: per-layer terms, then the per-worker scores in row K
@@ -315,7 +341,7 @@ sumsq_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const int c = c0 + u * kThreads + tid;
-                v[u] = (c < ncol) ? ld_stream4(g4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+                v[u] = (c < ncol && in_bounds(hb + 4LL * c, 4, sc.n)) ? ld_stream4(g4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
@@ -329,11 +355,11 @@ sumsq_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
                     (static_cast<double>(a2) + static_cast<double>(a3));
         }
         for (long long i = b + tid; i < hb; i += kThreads) {
-            const double v = static_cast<double>(ld_stream1(g + i));
+            const double v = in_bounds(i, 1, sc.n) ? static_cast<double>(ld_stream1(g + i)) : 0.0;
             dacc += v * v;
         }
         for (long long i = te + tid; i < e; i += kThreads) {
-            const double v = static_cast<double>(ld_stream1(g + i));
+            const double v = in_bounds(i, 1, sc.n) ? static_cast<double>(ld_stream1(g + i)) : 0.0;
             dacc += v * v;
         }
         // Fixed-order block sum.  Two alternating buffers need only one barrier per item: a warp
@@ -444,7 +470,7 @@ center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restric
 #pragma unroll
             for (int q = 0; q < COLS; ++q) {
                 const int c = c0 + q * kThreads + tid;
-                if (c < ncol) {
+                if (c < ncol && in_bounds(hb + static_cast<long long>(c) * VEC, VEC, n)) {
 #pragma unroll
                     for (int m = 0; m < M; ++m) VecIO<VEC>::ld(x.p[m] + hb + static_cast<long long>(c) * VEC, v[q][m]);
                 }
@@ -452,7 +478,7 @@ center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restric
 #pragma unroll
             for (int q = 0; q < COLS; ++q) {
                 const int c = c0 + q * kThreads + tid;
-                if (c < ncol) {
+                if (c < ncol && in_bounds(hb + static_cast<long long>(c) * VEC, VEC, n)) {
                     float cc[VEC];
 #pragma unroll
                     for (int t = 0; t < VEC; ++t) cc[t] = w[0] * v[q][0][t];
@@ -472,8 +498,10 @@ center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restric
                 }
             }
         }
-        for (long long i = b + tid; i < hb; i += kThreads) pull_scalar<M>(x, center, w, lambda, oml, i);
-        for (long long i = te + tid; i < e; i += kThreads) pull_scalar<M>(x, center, w, lambda, oml, i);
+        for (long long i = b + tid; i < hb; i += kThreads)
+            if (in_bounds(i, 1, n)) pull_scalar<M>(x, center, w, lambda, oml, i);
+        for (long long i = te + tid; i < e; i += kThreads)
+            if (in_bounds(i, 1, n)) pull_scalar<M>(x, center, w, lambda, oml, i);
     }
 }
 
@@ -501,6 +529,7 @@ center_pull_generic_kernel(MutPtrs x, float* __restrict__ center, const float* _
     __syncthreads();
     const float oml = 1.0f - lambda;
     for (long long i = b + threadIdx.x; i < e; i += kThreads) {
+        if (!in_bounds(i, 1, n)) continue;
         float c = w[0] * x.p[0][i];
         for (int m = 1; m < M; ++m) c = fmaf(w[m], x.p[m][i], c);
         if (center) center[i] = c;

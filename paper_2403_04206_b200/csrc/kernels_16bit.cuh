@@ -99,7 +99,7 @@ sumsq16_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const int c = c0 + u * kThreads + tid;
-                raw[u] = (c < ncol) ? __ldcs(g8 + c) : make_uint4(0u, 0u, 0u, 0u);      // all-zero bits are 0.0 in both types
+                raw[u] = (c < ncol && in_bounds(hb + 8LL * c, 8, sc.n)) ? __ldcs(g8 + c) : make_uint4(0u, 0u, 0u, 0u);      // all-zero bits are 0.0 in both types
             }
             float a[8];
 #pragma unroll
@@ -115,11 +115,11 @@ sumsq16_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
                     ((static_cast<double>(a[4]) + static_cast<double>(a[5])) + (static_cast<double>(a[6]) + static_cast<double>(a[7])));
         }
         for (long long i = b + tid; i < hb; i += kThreads) {
-            const double v = static_cast<double>(Pair16<T>::load1(g + i));
+            const double v = in_bounds(i, 1, sc.n) ? static_cast<double>(Pair16<T>::load1(g + i)) : 0.0;
             dacc += v * v;
         }
         for (long long i = te + tid; i < e; i += kThreads) {
-            const double v = static_cast<double>(Pair16<T>::load1(g + i));
+            const double v = in_bounds(i, 1, sc.n) ? static_cast<double>(Pair16<T>::load1(g + i)) : 0.0;
             dacc += v * v;
         }
 #pragma unroll
@@ -218,7 +218,7 @@ center_pull16_kernel(MutPtrs x, T* __restrict__ center, const float* __restrict_
 #pragma unroll
             for (int q = 0; q < COLS; ++q) {
                 const int c = c0 + q * kThreads + tid;
-                if (c < ncol) {
+                if (c < ncol && in_bounds(hb + static_cast<long long>(c) * VEC, VEC, n)) {
 #pragma unroll
                     for (int m = 0; m < M; ++m)
                         Words<WORDS>::ld(reinterpret_cast<const T*>(x.p[m]) + hb + static_cast<long long>(c) * VEC, raw[q][m]);
@@ -227,7 +227,7 @@ center_pull16_kernel(MutPtrs x, T* __restrict__ center, const float* __restrict_
 #pragma unroll
             for (int q = 0; q < COLS; ++q) {
                 const int c = c0 + q * kThreads + tid;
-                if (c < ncol) {
+                if (c < ncol && in_bounds(hb + static_cast<long long>(c) * VEC, VEC, n)) {
                     // centre of the column's elements (fp32 FMA chain over the workers)
                     float cc[VEC];
 #pragma unroll
@@ -267,8 +267,10 @@ center_pull16_kernel(MutPtrs x, T* __restrict__ center, const float* __restrict_
                 }
             }
         }
-        for (long long i = b + tid; i < hb; i += kThreads) pull16_scalar<T, M>(x, center, w, lambda, oml, i);
-        for (long long i = te + tid; i < e; i += kThreads) pull16_scalar<T, M>(x, center, w, lambda, oml, i);
+        for (long long i = b + tid; i < hb; i += kThreads)
+            if (in_bounds(i, 1, n)) pull16_scalar<T, M>(x, center, w, lambda, oml, i);
+        for (long long i = te + tid; i < e; i += kThreads)
+            if (in_bounds(i, 1, n)) pull16_scalar<T, M>(x, center, w, lambda, oml, i);
     }
 }
 
@@ -296,6 +298,7 @@ center_pull16_generic_kernel(MutPtrs x, T* __restrict__ center, const float* __r
     __syncthreads();
     const float oml = 1.0f - lambda;
     for (long long i = b + threadIdx.x; i < e; i += kThreads) {
+        if (!in_bounds(i, 1, n)) continue;
         float c = w[0] * Pair16<T>::load1(reinterpret_cast<const T*>(x.p[0]) + i);
         for (int m = 1; m < M; ++m) c = fmaf(w[m], Pair16<T>::load1(reinterpret_cast<const T*>(x.p[m]) + i), c);
         if (center) Pair16<T>::store1(center + i, c);
