@@ -216,18 +216,18 @@ def whole_job_steps_per_s(world, ms_per_step_max):
 
 
 # DRAM traffic of one centre+pull launch, from the ncu capture summarised in
-# profiles/center_pull_kernel_vit_b16_28layers.md (M = 16; 1916.09 MB for 14 918 400 elements),
+# profiles/center_pull_kernel_vit_b16_28layers.md (M = 16; 1916.46 MB for 14 918 400 elements),
 # scaled to a full launch by the number of elements.  Only valid for the kernel source it was taken
 # from: the hash below is that of the centre+pull kernel's text in csrc/kernels.cuh (from its
 # heading comment to the next kernel's) at capture time; anything else reports null.
-TRAFFIC_CAPTURE = {"M": 16, "dram_bytes_per_element": 1916.086016e6 / 14918400,
-                   "kernels_sha256": "dfe4c7fc8a7a1661c74c90bc473b55c2492cfc82aca6445c50cd3cb601430930"}
+TRAFFIC_CAPTURE = {"M": 16, "dram_bytes_per_element": (955.077376e6 + 961.380608e6) / 14918400,
+                   "kernels_sha256": "e63e74aaf440bb7584d4f7c4bf30a29a04d4fe74544ad2ec2a8e2d6753ce5a49"}
 
 
 # Same for the sum-of-squares kernel (profiles/sumsq_kernel_vit_b16_28layers.md: 954.82 MB read +
-# 4.01 MB written for 14 918 400 elements at M = 16).
-SUMSQ_TRAFFIC_CAPTURE = {"M": 16, "dram_bytes_per_element": (954.823424e6 + 4.00512e6) / 14918400,
-                         "kernels_sha256": "ed96401d750197f1f341cbb1f21abe7a9ec683a46225b06beab3b8644c3b75c2"}
+# 4.35 MB written for 14 918 400 elements at M = 16).
+SUMSQ_TRAFFIC_CAPTURE = {"M": 16, "dram_bytes_per_element": (954.82112e6 + 4.346368e6) / 14918400,
+                         "kernels_sha256": "3cad663f1177f4a514a5233796ed3df1eeae9242aa4c7b3b5f6ff7623fd66d56"}
 
 
 def sumsq_traffic(cfg):
