@@ -578,6 +578,7 @@ prox_kernel(MutPtrs x, const float* __restrict__ center, long long n, int tile, 
     split_range(b, e, vec_ok, hb, te);
     const int ncol = static_cast<int>((te - hb) >> 2);
     for (int c = threadIdx.x; c < ncol; c += kThreads) {
+        if (!in_bounds(hb + 4LL * c, 4, n)) continue;
         const float4 cc = ld_stream4(reinterpret_cast<const float4*>(center + hb) + c);
         int m = 0;
         for (; m + 4 <= M; m += 4) {
@@ -603,6 +604,7 @@ prox_kernel(MutPtrs x, const float* __restrict__ center, long long n, int tile, 
     for (int pass = 0; pass < 2; ++pass) {
         const long long lo = pass ? te : b, hi = pass ? e : hb;
         for (long long i = lo + threadIdx.x; i < hi; i += kThreads) {
+            if (!in_bounds(i, 1, n)) continue;
             const float c = center[i];
             for (int m = 0; m < M; ++m) x.p[m][i] = fmaf(a, c, oma * x.p[m][i]);
         }

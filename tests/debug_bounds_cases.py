@@ -38,6 +38,9 @@ def main():
                 c = torch.empty(cfg.n, dtype=dt, device="cuda")
                 grawa.grawa_step_typed("lgrawa", x, gr, 0.5, cfg.offsets(), c)
                 out["cases"] += 1
+            xs32 = [torch.from_numpy(a).cuda() for a in p]         # proximity step
+            grawa.grawa_prox_step(xs32, torch.from_numpy(g[0]).cuda(), 0.01)
+            out["cases"] += 1
             if M > 1 and cfg.n < 100000:                           # bulk-copy kernel and the host-buffer path
                 grawa.grawa_set_option("pull_variant", 2)
                 gpu_step(grawa, "lgrawa", p, g, 0.5, cfg.offsets())
