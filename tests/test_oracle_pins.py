@@ -228,6 +228,44 @@ def test_step_against_independent_numpy_statement(variant, M, sizes):
     assert np.allclose(np.stack(r["workers"]), xn, rtol=1e-12, atol=1e-14)
 
 
+@pytest.mark.parametrize("variant", ["grawa", "mgrawa", "lgrawa"])
+@pytest.mark.parametrize("sizes", [[4, 0, 9, 2, 0], [0, 0, 3, 0, 5], [0, 7], [3, 0, 0, 0, 1, 0], [2, 0, 2, 0, 2]])
+def test_empty_layers_against_independent_numpy_statement(variant, sizes):
+    """Layer tables with zero-size layers (first, last, several in a row): the element -> layer
+    lookup must skip them.  Every layer gets its own per-worker gradient scales, so the weights of
+    neighbouring layers differ by orders of magnitude and a lookup that lands one row off (the empty
+    layer's row, or the previous non-empty one) moves the centre far outside the tolerance."""
+    M = 5
+    off = np.concatenate([[0], np.cumsum(sizes)]).astype(np.int64)
+    n, K = int(off[-1]), len(sizes)
+    x = [f32(rng.normal(size=n) + 3.0 * m) for m in range(M)]
+    g = [f32(rng.normal(size=n)) for _ in range(M)]
+    for k in range(K):
+        scales = 10.0 ** np.roll(np.array([-2.0, -1.0, 0.0, 1.0, 2.0]), k)  # which worker is quiet rotates with k
+        for m in range(M):
+            g[m][off[k]:off[k + 1]] *= np.float32(scales[m])
+    r = oracle.step(x, g, 0.6, variant, off)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        S, beta, c, xn = numpy_statement(x, g, off, 0.6, variant)
+    full = np.diff(off) > 0
+    assert np.allclose(r["S"][full], S[full], rtol=1e-13) and np.all(r["S"][~full] == 0)
+    if variant == "lgrawa":
+        assert np.allclose(r["beta"][full], beta[full], rtol=1e-12)
+        b = r["beta"][full]
+        for a in range(len(b) - 1):
+            assert np.abs(b[a] - b[a + 1]).max() > 0.3   # consecutive non-empty layers have very different weights
+    else:
+        assert np.allclose(r["beta"], beta, rtol=1e-12)
+    assert np.allclose(r["center"], c, rtol=1e-12, atol=1e-14)
+    assert np.allclose(np.stack(r["workers"]), xn, rtol=1e-12, atol=1e-14)
+    # the ranged call, started at every element (so the lookup begins in front of, on and after
+    # each run of empty layers), against the numpy statement rather than the oracle's own whole call
+    for j0 in range(n):
+        cj, wj = oracle.center_pull(x, r["beta"], 0.6, off, j0, n)
+        assert np.allclose(cj, c[j0:], rtol=1e-12, atol=1e-14)
+        assert np.allclose(np.stack(wj), xn[:, j0:], rtol=1e-12, atol=1e-14)
+
+
 @pytest.mark.parametrize("variant", ["mgrawa", "lgrawa"])
 def test_equal_norms_give_the_plain_mean(variant):
     """Equal gradient norms -> uniform weights -> the centre is the arithmetic mean of the workers."""
