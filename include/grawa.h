@@ -251,6 +251,16 @@ grawa_status grawa_selftest_bounded_wait(int64_t limit_ns, grawa_stream_t stream
  * Returns -1 in the normal build, -2 on a CUDA error. */
 int64_t grawa_debug_bounds_violations(int selfcheck);
 
+/* Trace build only (the library compiled with -DGRAWA_TRACE): the sum-of-squares, finalisation and
+ * register centre+pull kernels stamp the device's nanosecond timer, one row per launch of each kind
+ * (64 rows, wrapping): {entry of the first CTA, first CTA past the dependency wait, last CTA past
+ * it, exit of the last CTA}.  Copies up to max_rows rows of 3 kinds x 4 uint64 to rows_out (HOST,
+ * may be NULL), then resets the rows and the launch counters; synchronises the device.  Call it
+ * once before the steps to be traced (reset) and once after.  All traced launches of one kind must
+ * have the same grid size.  Returns the number of rows kept (64), -1 in the normal build, -2 on a
+ * CUDA error. */
+int grawa_trace_read(uint64_t *rows_out, int max_rows);
+
 /* Tuning knobs, process wide; they change speed, never results beyond fp32 summation order
  * of the sums of squares ("sumsq_tile").  Returns GRAWA_ERR_INVALID_ARG for an unknown name
  * or a value out of range.

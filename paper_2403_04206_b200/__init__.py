@@ -29,6 +29,7 @@ from .binding import (  # noqa: F401
     grawa_step_host,
     grawa_step_typed,
     grawa_sumsq_static,
+    grawa_trace_read,
     grawa_version,
     grawa_workspace_bytes,
     library,

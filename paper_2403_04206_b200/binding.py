@@ -42,7 +42,8 @@ def library() -> ctypes.CDLL:
     if _lib is not None:
         return _lib
     import os
-    path = _build.build(debug_bounds=os.environ.get("GRAWA_DEBUG_BOUNDS", "0") == "1")
+    path = _build.build(debug_bounds=os.environ.get("GRAWA_DEBUG_BOUNDS", "0") == "1",
+                        trace=os.environ.get("GRAWA_TRACE", "0") == "1")
     lib = ctypes.CDLL(path)
     vp, i64, ci, cf = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int, ctypes.c_float
     step_args = [vp, vp, i64, ci, cf, vp, ci, vp, vp, vp]
@@ -84,6 +85,8 @@ def library() -> ctypes.CDLL:
     lib.grawa_sumsq_static.restype = ci
     lib.grawa_debug_bounds_violations.argtypes = [ci]
     lib.grawa_debug_bounds_violations.restype = i64
+    lib.grawa_trace_read.argtypes = [vp, ci]
+    lib.grawa_trace_read.restype = ci
     lib.grawa_selftest_bounded_wait.argtypes = [i64, vp]
     lib.grawa_selftest_bounded_wait.restype = ci
     lib.grawa_collect_kernel_times.argtypes = [vp, vp, vp, vp]
@@ -381,6 +384,18 @@ def grawa_selftest_bounded_wait(limit_ns: int, *, stream=None) -> None:
 def grawa_debug_bounds_violations(selfcheck: bool = False) -> int:
     """Violations counted by a bounds-checking debug build since the last call (-1 in a normal build)."""
     return int(library().grawa_debug_bounds_violations(1 if selfcheck else 0))
+
+
+def grawa_trace_read(max_rows: int = 64):
+    """Trace build (GRAWA_TRACE=1 in the environment): the rows stamped since the last call as an
+    array [rows, 3 kernels, 4 stamps] of uint64 nanoseconds, and a reset.  None in the normal build."""
+    buf = np.zeros((max_rows, 3, 4), dtype=np.uint64)
+    kept = int(library().grawa_trace_read(buf.ctypes.data, max_rows))
+    if kept == -1:
+        return None
+    if kept < 0:
+        raise GrawaError(-2, "grawa_trace_read")
+    return buf
 
 
 def grawa_clear_plans() -> None:

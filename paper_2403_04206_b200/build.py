@@ -10,6 +10,7 @@ _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "libgrawa.so")
 DEBUG_LIB_PATH = os.path.join(_HERE, "libgrawa_debug_bounds.so")
+TRACE_LIB_PATH = os.path.join(_HERE, "libgrawa_trace.so")
 SOURCES = [os.path.join(CSRC, "grawa.cu")]
 HEADERS = [os.path.join(CSRC, "kernels.cuh"), os.path.join(CSRC, "center_pull_bulk.cuh"), os.path.join(CSRC, "kernels_16bit.cuh"),
            os.path.join(_ROOT, "include", "grawa.h")]
@@ -33,18 +34,25 @@ def is_stale(path: str = LIB_PATH) -> bool:
     return any(os.path.getmtime(p) > t for p in SOURCES + HEADERS)
 
 
-def build(force: bool = False, verbose: bool = False, debug_bounds: bool = False) -> str:
+def _build_variant(path: str, define: str, force: bool) -> str:
+    if force or is_stale(path):
+        tmp = path + f".tmp{os.getpid()}"
+        cmd = [_nvcc()] + NVCC_FLAGS + [define, "-o", tmp] + SOURCES
+        res = subprocess.run(cmd, capture_output=True, text=True)
+        if res.returncode != 0:
+            raise RuntimeError("nvcc failed:\n" + " ".join(cmd) + "\n" + res.stdout + res.stderr)
+        os.replace(tmp, path)
+    return path
+
+
+def build(force: bool = False, verbose: bool = False, debug_bounds: bool = False, trace: bool = False) -> str:
     """Compile the CUDA library when missing or older than its sources; returns its path.
-    debug_bounds: the variant whose kernels check every global access against the vector length."""
+    debug_bounds: the variant whose kernels check their global accesses against the plan;
+    trace: the variant whose kernels stamp the device timer (see grawa_trace_read)."""
     if debug_bounds:
-        if force or is_stale(DEBUG_LIB_PATH):
-            tmp = DEBUG_LIB_PATH + f".tmp{os.getpid()}"
-            cmd = [_nvcc()] + NVCC_FLAGS + ["-DGRAWA_DEBUG_BOUNDS", "-o", tmp] + SOURCES
-            res = subprocess.run(cmd, capture_output=True, text=True)
-            if res.returncode != 0:
-                raise RuntimeError("nvcc failed:\n" + " ".join(cmd) + "\n" + res.stdout + res.stderr)
-            os.replace(tmp, DEBUG_LIB_PATH)
-        return DEBUG_LIB_PATH
+        return _build_variant(DEBUG_LIB_PATH, "-DGRAWA_DEBUG_BOUNDS", force)
+    if trace:
+        return _build_variant(TRACE_LIB_PATH, "-DGRAWA_TRACE", force)
     if force or is_stale():
         tmp = LIB_PATH + f".tmp{os.getpid()}"
         cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + ["-o", tmp] + SOURCES

@@ -31,6 +31,7 @@ static int64_t g_pull_variant = 0;
 static int64_t g_bulk_tile = 0;           // 0 = chosen from M so that at least three stages fit
 static int64_t g_kernel_timing = 0;
 static int64_t g_pdl = 1;
+static int64_t g_pull_preload = 1;
 static int64_t g_sumsq_ctas_per_sm = 0;   // 0 = one CTA per work item
 static int64_t g_pull_ctas_per_sm = 0;    // 0 = one CTA per work item
 static thread_local std::string t_cuda_error;
@@ -80,53 +81,38 @@ static int64_t layer_tile(int64_t layer_elems, int64_t tile, int64_t max_items)
 constexpr int64_t kMaxSumsqItemsPerLayer = 1024;
 
 // Cuts every non-empty layer at the absolute multiples of its tile that fall inside it.
-static void build_segments(const std::vector<int64_t>& off, int64_t tile, int64_t max_items, std::vector<Segment>* segs,
-                           std::vector<int>* layer_first)
+static void build_segments(const std::vector<int64_t>& off, int64_t tile, int64_t max_items, std::vector<Segment>* segs)
 {
     const int K = static_cast<int>(off.size()) - 1;
-    if (layer_first) layer_first->assign(K + 1, 0);
-    int64_t count = 0;
     for (int k = 0; k < K; ++k) {
-        if (layer_first) (*layer_first)[k] = static_cast<int>(count);
         int64_t pos = off[k];
         const int64_t end = off[k + 1];
         const int64_t t = layer_tile(end - pos, tile, max_items);
         while (pos < end) {
             const int64_t next = std::min(end, (pos / t + 1) * t);
-            if (segs) segs->push_back(Segment{pos, static_cast<int>(next - pos), k});
-            ++count;
+            segs->push_back(Segment{pos, static_cast<int>(next - pos), k});
             pos = next;
         }
     }
-    if (layer_first) (*layer_first)[K] = static_cast<int>(count);
-}
-
-static int64_t count_segments(const std::vector<int64_t>& off, int64_t tile, int64_t max_items)
-{
-    int64_t count = 0;
-    for (size_t k = 0; k + 1 < off.size(); ++k) {
-        if (off[k + 1] > off[k]) {
-            const int64_t t = layer_tile(off[k + 1] - off[k], tile, max_items);
-            count += (off[k + 1] - 1) / t - off[k] / t + 1;
-        }
-    }
-    return count;
 }
 
 // Scratch layout (all offsets 256-byte aligned).
 struct WorkspaceLayout {
-    size_t partials, S, A, beta, words, total;
+    size_t words, bins, state_end, S, A, beta, total;
 };
 
-static WorkspaceLayout workspace_layout(int64_t C1, int K, int M)
+// The first `state_end` bytes carry state from one step to the next (which copy of the digit rows
+// is clean) and must start out as zeros; the rest is overwritten before it is read.
+static WorkspaceLayout workspace_layout(int K, int M)
 {
     WorkspaceLayout w{};
     size_t p = 0;
-    w.partials = p; p = align_up(p + sizeof(double) * static_cast<size_t>(C1) * M, 256);
+    w.words = p;    p = align_up(p + 256, 256);   // ints: [0] next_buf, [1] status, [2] work counter (unsigned)
+    w.bins = p;     p = align_up(p + sizeof(unsigned long long) * 2 * static_cast<size_t>(K) * M * kRowWords, 256);
+    w.state_end = p;
     w.S = p;        p = align_up(p + sizeof(double) * static_cast<size_t>(K) * M, 256);
     w.A = p;        p = align_up(p + sizeof(double) * (static_cast<size_t>(K) + 1) * M, 256);   // K rows of terms + scores
     w.beta = p;     p = align_up(p + sizeof(float) * static_cast<size_t>(K) * M, 256);
-    w.words = p;    p = align_up(p + 256, 256);   // [1] status (int), [2] work counter (unsigned)
     w.total = p;
     return w;
 }
@@ -141,9 +127,7 @@ struct Plan {
     int C1 = 0, C2 = 0;
     Segment* d_segs1 = nullptr;      // sum-of-squares items
     Segment* d_segs2 = nullptr;      // per-layer centre+pull items
-    int* d_layer_first = nullptr;    // first sum-of-squares item of each layer, K+1 entries
-    unsigned* d_tickets = nullptr;   // the finalisation's arrival counter; zero between steps
-    int* d_layer_flag = nullptr;     // K per-layer non-finite flags
+    bool ws_dirty = false;           // a step failed half-way: the owned scratch is cleared before the next one
     void* d_ws = nullptr;            // owned scratch (used when the caller passes none)
     WorkspaceLayout ws{};
     float* d_stage = nullptr;        // owned staging for the host-buffer entry point
@@ -154,8 +138,7 @@ struct Plan {
     bool bulk = false;               // centre+pull items are cut for the bulk-copy kernel
     ~Plan()
     {
-        cudaFree(d_segs1); cudaFree(d_segs2); cudaFree(d_layer_first); cudaFree(d_ws); cudaFree(d_stage);
-        cudaFree(d_tickets); cudaFree(d_layer_flag);
+        cudaFree(d_segs1); cudaFree(d_segs2); cudaFree(d_ws); cudaFree(d_stage);
         if (d2h_stream) cudaStreamDestroy(d2h_stream);
         for (cudaEvent_t ev : events) cudaEventDestroy(ev);
     }
@@ -201,23 +184,16 @@ static grawa_status get_plan(int64_t n, int M, const std::vector<int64_t>& off, 
     p->tile2 = p->bulk ? bulk_tile_for(M) : (g_pull_tile > 0 ? g_pull_tile : pull_pass_elems(std::min(M, kMaxRegWorkers)));
     GRAWA_CUDA_TRY(cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, device));
     std::vector<Segment> s1, s2;
-    std::vector<int> first;
-    build_segments(off, p->tile1, kMaxSumsqItemsPerLayer, &s1, &first);
-    build_segments(off, p->tile2, 0, &s2, nullptr);
+    build_segments(off, p->tile1, kMaxSumsqItemsPerLayer, &s1);
+    build_segments(off, p->tile2, 0, &s2);
     if (s1.size() * static_cast<size_t>(M) > 0x7fffffffull || s2.size() > 0x7fffffffull) return GRAWA_ERR_INVALID_ARG;
     p->C1 = static_cast<int>(s1.size()); p->C2 = static_cast<int>(s2.size());
     p->h_segs2 = s2;
-    p->ws = workspace_layout(p->C1, p->K, M);
+    p->ws = workspace_layout(p->K, M);
     GRAWA_CUDA_TRY(cudaMalloc(&p->d_segs1, sizeof(Segment) * std::max<size_t>(1, s1.size())));
     GRAWA_CUDA_TRY(cudaMalloc(&p->d_segs2, sizeof(Segment) * std::max<size_t>(1, s2.size())));
-    GRAWA_CUDA_TRY(cudaMalloc(&p->d_layer_first, sizeof(int) * first.size()));
     GRAWA_CUDA_TRY(cudaMemcpy(p->d_segs1, s1.data(), sizeof(Segment) * s1.size(), cudaMemcpyHostToDevice));
     GRAWA_CUDA_TRY(cudaMemcpy(p->d_segs2, s2.data(), sizeof(Segment) * s2.size(), cudaMemcpyHostToDevice));
-    GRAWA_CUDA_TRY(cudaMemcpy(p->d_layer_first, first.data(), sizeof(int) * first.size(), cudaMemcpyHostToDevice));
-    GRAWA_CUDA_TRY(cudaMalloc(&p->d_tickets, sizeof(unsigned)));
-    GRAWA_CUDA_TRY(cudaMemset(p->d_tickets, 0, sizeof(unsigned)));
-    GRAWA_CUDA_TRY(cudaMalloc(&p->d_layer_flag, sizeof(int) * static_cast<size_t>(p->K)));
-    GRAWA_CUDA_TRY(cudaMemset(p->d_layer_flag, 0, sizeof(int) * static_cast<size_t>(p->K)));
     *out = p.get();
     g_plans[key] = std::move(p);
     return GRAWA_OK;
@@ -332,13 +308,13 @@ struct CenterPullBulkDispatch<1> {
 template <int M>
 static cudaError_t launch_center_pull(bool per_layer, int grid, int item_begin, int item_end, cudaStream_t stream, bool pdl,
                                       const MutPtrs& x, float* center, const float* beta, const Segment* segs, long long n, int tile,
-                                      float pull)
+                                      float pull, int preload)
 {
     if (per_layer)
         return launch_kernel(center_pull_kernel<M, true>, grid, kThreads, stream, pdl, x, center, beta, segs, item_begin, item_end, n,
-                             tile, pull, 1);
+                             tile, pull, 1, preload);
     return launch_kernel(center_pull_kernel<M, false>, grid, kThreads, stream, pdl, x, center, beta, segs, item_begin, item_end, n, tile,
-                         pull, 1);
+                         pull, 1, preload);
 }
 
 template <int M>
@@ -407,6 +383,7 @@ struct StepContext {
     TimedStep* ts = nullptr;
     int pull_items = 0;            // centre+pull work items of the whole vector
     int dtype = 0;                 // storage of params / grads / centre: 0 fp32, 1 bfloat16, 2 half
+    bool preload = false;          // centre+pull may load parameters before its dependency wait (see the kernel)
 };
 
 static grawa_status make_context(int variant, float* const* params, const float* const* grads, int64_t n, int M, float pull,
@@ -418,8 +395,18 @@ static grawa_status make_context(int variant, float* const* params, const float*
         if ((reinterpret_cast<uintptr_t>(ws) & 255u) || opt->workspace_bytes < plan->ws.total) return GRAWA_ERR_WORKSPACE;
     } else {
         if (opt && opt->workspace_bytes != 0) return GRAWA_ERR_WORKSPACE;
-        if (!plan->d_ws) GRAWA_CUDA_TRY(cudaMalloc(&plan->d_ws, plan->ws.total));
+        if (!plan->d_ws) {
+            GRAWA_CUDA_TRY(cudaMalloc(&plan->d_ws, plan->ws.total));
+            plan->ws_dirty = true;
+        }
         ws = static_cast<char*>(plan->d_ws);
+    }
+    // The state part of the scratch must be zero when a step starts from scratch: always for a
+    // caller's buffer (its contents are the caller's business between calls), and for the plan's own
+    // buffer when it is new or a step was abandoned half-way.
+    if (ws != plan->d_ws || plan->ws_dirty) {
+        GRAWA_CUDA_TRY(cudaMemsetAsync(ws, 0, plan->ws.state_end, stream));
+        if (ws == plan->d_ws) plan->ws_dirty = false;
     }
     ctx->plan = plan; ctx->variant = variant; ctx->M = M; ctx->n = n; ctx->pull = pull; ctx->stream = stream;
     ctx->center = center_out;
@@ -434,15 +421,14 @@ static grawa_status make_context(int variant, float* const* params, const float*
         ctx->vec_x = ctx->vec_x && aligned16(params[m]);
     }
     StepScratch& sc = ctx->sc;
-    sc.segs = plan->d_segs1; sc.layer_seg_first = plan->d_layer_first;
+    sc.segs = plan->d_segs1;
     sc.C = plan->C1; sc.K = K; sc.M = M; sc.variant = variant; sc.n = n;
-    sc.partials = reinterpret_cast<double*>(ws + plan->ws.partials);
+    sc.bins = reinterpret_cast<unsigned long long*>(ws + plan->ws.bins);
+    sc.next_buf = reinterpret_cast<int*>(ws + plan->ws.words);
     sc.S = reinterpret_cast<double*>(ws + plan->ws.S);
     sc.A = reinterpret_cast<double*>(ws + plan->ws.A);
     sc.beta = reinterpret_cast<float*>(ws + plan->ws.beta);
-    sc.layer_flag = plan->d_layer_flag;
-    sc.global_ticket = plan->d_tickets;
-    sc.global_target = static_cast<unsigned>(K);
+    sc.status_copy = nullptr;
     sc.status = ctx->status; sc.work_counter = ctx->counter;
     sc.weights_out = opt ? opt->weights_out : nullptr;
     sc.scores_out = opt ? opt->scores_out : nullptr;
@@ -456,13 +442,33 @@ static grawa_status make_context(int variant, float* const* params, const float*
     return GRAWA_OK;
 }
 
+// Steps 2-3.  LGRAWA from the sums of a sum-of-squares kernel: one warp per layer in as many CTAs
+// as that takes.  Everything else (one weight per worker, or given scores): one CTA.
+static cudaError_t launch_finalize(const StepContext& c)
+{
+    const Plan* plan = c.plan;
+    const bool layered = c.variant == kLgrawa && c.sc.given == nullptr;
+    const int warps = kFinThreadsLayered / 32;
+    const int grid = layered ? std::max(1, std::min((plan->K + warps - 1) / warps, 4 * plan->sm_count)) : 1;
+    const int block = layered ? kFinThreadsLayered : kFinThreadsFlat;
+    return launch_kernel(finalize_kernel, grid, block, c.stream, c.pdl, c.sc);
+}
+
 // Steps 1-3: sums of squares, scores, weights (two launches).
+static grawa_status enqueue_weights_launches(StepContext& c);
 static grawa_status enqueue_weights(StepContext& c)
+{
+    const grawa_status st = enqueue_weights_launches(c);
+    if (st != GRAWA_OK) c.plan->ws_dirty = true;       // the two copies of the digit rows may be out of step
+    return st;
+}
+
+static grawa_status enqueue_weights_launches(StepContext& c)
 {
     Plan* plan = c.plan;
     if (c.sc.given != nullptr) {                     // scores are given: no pass over gradients
         if (c.ts) GRAWA_CUDA_TRY(cudaEventRecord(c.ts->e[1], c.stream));
-        GRAWA_CUDA_TRY(launch_kernel(finalize_kernel, plan->K, kThreads, c.stream, c.pdl, c.sc));
+        GRAWA_CUDA_TRY(launch_finalize(c));
         if (c.ts) GRAWA_CUDA_TRY(cudaEventRecord(c.ts->e[2], c.stream));
         return GRAWA_OK;
     }
@@ -477,7 +483,7 @@ static grawa_status enqueue_weights(StepContext& c)
     else
         GRAWA_CUDA_TRY(launch_kernel(sumsq_kernel<8>, grid1, kThreads, c.stream, c.pdl, c.gp, c.sc, items1, vg));
     if (c.ts) GRAWA_CUDA_TRY(cudaEventRecord(c.ts->e[1], c.stream));
-    GRAWA_CUDA_TRY(launch_kernel(finalize_kernel, plan->K, kThreads, c.stream, c.pdl, c.sc));
+    GRAWA_CUDA_TRY(launch_finalize(c));
     if (c.ts) GRAWA_CUDA_TRY(cudaEventRecord(c.ts->e[2], c.stream));
     return GRAWA_OK;
 }
@@ -531,7 +537,8 @@ static grawa_status enqueue_center_pull(StepContext& c, int item_begin, int item
         const int grid2 = g_pull_ctas_per_sm > 0
                               ? static_cast<int>(std::min<int64_t>(grid, g_pull_ctas_per_sm * plan->sm_count)) : grid;
         GRAWA_CUDA_TRY(CenterPullDispatch<kMaxRegWorkers>::run(M, per_layer, grid2, item_begin, item_end, c.stream, c.pdl, c.xp,
-                                                               c.center, beta, plan->d_segs2, c.n, tile, c.pull));
+                                                               c.center, beta, plan->d_segs2, c.n, tile, c.pull,
+                                                               (c.preload && g_pull_preload) ? 1 : 0));
     } else {
         GRAWA_CUDA_TRY(launch_kernel(center_pull_generic_kernel, grid, kThreads, c.stream, c.pdl, c.xp, c.center, beta, plan->d_segs2,
                                      per_layer ? 1 : 0, item_begin, c.n, tile, c.pull, M));
@@ -582,6 +589,7 @@ static grawa_status enqueue_step(int variant, float* const* params, const float*
                 GRAWA_CUDA_TRY(launch_kernel(copy_kernel, grid, kThreads, stream, c.pdl, params[0], center_out, n, v ? 1 : 0));
         }
     } else {
+        c.preload = true;          // the kernels in front of it on the stream are this step's own
         st = enqueue_center_pull(c, 0, c.pull_items);
         if (st != GRAWA_OK) return st;
     }
@@ -712,7 +720,7 @@ size_t grawa_workspace_bytes(int64_t n, int M, const int64_t* layer_offsets, int
         off.assign({0, n});
     }
     std::lock_guard<std::mutex> lock(g_mutex);
-    return workspace_layout(count_segments(off, g_sumsq_tile, kMaxSumsqItemsPerLayer), static_cast<int>(off.size()) - 1, M).total;
+    return workspace_layout(static_cast<int>(off.size()) - 1, M).total;
 }
 
 grawa_status grawa_mgrawa_step(float* const* params, const float* const* grads, int64_t n, int M, float pull,
@@ -1024,6 +1032,28 @@ int64_t grawa_debug_bounds_violations(int selfcheck)
 #endif
 }
 
+int grawa_trace_read(uint64_t* rows_out, int max_rows)
+{
+#ifdef GRAWA_TRACE
+    if (cudaDeviceSynchronize() != cudaSuccess) return -2;
+    static TraceRow host[kTraceRows][kTraceKinds];
+    unsigned arrivals[kTraceKinds] = {};
+    if (rows_out != nullptr && max_rows > 0) {
+        if (cudaMemcpyFromSymbol(host, g_trace, sizeof host) != cudaSuccess) return -2;
+        const int rows = std::min(max_rows, kTraceRows);
+        std::memcpy(rows_out, host, sizeof(TraceRow) * kTraceKinds * static_cast<size_t>(rows));
+    }
+    for (auto& row : host)
+        for (auto& r : row) r = TraceRow{~0ull, ~0ull, 0ull, 0ull};
+    if (cudaMemcpyToSymbol(g_trace, host, sizeof host) != cudaSuccess) return -2;
+    if (cudaMemcpyToSymbol(g_trace_arrivals, arrivals, sizeof arrivals) != cudaSuccess) return -2;
+    return kTraceRows;
+#else
+    (void)rows_out; (void)max_rows;
+    return -1;
+#endif
+}
+
 static void clear_plans_locked()
 {
     cudaDeviceSynchronize();
@@ -1066,6 +1096,11 @@ grawa_status grawa_set_option(const char* name, int64_t value)
         g_pdl = value;
         return GRAWA_OK;
     }
+    if (std::strcmp(name, "pull_preload") == 0) {
+        if (value < 0 || value > 1) return GRAWA_ERR_INVALID_ARG;
+        g_pull_preload = value;
+        return GRAWA_OK;
+    }
     if (std::strcmp(name, "sumsq_ctas_per_sm") == 0 || std::strcmp(name, "pull_ctas_per_sm") == 0) {
         if (value < 0 || value > 32) return GRAWA_ERR_INVALID_ARG;
         (name[0] == 's' ? g_sumsq_ctas_per_sm : g_pull_ctas_per_sm) = value;
@@ -1084,6 +1119,7 @@ int64_t grawa_get_option(const char* name)
     if (std::strcmp(name, "bulk_tile") == 0) return g_bulk_tile;
     if (std::strcmp(name, "kernel_timing") == 0) return g_kernel_timing;
     if (std::strcmp(name, "dependent_launch") == 0) return g_pdl;
+    if (std::strcmp(name, "pull_preload") == 0) return g_pull_preload;
     if (std::strcmp(name, "sumsq_ctas_per_sm") == 0) return g_sumsq_ctas_per_sm;
     if (std::strcmp(name, "pull_ctas_per_sm") == 0) return g_pull_ctas_per_sm;
     return -1;

@@ -10,7 +10,6 @@ namespace grawa {
 constexpr int kMaxWorkers = 64;
 constexpr int kThreads = 256;          // threads per CTA of the streaming kernels
 constexpr int kFinalizeThreads = 256;
-constexpr int kStageDoubles = 1024;    // shared-memory staging of the finalisation (8 KB)
 constexpr int kMaxRegWorkers = 16;     // largest M the register-resident centre+pull kernel is built for
 
 enum Variant { kGrawa = 0, kMgrawa = 1, kLgrawa = 2 };
@@ -37,6 +36,54 @@ __device__ __forceinline__ void grid_dependency_sync()
     asm volatile("griddepcontrol.wait;" ::: "memory");
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
+
+__device__ __forceinline__ unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Trace build (-DGRAWA_TRACE): the three kernels of a step stamp the device's nanosecond timer when
+// their first CTA enters, when the first and the last CTA get past the dependency wait, and when
+// the last CTA leaves, one row per launch (see grawa_trace_read).  Nothing is skipped or reordered;
+// thread 0 of every CTA issues one counting atomic and four min/max reductions.  In the normal
+// build the tracer is an empty object.
+#ifdef GRAWA_TRACE
+struct TraceRow { unsigned long long first_entry, first_go, last_go, last_exit; };
+constexpr int kTraceKinds = 3;         // 0 sum of squares, 1 finalisation, 2 centre+pull
+constexpr int kTraceRows = 64;         // launches of one kind wrap around after this many
+__device__ TraceRow g_trace[kTraceRows][kTraceKinds];
+__device__ unsigned g_trace_arrivals[kTraceKinds];
+struct KernelTrace {
+    unsigned long long t_entry = 0, t_go = 0;
+    unsigned arrival = 0;
+    int kind;
+    __device__ __forceinline__ explicit KernelTrace(int k) : kind(k)
+    {
+        if (threadIdx.x == 0) {
+            t_entry = global_timer_ns();
+            arrival = atomicAdd(&g_trace_arrivals[kind], 1u);
+        }
+    }
+    __device__ __forceinline__ void go() { if (threadIdx.x == 0) t_go = global_timer_ns(); }
+    __device__ __forceinline__ void done()
+    {
+        if (threadIdx.x != 0) return;
+        TraceRow& r = g_trace[(arrival / gridDim.x) % kTraceRows][kind];
+        atomicMin(&r.first_entry, t_entry);
+        atomicMin(&r.first_go, t_go);
+        atomicMax(&r.last_go, t_go);
+        atomicMax(&r.last_exit, global_timer_ns());
+    }
+};
+#else
+struct KernelTrace {
+    __device__ __forceinline__ explicit KernelTrace(int) {}
+    __device__ __forceinline__ void go() {}
+    __device__ __forceinline__ void done() {}
+};
+#endif
 
 // Debug build (-DGRAWA_DEBUG_BOUNDS): every global access of the streaming kernels is first checked
 // against the vector's length; a violation is counted and the access skipped (nothing traps).
@@ -103,20 +150,89 @@ __device__ __forceinline__ double block_sum_fixed_order(double v)
     return total;
 }
 
+// ---------------------------------------------------------------------------------------------
+// Exact accumulation of the sums of squares.  S[k][m] of one step is kept as a fixed-point integer
+// of kBinWords 32-bit digits, each digit in its own 64-bit word (32 bits of head-room for carries, so
+// a word absorbs 2^32 additions before it could overflow), least significant bit 2^-149, the
+// smallest positive fp32 value.  A CTA adds its fp64 partial sum with up to three integer atomic
+// adds that return nothing.  Integer addition is associative: the total does not depend on the
+// order in which the CTAs arrive, so the result is bitwise reproducible without a second reduction
+// pass over stored partial sums.  Digits below 2^-149 (they can only come from the fp64 squares of
+// a layer's few unaligned edge elements) are dropped; a partial sum that is not finite or is
+// >= 2^170 sets the row's marker word instead and the row reads back as +infinity.
+// ---------------------------------------------------------------------------------------------
+constexpr int kBinWords = 10;          // digits: bit positions 0..319, values below 2^171
+constexpr int kRowWords = 11;          // words per (layer, worker) row: the digits and the marker
+constexpr int kBinLsbExp = -149;
+constexpr int kBinMaxExp = 170;        // partial sums must be < 2^170
+
+// Layout: digit-major, [copy][kRowWords][K][M] words, so that the threads of a warp that read the same
+// digit of neighbouring (layer, worker) rows touch neighbouring words.  `row` points at digit 0 of
+// a (layer, worker) pair and `stride` = K * M is the distance between its digits.
+__device__ __forceinline__ void bins_add(unsigned long long* __restrict__ row, size_t stride, double v)
+{
+    if (!(v < 1.4965776766268446e51)) {                 // 2^170; also catches NaN
+        atomicOr(row + kBinWords * stride, 1ull);
+        return;
+    }
+    const unsigned long long bits = static_cast<unsigned long long>(__double_as_longlong(v));
+    const int ex = static_cast<int>((bits >> 52) & 0x7ffu);
+    if (ex == 0) return;                                // zero, or an fp64 subnormal (far below 2^-149)
+    unsigned long long man = (bits & 0x000fffffffffffffull) | 0x0010000000000000ull;    // v = man * 2^(ex - 1075)
+    int sh = ex - 1075 - kBinLsbExp;                    // bit position of man's least significant bit
+    if (sh < 0) {
+        if (sh <= -53) return;
+        man >>= -sh;
+        sh = 0;
+    }
+    const int b0 = sh >> 5, r = sh & 31;
+    const unsigned long long lo = man << r;             // bits 0..63 of man * 2^r
+    const unsigned long long hi = r ? (man >> (64 - r)) : 0ull;    // bits 64..84
+    const unsigned long long d0 = lo & 0xffffffffull, d1 = lo >> 32;
+    if (d0) atomicAdd(row + b0 * stride, d0);
+    if (d1) atomicAdd(row + (b0 + 1) * stride, d1);
+    if (hi) atomicAdd(row + (b0 + 2) * stride, hi);     // b0 + 2 <= 9 because v < 2^170
+}
+
+// The value of a row: digits added from the most significant one down (a fixed order).  The digit
+// rows exist twice (see StepScratch) and the copy not in use is all zeros, so the reader adds the
+// two copies digit by digit instead of first finding out which one holds the sums: all loads are
+// independent of one another.
+__device__ __forceinline__ double bins_value(const unsigned long long* __restrict__ row, size_t stride)
+{
+    const size_t copy_words = stride * kRowWords;
+    unsigned long long w[kBinWords + 1];
+#pragma unroll
+    for (int b = 0; b <= kBinWords; ++b) w[b] = __ldcg(row + b * stride) + __ldcg(row + copy_words + b * stride);
+    if (w[kBinWords]) return __longlong_as_double(0x7ff0000000000000ll);      // +infinity
+    double s = 0.0;
+#pragma unroll
+    for (int b = kBinWords - 1; b >= 0; --b) {
+        const double scale = __longlong_as_double(static_cast<long long>(1023 + 32 * b + kBinLsbExp) << 52);   // 2^(32 b - 149)
+        s += static_cast<double>(w[b]) * scale;
+    }
+    return s;
+}
+
 // Everything the sum-of-squares and finalisation code needs to know about one step.
+//
+// The digit rows exist twice.  A sum-of-squares kernel adds into the copy named by *next_buf and
+// clears the other copy for the step after it; the finalisation that consumes the sums (it adds the
+// two copies, one of which is zero) then points the word at the other copy.  The word is written
+// only while none of its readers can be running (the kernels of a step follow one another on the
+// stream), and it lives in device memory, so a replayed CUDA graph alternates between the copies
+// like eager calls do.
 struct StepScratch {
     const Segment* segs;           // sum-of-squares work items of one worker, C of them
-    const int* layer_seg_first;    // first item of each layer, K+1 entries
     int C, K, M, variant;
     long long n;                   // elements per worker (bounds checks of the debug build)
-    double* partials;              // [M][C]
+    unsigned long long* bins;      // [2][kRowWords][K][M]
+    int* next_buf;                 // copy the next sum-of-squares kernel adds into
     double* S;                     // [K][M]
     double* A;                     // [K+1][M]: per-layer terms, then the per-worker scores in row K
     float* beta;                   // [K][M] (LGRAWA) or [M]
-    int* layer_flag;               // [K] non-finite flag of each layer's group (LGRAWA)
-    unsigned* global_ticket;       // zero between steps
-    unsigned global_target;        // arrivals that complete the step's finalisation
-    int* status;                   // written (not or-ed) when the finalisation completes
+    int* status;                   // rewritten by every finalisation
+    int* status_copy;              // optional caller-owned copy of the status word, else NULL
     unsigned* work_counter;        // cleared for the bulk-copy centre+pull kernel
     const double* given;           // [given_parts][K][M] given per-layer norms or sums of squares, else NULL
     int given_parts;               // parts (e.g. ranks) whose sums are added in part order; 1 for norms
@@ -126,185 +242,204 @@ struct StepScratch {
     double* sumsq_out;
 };
 
-// Step 3 for one group of M scores (Eq. 2 / 4 / 7) with the zero-score limit and the non-finite
-// fallback, computed by the whole CTA: thread m < M passes its score `a` and gets beta_m back.
-// The reciprocals are taken in parallel and added by one thread in worker order, so the value is
-// the one a sequential loop over m = 0..M-1 gives.  Every thread of the CTA must call it.
-struct WeightsSmem {
-    double r[kMaxWorkers];
-    double z;
-};
+__device__ __forceinline__ size_t bins_copy_words(const StepScratch& sc) { return static_cast<size_t>(sc.K) * sc.M * kRowWords; }
 
-__device__ __forceinline__ float weights_parallel(double a, int M, WeightsSmem& sm, int& flagged)
+// End of a sum-of-squares CTA's work: clear this CTA's share of the other copy of the digit rows.
+__device__ __forceinline__ void bins_turnover(const StepScratch& sc, int buf)
 {
-    const int tid = threadIdx.x;
-    const bool active = tid < M;
-    const bool fin = active && isfinite(a);
-    const bool zero = fin && a == 0.0;
-    const int finite = __syncthreads_count(fin);
-    const int zeros = __syncthreads_count(zero);
-    if (active) sm.r[tid] = (fin && !zero) ? 1.0 / a : 0.0;
-    __syncthreads();
-    if (tid == 0) {
-        double z = 0.0;
-        for (int m = 0; m < M; ++m) z += sm.r[m];     // adding the 0.0 of a skipped worker is exact
-        sm.z = z;
+    const size_t words = bins_copy_words(sc);
+    unsigned long long* other = sc.bins + static_cast<size_t>(buf ^ 1) * words;
+    for (size_t i = static_cast<size_t>(blockIdx.x) * blockDim.x + threadIdx.x; i < words; i += static_cast<size_t>(gridDim.x) * blockDim.x)
+        other[i] = 0ull;
+    if (blockIdx.x == 0 && threadIdx.x == 0) {
+        *sc.status = 0;                  // the finalisation that follows only adds flags to it
+        if (sc.status_copy) *sc.status_copy = 0;
     }
-    __syncthreads();
+}
+
+// Step 3 for one group of M <= 64 scores (Eq. 2 / 4 / 7) with the zero-score limit and the
+// non-finite fallback, by one full warp: lane l passes the scores of workers l and l + 32 and gets
+// their weights back.  The reciprocals are taken in parallel and added in worker order by every
+// lane (shuffles), so the normaliser is the value a sequential loop over m = 0..M-1 gives.
+__device__ __forceinline__ void weights_warp(double a0, double a1, int M, float& w0, float& w1, int& flagged)
+{
+    const int lane = threadIdx.x & 31;
+    const bool act0 = lane < M, act1 = lane + 32 < M;
+    const bool fin0 = act0 && isfinite(a0), fin1 = act1 && isfinite(a1);
+    const bool zero0 = fin0 && a0 == 0.0, zero1 = fin1 && a1 == 0.0;
+    const int finite = __popc(__ballot_sync(0xffffffffu, fin0)) + __popc(__ballot_sync(0xffffffffu, fin1));
+    const int zeros = __popc(__ballot_sync(0xffffffffu, zero0)) + __popc(__ballot_sync(0xffffffffu, zero1));
+    const double r0 = (fin0 && !zero0) ? 1.0 / a0 : 0.0;      // adding the 0.0 of a skipped worker is exact
+    const double r1 = (fin1 && !zero1) ? 1.0 / a1 : 0.0;
+    double z = 0.0;
+    for (int m = 0; m < M && m < 32; ++m) z += __shfl_sync(0xffffffffu, r0, m);
+    for (int m = 32; m < M; ++m) z += __shfl_sync(0xffffffffu, r1, m - 32);
     flagged = finite < M;
-    double w = 0.0;
-    if (active) {
-        if (finite == 0) w = 1.0 / M;
-        else if (zeros > 0) w = zero ? 1.0 / zeros : 0.0;
-        else w = fin ? sm.r[tid] / sm.z : 0.0;
-    }
-    return static_cast<float>(w);
-}
-
-struct FinalizeSmem {
-    double layer_sum[kMaxWorkers];
-    WeightsSmem w;
-    double stage[kStageDoubles];
-    int flag;
-};
-
-// Steps 1b-3 for one non-empty layer, by a whole CTA of kThreads threads.  Warp w adds the partials
-// of workers w, w+8, ... of layer k in a fixed order into S[k][m]; the layer's terms sqrt(S) (S
-// itself for the flat norm) go to row k of A; LGRAWA turns them into the layer's weights (Eq. 7).
-// With `given` set no partials are read: either the given norm of (layer, worker) takes the place
-// of sqrt(S) (the running estimates of the Local variants), or S is the sum, in part order, of
-// given partial sums of squares (element-range shards of the vector on several GPUs).
-__device__ __forceinline__ void finalize_layer(const StepScratch& sc, int k, FinalizeSmem& sm)
-{
-    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int M = sc.M;
-    if (sc.given == nullptr) {
-        const int s0 = sc.layer_seg_first[k], s1 = sc.layer_seg_first[k + 1];
-        for (int m = warp; m < M; m += kThreads / 32) {
-            const double* row = sc.partials + static_cast<size_t>(m) * sc.C;
-            // eight independent running sums per lane keep eight loads in flight; the order in which
-            // they are combined is fixed, so the sum is the same on every run
-            double part[8] = {0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0, 0.0};
-            int s = s0 + lane;
-            for (; s + 7 * 32 < s1; s += 8 * 32) {
-#pragma unroll
-                for (int u = 0; u < 8; ++u) part[u] += __ldcg(row + s + u * 32);
-            }
-            for (int u = 0; s < s1; s += 32, ++u) part[u] += __ldcg(row + s);
-            double acc = ((part[0] + part[1]) + (part[2] + part[3])) + ((part[4] + part[5]) + (part[6] + part[7]));
-#pragma unroll
-            for (int d = 16; d > 0; d >>= 1) acc += __shfl_down_sync(0xffffffffu, acc, d);
-            if (lane == 0) sm.layer_sum[m] = acc;
-        }
-    }
-    __syncthreads();
-    double term = 0.0;
-    const size_t idx = static_cast<size_t>(k) * M + tid;
-    if (tid < M) {
-        double s;
-        if (sc.given == nullptr) {
-            s = sm.layer_sum[tid];
-            term = (sc.variant == kGrawa) ? s : sqrt(s);
-        } else if (sc.given_sums) {                // sums of squares of the parts, added in part order
-            s = 0.0;
-            for (int r = 0; r < sc.given_parts; ++r) s += sc.given[static_cast<size_t>(r) * sc.K * M + idx];
-            term = (sc.variant == kGrawa) ? s : sqrt(s);
-        } else {                                   // the caller's norm estimate stands in for sqrt(S)
-            const double a = sc.given[idx];
-            s = a * a;
-            term = (sc.variant == kGrawa) ? s : a;
-        }
-        sc.S[idx] = s;
-        if (sc.sumsq_out) sc.sumsq_out[idx] = s;
-        sc.A[idx] = term;
-    }
-    if (sc.variant == kLgrawa) {
-        int flagged = 0;
-        const float w = weights_parallel(term, M, sm.w, flagged);
-        if (tid < M) {
-            if (sc.scores_out) sc.scores_out[idx] = term;
-            sc.beta[idx] = w;
-            if (sc.weights_out) sc.weights_out[idx] = w;
-        }
-        if (tid == 0) sc.layer_flag[k] = flagged;
-    }
-}
-
-// Called by a whole CTA after its part of the finalisation.  The CTA that makes the count reach
-// `global_target` finishes the step: rows of empty layers, MGRAWA / GRAWA scores (the K rows of A
-// added per worker in layer order, Eq. 3 / Eq. 2) and weights (Eq. 4), the status word, and the
-// reset of the counters for the next step.  No CTA waits for another.
-__device__ __forceinline__ void finalize_arrive(const StepScratch& sc, FinalizeSmem& sm)
-{
-    const int tid = threadIdx.x;
-    const int M = sc.M, K = sc.K;
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        const bool last = atomicAdd(sc.global_ticket, 1u) == sc.global_target - 1u;
-        if (last) *sc.global_ticket = 0u;
-        sm.flag = last;
-    }
-    __syncthreads();
-    if (!sm.flag) return;
-    __threadfence();
-
-    // empty layers: zero sums and terms, uniform weights (they are never applied).  With given
-    // norms or sums every layer has been processed, whether it has local elements or not.
-    const bool all_layers = sc.given != nullptr;
-    for (int k = tid; k < K; k += kThreads) {
-        if (all_layers || sc.layer_seg_first[k] != sc.layer_seg_first[k + 1]) continue;
-        for (int m = 0; m < M; ++m) {
-            const size_t idx = static_cast<size_t>(k) * M + m;
-            sc.S[idx] = 0.0;
-            sc.A[idx] = 0.0;
-            if (sc.sumsq_out) sc.sumsq_out[idx] = 0.0;
-            if (sc.variant == kLgrawa) {
-                const float u = static_cast<float>(1.0 / M);
-                sc.beta[idx] = u;
-                if (sc.weights_out) sc.weights_out[idx] = u;
-                if (sc.scores_out) sc.scores_out[idx] = 0.0;
-            }
-        }
-    }
-    int flagged = 0;
-    if (sc.variant == kLgrawa) {
-        int f = 0;
-        for (int k = tid; k < K; k += kThreads)
-            if (all_layers || sc.layer_seg_first[k] != sc.layer_seg_first[k + 1]) f |= __ldcg(sc.layer_flag + k);
-        flagged = __syncthreads_or(f);
+    double v0 = 0.0, v1 = 0.0;
+    if (finite == 0) {
+        v0 = act0 ? 1.0 / M : 0.0;
+        v1 = act1 ? 1.0 / M : 0.0;
+    } else if (zeros > 0) {
+        v0 = zero0 ? 1.0 / zeros : 0.0;
+        v1 = zero1 ? 1.0 / zeros : 0.0;
     } else {
-        // Rows of A are staged through shared memory in blocks (parallel loads); thread m then adds
-        // its column in layer order.  Rows of empty layers count as 0.
-        const int rows_per_block = kStageDoubles / M;
-        double a = 0.0;
-        for (int k0 = 0; k0 < K; k0 += rows_per_block) {
-            const int rows = min(rows_per_block, K - k0);
-            for (int i = tid; i < rows * M; i += kThreads) {
-                const int k = k0 + i / M;
-                const bool empty = !all_layers && sc.layer_seg_first[k] == sc.layer_seg_first[k + 1];
-                sm.stage[i] = empty ? 0.0 : __ldcg(sc.A + static_cast<size_t>(k0) * M + i);
+        v0 = fin0 ? r0 / z : 0.0;
+        v1 = fin1 ? r1 / z : 0.0;
+    }
+    w0 = static_cast<float>(v0);
+    w1 = static_cast<float>(v1);
+}
+
+// S[k][m] of one row from whichever source the step has: the digit rows of the sum-of-squares
+// kernel, given partial sums of squares added in part order (element-range shards on several GPUs),
+// or a given norm estimate (the running estimates of the Local variants).
+__device__ __forceinline__ double row_sumsq(const StepScratch& sc, const unsigned long long* __restrict__ bins, size_t idx)
+{
+    if (sc.given == nullptr) return bins_value(bins + idx, static_cast<size_t>(sc.K) * sc.M);
+    if (sc.given_sums) {
+        double s = 0.0;
+        const size_t stride = static_cast<size_t>(sc.K) * sc.M;
+#pragma unroll 4
+        for (int p = 0; p < sc.given_parts; ++p) s += __ldcg(sc.given + p * stride + idx);
+        return s;
+    }
+    const double a = __ldcg(sc.given + idx);
+    return a * a;
+}
+
+// The row's term: its norm (the given estimate itself where there is one), or S for the flat norm.
+__device__ __forceinline__ double row_term(const StepScratch& sc, size_t idx, double s)
+{
+    if (sc.variant == kGrawa) return s;
+    if (sc.given != nullptr && !sc.given_sums) return __ldcg(sc.given + idx);
+    return sqrt(s);
+}
+
+__device__ __forceinline__ void store_row(const StepScratch& sc, size_t idx, double s, double term)
+{
+    sc.S[idx] = s;
+    sc.A[idx] = term;
+    if (sc.sumsq_out) sc.sumsq_out[idx] = s;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Steps 2-3: S -> scores -> weights.
+// LGRAWA: one warp per layer, any number of CTAs, no CTA depends on another (Eq. 5-7).
+// MGRAWA / GRAWA: one CTA; thread (p, m) adds worker m's terms of a contiguous run of layers in
+// layer order, thread m adds the runs in order (Eq. 3 / Eq. 2), one warp normalises (Eq. 4).
+// Every sum has a fixed order.  The status word is rewritten by every launch.
+// ---------------------------------------------------------------------------------------------
+constexpr int kFinThreadsLayered = 256;     // LGRAWA: 8 layers per CTA
+constexpr int kFinThreadsFlat = 1024;       // MGRAWA / GRAWA: the one CTA
+
+__global__ void __launch_bounds__(kFinThreadsFlat, 1)
+finalize_kernel(StepScratch sc)
+{
+    __shared__ double part_sm[kFinThreadsFlat];
+    __shared__ double score_sm[kMaxWorkers];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int M = sc.M, K = sc.K;
+    KernelTrace trace(1);
+    grid_dependency_sync();
+    trace.go();
+
+    const unsigned long long* bins = sc.bins;
+    if (sc.given == nullptr && blockIdx.x == 0 && tid == 0) *sc.next_buf = __ldcg(sc.next_buf) ^ 1;
+    if (blockIdx.x == 0 && tid == 0) *sc.work_counter = 0u;
+
+    if (sc.variant == kLgrawa) {
+        int any_flag = 0;
+        const int warps = blockDim.x >> 5;
+        for (int k = blockIdx.x * warps + warp; k < K; k += gridDim.x * warps) {
+            const size_t base = static_cast<size_t>(k) * M;
+            double a0 = 0.0, a1 = 0.0;
+            if (lane < M) {
+                const double s = row_sumsq(sc, bins, base + lane);
+                a0 = row_term(sc, base + lane, s);
+                store_row(sc, base + lane, s, a0);
             }
-            __syncthreads();
-            if (tid < M)
-                for (int r = 0; r < rows; ++r) a += sm.stage[r * M + tid];
-            __syncthreads();
+            if (lane + 32 < M) {
+                const double s = row_sumsq(sc, bins, base + lane + 32);
+                a1 = row_term(sc, base + lane + 32, s);
+                store_row(sc, base + lane + 32, s, a1);
+            }
+            float w0, w1;
+            int flagged;
+            weights_warp(a0, a1, M, w0, w1, flagged);
+            any_flag |= flagged;
+            if (lane < M) {
+                sc.beta[base + lane] = w0;
+                if (sc.weights_out) sc.weights_out[base + lane] = w0;
+                if (sc.scores_out) sc.scores_out[base + lane] = a0;
+            }
+            if (lane + 32 < M) {
+                sc.beta[base + lane + 32] = w1;
+                if (sc.weights_out) sc.weights_out[base + lane + 32] = w1;
+                if (sc.scores_out) sc.scores_out[base + lane + 32] = a1;
+            }
         }
-        if (tid < M) {
-            if (sc.variant == kGrawa) a = sqrt(a);
-            sc.A[static_cast<size_t>(K) * M + tid] = a;
-            if (sc.scores_out) sc.scores_out[tid] = a;
+        // the status word: a launch of one CTA (always the case with given scores, where no
+        // sum-of-squares kernel has cleared the word) writes it; several CTAs only add their flags
+        const int cta_flag = __syncthreads_or(any_flag);
+        if (tid == 0) {
+            if (gridDim.x == 1) {
+                *sc.status = cta_flag ? kStatusNonFinite : 0;
+                if (sc.status_copy) *sc.status_copy = cta_flag ? kStatusNonFinite : 0;
+            } else if (cta_flag) {
+                atomicOr(sc.status, kStatusNonFinite);
+                if (sc.status_copy) atomicOr(sc.status_copy, kStatusNonFinite);
+            }
         }
-        const float w = weights_parallel(a, M, sm.w, flagged);
-        if (tid < M) {
-            sc.beta[tid] = w;
-            if (sc.weights_out) sc.weights_out[tid] = w;
+        trace.done();
+        return;
+    }
+
+    // MGRAWA / GRAWA (launched as one CTA)
+    const int P = max(1, min((K + 1) / 2, static_cast<int>(blockDim.x) / M));
+    const int run = (K + P - 1) / P;
+    if (tid < P * M) {
+        const int p = tid / M, m = tid - p * M;
+        const int k1 = min(K, (p + 1) * run);
+        double a = 0.0;
+        for (int k = p * run; k < k1; ++k) {
+            const size_t idx = static_cast<size_t>(k) * M + m;
+            const double s = row_sumsq(sc, bins, idx);
+            const double term = row_term(sc, idx, s);
+            store_row(sc, idx, s, term);
+            a += term;
+        }
+        part_sm[tid] = a;
+    }
+    __syncthreads();
+    if (tid < M) {
+        double a = 0.0;
+        for (int p = 0; p < P; ++p) a += part_sm[p * M + tid];
+        if (sc.variant == kGrawa) a = sqrt(a);
+        sc.A[static_cast<size_t>(K) * M + tid] = a;
+        if (sc.scores_out) sc.scores_out[tid] = a;
+        score_sm[tid] = a;
+    }
+    __syncthreads();
+    if (warp == 0) {
+        const double a0 = lane < M ? score_sm[lane] : 0.0;
+        const double a1 = lane + 32 < M ? score_sm[lane + 32] : 0.0;
+        float w0, w1;
+        int flagged;
+        weights_warp(a0, a1, M, w0, w1, flagged);
+        if (lane < M) {
+            sc.beta[lane] = w0;
+            if (sc.weights_out) sc.weights_out[lane] = w0;
+        }
+        if (lane + 32 < M) {
+            sc.beta[lane + 32] = w1;
+            if (sc.weights_out) sc.weights_out[lane + 32] = w1;
+        }
+        if (lane == 0) {
+            *sc.status = flagged ? kStatusNonFinite : 0;
+            if (sc.status_copy) *sc.status_copy = flagged ? kStatusNonFinite : 0;
         }
     }
-    if (tid == 0) {
-        *sc.status = flagged ? kStatusNonFinite : 0;
-        *sc.work_counter = 0u;
-    }
+    trace.done();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -318,16 +453,23 @@ template <int UNROLL>
 __global__ void __launch_bounds__(kThreads, 6)
 sumsq_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
 {
-    grid_dependency_sync();
     __shared__ double warp_part[2][kThreads / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int C = sc.C;
+    // the work list belongs to the plan, not to the kernel before this one: fetch the first item early
+    Segment first_sg = Segment{0, 0, 0};
+    if (static_cast<int>(blockIdx.x) < items) first_sg = sc.segs[blockIdx.x % C];
+    KernelTrace trace(0);
+    grid_dependency_sync();
+    trace.go();
+    const int buf = __ldcg(sc.next_buf);
+    unsigned long long* bins = sc.bins + static_cast<size_t>(buf) * bins_copy_words(sc);
 
     int parity = 0;
     for (int item = blockIdx.x; item < items; item += gridDim.x, parity ^= 1) {
         const int m = item / C;
         const int s = item - m * C;
-        const Segment sg = sc.segs[s];
+        const Segment sg = (item == static_cast<int>(blockIdx.x)) ? first_sg : sc.segs[s];
         const float* __restrict__ g = grads.p[m];
         const long long b = sg.begin, e = b + sg.len;
         long long hb, te;
@@ -373,23 +515,11 @@ sumsq_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
             double total = 0.0;
 #pragma unroll
             for (int w = 0; w < kThreads / 32; ++w) total += warp_part[parity][w];
-            sc.partials[static_cast<size_t>(m) * C + s] = total;
+            bins_add(bins + static_cast<size_t>(sg.layer) * sc.M + m, static_cast<size_t>(sc.K) * sc.M, total);
         }
     }
-}
-
-// Steps 1b-3: one CTA per layer reduces the layer's partials and, for LGRAWA, computes its
-// weights; the CTA that arrives last completes the step (see finalize_arrive).
-// (Folding this into the sum-of-squares kernel with one ticket per layer was measured slower: the
-// fence and atomic each CTA then needs before it can retire cost more than the launch they save.)
-__global__ void __launch_bounds__(kThreads)
-finalize_kernel(StepScratch sc)
-{
-    grid_dependency_sync();
-    __shared__ FinalizeSmem fsm;
-    const int k = blockIdx.x;
-    if (sc.given != nullptr || sc.layer_seg_first[k] != sc.layer_seg_first[k + 1]) finalize_layer(sc, k, fsm);
-    finalize_arrive(sc, fsm);
+    bins_turnover(sc, buf);
+    trace.done();
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -433,48 +563,75 @@ template <> struct VecIO<2> {
     static __device__ __forceinline__ void st(float* p, const float (&o)[2]) { __stcs(reinterpret_cast<float2*>(p), make_float2(o[0], o[1])); }
 };
 
+// `preload` != 0: the first chunk of parameters is loaded BEFORE the dependency wait, so that these
+// loads overlap the tail of the kernels that produce the weights.  Only valid when every kernel
+// that may still be running at that point leaves the parameters alone, i.e. when the kernels in
+// front of this one on the stream are this library's own sum-of-squares / finalisation kernels
+// (they pass their own dependency wait before they let this kernel start, so whatever the caller
+// ran earlier has completed by then).
 template <int M, bool PER_LAYER>
 __global__ void __launch_bounds__(kThreads, 2)
 center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restrict__ beta,
                    const Segment* __restrict__ segs, int item_begin, int item_end, long long n, int tile, float lambda,
-                   int vec_ok)
+                   int vec_ok, int preload)
 {
-    grid_dependency_sync();
     constexpr int COLS = pull_cols(M);
     constexpr int VEC = pull_vec(M);
-    const float oml = 1.0f - lambda;
     const int tid = threadIdx.x;
+    int item = item_begin + blockIdx.x;
+    // the work list belongs to the plan, not to the kernel before this one: fetch the first item early
+    int layer = 0, ncol = 0;
+    long long b = 0, e = 0, hb = 0, te = 0;
+    auto locate = [&](int it) {
+        if (PER_LAYER) {
+            const Segment sg = segs[it];
+            b = sg.begin;
+            e = b + sg.len;
+            layer = sg.layer;
+        } else {
+            b = static_cast<long long>(it) * tile;
+            e = min(n, b + tile);
+        }
+        split_range(b, e, vec_ok, hb, te);
+        ncol = static_cast<int>((te - hb) / VEC);               // te - hb is a multiple of 4
+    };
+    float v[COLS][M][VEC];
+    auto load_chunk = [&](int c0) {
+#pragma unroll
+        for (int q = 0; q < COLS; ++q) {
+            const int c = c0 + q * kThreads + tid;
+            if (c < ncol && in_bounds(hb + static_cast<long long>(c) * VEC, VEC, n)) {
+#pragma unroll
+                for (int m = 0; m < M; ++m) VecIO<VEC>::ld(x.p[m] + hb + static_cast<long long>(c) * VEC, v[q][m]);
+            }
+        }
+    };
+    bool loaded = false;
+    if (item < item_end) {
+        locate(item);
+        if (preload) {
+            load_chunk(0);
+            loaded = true;
+        }
+    }
+    KernelTrace trace(2);
+    grid_dependency_sync();
+    trace.go();
+    const float oml = 1.0f - lambda;
     float w[M];
     if (!PER_LAYER) {
 #pragma unroll
         for (int m = 0; m < M; ++m) w[m] = beta[m];
     }
-    for (int item = item_begin + blockIdx.x; item < item_end; item += gridDim.x) {
-        long long b, e;
+    while (item < item_end) {
         if (PER_LAYER) {
-            const Segment sg = segs[item];
-            b = sg.begin;
-            e = b + sg.len;
-            const float* __restrict__ bt = beta + static_cast<size_t>(sg.layer) * M;
+            const float* __restrict__ bt = beta + static_cast<size_t>(layer) * M;
 #pragma unroll
             for (int m = 0; m < M; ++m) w[m] = bt[m];
-        } else {
-            b = static_cast<long long>(item) * tile;
-            e = min(n, b + tile);
         }
-        long long hb, te;
-        split_range(b, e, vec_ok, hb, te);
-        const int ncol = static_cast<int>((te - hb) / VEC);      // te - hb is a multiple of 4
         for (int c0 = 0; c0 < ncol; c0 += kThreads * COLS) {
-            float v[COLS][M][VEC];
-#pragma unroll
-            for (int q = 0; q < COLS; ++q) {
-                const int c = c0 + q * kThreads + tid;
-                if (c < ncol && in_bounds(hb + static_cast<long long>(c) * VEC, VEC, n)) {
-#pragma unroll
-                    for (int m = 0; m < M; ++m) VecIO<VEC>::ld(x.p[m] + hb + static_cast<long long>(c) * VEC, v[q][m]);
-                }
-            }
+            if (!loaded) load_chunk(c0);
+            loaded = false;
 #pragma unroll
             for (int q = 0; q < COLS; ++q) {
                 const int c = c0 + q * kThreads + tid;
@@ -498,11 +655,15 @@ center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restric
                 }
             }
         }
+        loaded = false;                                  // an item without a vector body used nothing
         for (long long i = b + tid; i < hb; i += kThreads)
             if (in_bounds(i, 1, n)) pull_scalar<M>(x, center, w, lambda, oml, i);
         for (long long i = te + tid; i < e; i += kThreads)
             if (in_bounds(i, 1, n)) pull_scalar<M>(x, center, w, lambda, oml, i);
+        item += gridDim.x;
+        if (item < item_end) locate(item);
     }
+    trace.done();
 }
 
 // Steps 4-5 for any M up to kMaxWorkers and any alignment: scalar, two passes over the workers

@@ -76,16 +76,21 @@ template <typename T, int UNROLL>
 __global__ void __launch_bounds__(kThreads, 5)
 sumsq16_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
 {
-    grid_dependency_sync();
     __shared__ double warp_part[2][kThreads / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int C = sc.C;
+    // the work list belongs to the plan, not to the kernel before this one: fetch the first item early
+    Segment first_sg = Segment{0, 0, 0};
+    if (static_cast<int>(blockIdx.x) < items) first_sg = sc.segs[blockIdx.x % C];
+    grid_dependency_sync();
+    const int buf = __ldcg(sc.next_buf);
+    unsigned long long* bins = sc.bins + static_cast<size_t>(buf) * bins_copy_words(sc);
 
     int parity = 0;
     for (int item = blockIdx.x; item < items; item += gridDim.x, parity ^= 1) {
         const int m = item / C;
         const int s = item - m * C;
-        const Segment sg = sc.segs[s];
+        const Segment sg = (item == static_cast<int>(blockIdx.x)) ? first_sg : sc.segs[s];
         const T* __restrict__ g = reinterpret_cast<const T*>(grads.p[m]);
         const long long b = sg.begin, e = b + sg.len;
         long long hb, te;
@@ -130,9 +135,10 @@ sumsq16_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
             double total = 0.0;
 #pragma unroll
             for (int w = 0; w < kThreads / 32; ++w) total += warp_part[parity][w];
-            sc.partials[static_cast<size_t>(m) * C + s] = total;
+            bins_add(bins + static_cast<size_t>(sg.layer) * sc.M + m, static_cast<size_t>(sc.K) * sc.M, total);
         }
     }
+    bins_turnover(sc, buf);
 }
 
 // Shape of the 16-bit centre+pull kernel: columns of WORDS 32-bit words (two elements each) kept
@@ -186,6 +192,8 @@ __global__ void __launch_bounds__(kThreads, 2)
 center_pull16_kernel(MutPtrs x, T* __restrict__ center, const float* __restrict__ beta, const Segment* __restrict__ segs,
                      int item_begin, int item_end, long long n, int tile, float lambda, int vec_ok)
 {
+    Segment first_sg = Segment{0, 0, 0};           // plan data: independent of the kernel before this one
+    if (PER_LAYER && item_begin + static_cast<int>(blockIdx.x) < item_end) first_sg = segs[item_begin + blockIdx.x];
     grid_dependency_sync();
     constexpr int COLS = pull16_cols(M);
     constexpr int WORDS = pull16_words(M);
@@ -197,10 +205,10 @@ center_pull16_kernel(MutPtrs x, T* __restrict__ center, const float* __restrict_
 #pragma unroll
         for (int m = 0; m < M; ++m) w[m] = beta[m];
     }
-    for (int item = item_begin + blockIdx.x; item < item_end; item += gridDim.x) {
+    for (int item = item_begin + blockIdx.x; item < item_end;) {
         long long b, e;
         if (PER_LAYER) {
-            const Segment sg = segs[item];
+            const Segment sg = first_sg;
             b = sg.begin;
             e = b + sg.len;
             const float* __restrict__ bt = beta + static_cast<size_t>(sg.layer) * M;
@@ -271,6 +279,8 @@ center_pull16_kernel(MutPtrs x, T* __restrict__ center, const float* __restrict_
             if (in_bounds(i, 1, n)) pull16_scalar<T, M>(x, center, w, lambda, oml, i);
         for (long long i = te + tid; i < e; i += kThreads)
             if (in_bounds(i, 1, n)) pull16_scalar<T, M>(x, center, w, lambda, oml, i);
+        item += gridDim.x;
+        if (PER_LAYER && item < item_end) first_sg = segs[item];
     }
 }
 

@@ -36,10 +36,13 @@ def test_version_and_strings():
     assert grawa.grawa_status_string(-3) and grawa.grawa_status_string(-99)
 
 
-def test_workspace_bytes_grows_with_work_and_rejects_bad_tables():
+def test_workspace_bytes_grows_with_layers_and_workers_and_rejects_bad_tables():
     small = grawa.grawa_workspace_bytes(1000, 4, [0, 10, 1000])
-    big = grawa.grawa_workspace_bytes(10_000_000, 4, [0, 10, 10_000_000])
-    assert 0 < small < big and small % 256 == 0
+    more_layers = grawa.grawa_workspace_bytes(1000, 4, [0, 10, 20, 30, 40, 1000])
+    more_workers = grawa.grawa_workspace_bytes(1000, 16, [0, 10, 1000])
+    assert 0 < small < more_layers and small < more_workers and small % 256 == 0
+    # the scratch holds per-(layer, worker) tables only: it does not grow with the vector
+    assert grawa.grawa_workspace_bytes(10_000_000, 4, [0, 10, 10_000_000]) == small
     assert grawa.grawa_workspace_bytes(1000, 4) > 0
     assert grawa.grawa_workspace_bytes(1000, 0) == 0
     assert grawa.grawa_workspace_bytes(1000, 65) == 0
