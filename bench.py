@@ -3,16 +3,22 @@
 CPU oracle.
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--variant lgrawa|mgrawa|grawa]
+                    [--op step|prox|from_norms] [--dtype f32|bf16|f16] [--sharded]
     python bench.py --impl reference ...        # times the float64 CPU oracle instead
 
 A step is one whole update (gradient sums of squares -> scores -> weights -> centre -> pull of all
-M workers) on one synthetic workload through the library's C ABI.  Prints one JSON line.
-The update does not shard across GPUs by itself ("replicas only"): with --gpus N each rank runs
-the same workload on its own GPU and the line reports the aggregate.
+M workers) on one synthetic workload through the library's C ABI.  Prints one JSON line.  Besides
+the headline (ViT-B/16 table, LGRAWA) the default line carries short runs of every workload of at
+least 10 M parameters in both variants (`targets`), of the proximity step, the step from given norms
+and the step on bfloat16 storage (`ops`), and of the two small workloads eagerly and in a CUDA graph
+(`small`).  The update does not shard across GPUs by itself ("replicas only"): with --gpus N each
+rank runs the same workload on its own GPU and the line reports the aggregate; --sharded instead cuts
+ONE problem by element range over the ranks (one all-gather of a [K, M] table per step).
 """
 from __future__ import annotations
 
 import argparse
+import hashlib
 import json
 import os
 import subprocess
@@ -31,8 +37,11 @@ import gen  # noqa: E402
 METRIC = "GRAWA update steps/sec (achieved HBM GB/s and fraction of roofline in `roofline`)"
 DEFAULT_WORKLOAD = "vit_b16"
 DEFAULT_VARIANT = "lgrawa"
+TARGET_WORKLOADS = ("resnet18_imagenet", "vgg16", "vit_b16")       # the workloads of at least 10 M parameters
+SMALL_WORKLOADS = ("toy10", "resnet20_cifar")
 NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
+ELEM_BYTES = {"f32": 4, "bf16": 2, "f16": 2}
 
 
 def measured_peak_gbs():
@@ -46,7 +55,7 @@ def measured_peak_gbs():
 # ------------------------------------------------------------------ clocks
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
+    """Samples SM clock and throttle reasons with nvidia-smi while the timed regions run."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
@@ -80,12 +89,16 @@ class ClockSampler:
             os.unlink(self.path)
         except Exception:
             return out
-        sm, reasons = [], set()
+        sm, power, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for r in rows:
             try:
-                sm.append(float(r[0]))
+                watts = float(r[2])
                 out["sm_max_mhz"] = float(r[1])
+                if watts < 300.0:                    # idle sample (input generation on the host): not "under load"
+                    continue
+                sm.append(float(r[0]))
+                power.append(watts)
                 for name, v in zip(names, r[3:7]):
                     if v.strip().lower().startswith("active"):
                         reasons.add(name)
@@ -94,20 +107,13 @@ class ClockSampler:
         if sm:
             out["sm_mhz"] = float(np.median(sm))
             out["samples"] = len(sm)
+            out["power_w_max"] = max(power)
+        out["samples_total"] = len(rows)
         out["reasons"] = sorted(reasons)
         return out
 
 
-# ------------------------------------------------------------------ the CUDA arm
-
-def pinned_inputs(cfg):
-    """Generates the workload straight into pinned host tensors (also used as the e2e source)."""
-    import torch
-    hp = [torch.empty(cfg.n, dtype=torch.float32).pin_memory() for _ in range(cfg.M)]
-    hg = [torch.empty(cfg.n, dtype=torch.float32).pin_memory() for _ in range(cfg.M)]
-    gen.make_inputs(cfg, [t.numpy() for t in hp], [t.numpy() for t in hg])
-    return hp, hg
-
+# ------------------------------------------------------------------ workloads on the device
 
 def workload_config(args):
     """The named workload, or (for small profiling captures) only its first --layers-limit layers
@@ -121,32 +127,118 @@ def workload_config(args):
     return cfg
 
 
-def step_fn(grawa, variant):
-    return {"lgrawa": grawa.grawa_lgrawa_step, "mgrawa": grawa.grawa_mgrawa_step, "grawa": grawa.grawa_grawa_step}[variant]
+def describe(cfg, variant, op="step", dtype="f32", world=1, sharded=False):
+    """The `config` object of a line; both arms build it here so that they agree key by key."""
+    what = {"step": f"{variant.upper()} step", "prox": "proximity step", "from_norms": f"{variant.upper()} step from given layer norms"}[op]
+    par = "single GPU" if world == 1 else ("element-range sharded" if sharded else "replicas only")
+    return {"workload": f"{cfg.name} layer table, M={cfg.M} workers, n={cfg.n}, K={cfg.K} layers, "
+                        f"{what}, pull={cfg.pull}, seed={cfg.seed}",
+            "variant": variant, "op": op, "storage": dtype, "M": cfg.M, "n": cfg.n, "n_layers": cfg.K, "parallelism": par,
+            "l2": "inputs larger than L2 (no flush needed)" if op_bytes(cfg, op, dtype) > 4 * 126e6 else "L2-resident workload",
+            "algorithmic_bytes_per_step": op_bytes(cfg, op, dtype)}
 
 
-def time_device_steps(grawa, cfg, variant, x, g, center, steps, warmup, kernel_timing):
-    """K back-to-back steps between two CUDA events on the launching stream.  Returns ms per step,
-    launches in the timed region and (if asked) the per-phase kernel times."""
+def op_bytes(cfg, op, dtype="f32", n=None):
+    """Algorithmic bytes of one call: gradients read once (step only), parameters read and written
+    once, centre written once (step) or read once (proximity step)."""
+    n = cfg.n if n is None else n
+    e = ELEM_BYTES[dtype]
+    streams = {"step": 3 * cfg.M + 1, "from_norms": 2 * cfg.M + 1, "prox": 2 * cfg.M + 1}[op]
+    return streams * e * n
+
+
+def pinned_inputs(cfg):
+    """Generates the workload straight into pinned host tensors (also the source of the e2e run)."""
     import torch
-    fn = step_fn(grawa, variant)
-    off = cfg.offsets()
-    for _ in range(warmup):
-        fn(x, g, cfg.pull, off, center)
-    torch.cuda.synchronize()
-    grawa.grawa_set_option("kernel_timing", 1 if kernel_timing else 0)
-    grawa.grawa_collect_kernel_times()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    launches = grawa.grawa_launch_count()
-    e0.record()
-    for _ in range(steps):
-        fn(x, g, cfg.pull, off, center)
-    e1.record()
-    torch.cuda.synchronize()
-    launches = grawa.grawa_launch_count() - launches
-    grawa.grawa_set_option("kernel_timing", 0)
-    phases = grawa.grawa_collect_kernel_times() if kernel_timing else None
-    return e0.elapsed_time(e1) / steps, launches, phases
+    hp = [torch.empty(cfg.n, dtype=torch.float32).pin_memory() for _ in range(cfg.M)]
+    hg = [torch.empty(cfg.n, dtype=torch.float32).pin_memory() for _ in range(cfg.M)]
+    gen.make_inputs(cfg, [t.numpy() for t in hp], [t.numpy() for t in hg])
+    return hp, hg
+
+
+def device_inputs(cfg, j0=0, j1=None):
+    """The workload (or the element range [j0, j1) of it) in device memory, generated on the host."""
+    import torch
+    p, g = gen.make_inputs(cfg)
+    j1 = cfg.n if j1 is None else j1
+    x = [torch.from_numpy(a[j0:j1]).cuda() for a in p]
+    gr = [torch.from_numpy(a[j0:j1]).cuda() for a in g]
+    return x, gr
+
+
+class Call:
+    """One timed operation bound to its buffers: `fn()` enqueues one call on the current stream."""
+
+    def __init__(self, grawa, cfg, variant, op, dtype, x, g, center, off=None):
+        import torch
+        self.grawa, self.cfg, self.variant, self.op, self.dtype = grawa, cfg, variant, op, dtype
+        off = cfg.offsets() if off is None else off
+        tdt = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[dtype]
+        if dtype != "f32":
+            x, g, center = [t.to(tdt) for t in x], [t.to(tdt) for t in g], center.to(tdt)
+        self.x, self.g, self.center = x, g, center
+        if op == "prox":
+            if dtype != "f32":
+                raise SystemExit("the proximity step runs on fp32 storage")
+            self.fn = lambda: grawa.grawa_prox_step(x, center, 0.05 / 16)        # mu / tau of the paper's grid
+        elif op == "from_norms":
+            if dtype != "f32":
+                raise SystemExit("the step from given norms runs on fp32 storage")
+            K, G = cfg.K, (cfg.K if variant == "lgrawa" else 1)
+            norms = torch.empty(K * cfg.M, dtype=torch.float64, device="cuda")
+            grawa.grawa_lgrawa_step(x, g, 0.0, off, None, scores_out=norms)      # per-layer norms, workers untouched
+            torch.cuda.synchronize()
+            self.norms = norms
+            self.fn = lambda: grawa.grawa_step_from_layer_norms(variant, x, norms, cfg.pull, off, center)
+        elif dtype == "f32":
+            step = {"lgrawa": grawa.grawa_lgrawa_step, "mgrawa": grawa.grawa_mgrawa_step, "grawa": grawa.grawa_grawa_step}[variant]
+            self.fn = lambda: step(x, g, cfg.pull, off, center)
+        else:
+            self.fn = lambda: grawa.grawa_step_typed(variant, x, g, cfg.pull, off, center)
+
+    def time(self, steps, warmup, phases=False):
+        """K back-to-back calls between two CUDA events on the launching stream.  Returns ms per call,
+        the library's launches inside the region and (if asked) the per-kernel times of a step."""
+        import torch
+        grawa = self.grawa
+        for _ in range(warmup):
+            self.fn()
+        torch.cuda.synchronize()
+        grawa.grawa_set_option("kernel_timing", 1 if phases else 0)
+        grawa.grawa_collect_kernel_times()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        launches = grawa.grawa_launch_count()
+        e0.record()
+        for _ in range(steps):
+            self.fn()
+        e1.record()
+        torch.cuda.synchronize()
+        launches = grawa.grawa_launch_count() - launches
+        grawa.grawa_set_option("kernel_timing", 0)
+        ph = grawa.grawa_collect_kernel_times() if phases else None
+        return e0.elapsed_time(e1) / steps, launches, ph
+
+
+def rates(bytes_per_call, ms, peak):
+    gbs = bytes_per_call / (ms * 1e-3) / 1e9
+    return {"ms_per_step": ms, "steps_per_s": 1e3 / ms, "achieved_gbs": gbs, "frac_of_measured_peak": gbs / peak,
+            "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS}
+
+
+def kernel_table(cfg, dtype, ph, peak, with_sumsq=True):
+    """Per-kernel times of a step (library CUDA events around each kernel, dependent launch off) and the
+    roofline of the two streaming kernels."""
+    e, n, M = ELEM_BYTES[dtype], cfg.n, cfg.M
+    k = ph["steps"]
+    out = {"finalize": {"kernel_ms": ph["finalize_ms"] / k}}
+    pull_ms, pull_bytes = ph["center_pull_ms"] / k, (2 * M + 1) * e * n
+    out["center_pull"] = {"kernel_ms": pull_ms, "algorithmic_bytes_per_launch": pull_bytes,
+                          "achieved_gbs": pull_bytes / (pull_ms * 1e-3) / 1e9, "frac_of_measured_peak": pull_bytes / (pull_ms * 1e-3) / 1e9 / peak}
+    if with_sumsq:
+        s_ms, s_bytes = ph["sumsq_ms"] / k, M * e * n
+        out["sumsq"] = {"kernel_ms": s_ms, "algorithmic_bytes_per_launch": s_bytes,
+                        "achieved_gbs": s_bytes / (s_ms * 1e-3) / 1e9, "frac_of_measured_peak": s_bytes / (s_ms * 1e-3) / 1e9 / peak}
+    return out
 
 
 def time_e2e_steps(grawa, cfg, variant, hp, hg, hc, steps, warmup):
@@ -164,47 +256,67 @@ def time_e2e_steps(grawa, cfg, variant, hp, hg, hc, steps, warmup):
     return (time.perf_counter() - t0) * 1e3 / steps
 
 
-def oracle_baseline(cfg, variant, params_np, grads_np, budget_s=15.0):
-    """The CPU oracle as it stands (plain C, one thread) on a bounded sample of the workload: the
-    first layers, all M workers, sized from a short probe to about `budget_s` seconds."""
-    import oracle
-    off = cfg.offsets()
-    probe_n = min(cfg.n, 1 << 20)
-    view = lambda arrs, hi: [a[:hi] for a in arrs]
-    t0 = time.perf_counter()
-    _oracle_sample(oracle, variant, view(params_np, probe_n), view(grads_np, probe_n), cfg.pull, np.array([0, probe_n]))
-    per_elem = (time.perf_counter() - t0) / (probe_n * cfg.M)
-    want = int(budget_s / (per_elem * cfg.M))
-    k_hi = max(1, int(np.searchsorted(off, min(want, cfg.n), side="right")) - 1)
-    n_s = int(off[k_hi])
-    if n_s == 0:
-        k_hi, n_s = cfg.K, cfg.n
-    t0 = time.perf_counter()
-    _oracle_sample(oracle, variant, view(params_np, n_s), view(grads_np, n_s), cfg.pull, off[:k_hi + 1])
-    dt = time.perf_counter() - t0
-    full = dt * cfg.n / n_s
-    return {"value": 1.0 / full, "unit": "steps/s", "cores": 1, "kind": "oracle",
-            "sample": f"first {k_hi} of {cfg.K} layers ({n_s} of {cfg.n} elements, all {cfg.M} workers), "
-                      f"{dt:.2f} s measured, scaled by elements to a full step",
-            "seconds_per_step_scaled": full}
+# ------------------------------------------------------------------ the CPU oracle, timed
 
-
-def _oracle_sample(oracle, variant, p, g, pull, off):
-    """One oracle step, streamed in chunks with reused output buffers (allocation is not the method)."""
-    n, M = p[0].size, len(p)
+def _oracle_step(oracle, variant, p, g, pull, off, bufs):
+    """One whole oracle step, streamed in chunks with reused output buffers (allocation is not the method)."""
+    n = p[0].size
     S = oracle.sumsq(g, off)
     beta, _ = oracle.weights(oracle.scores(S, variant))
-    chunk = 1 << 18
-    bufs = (np.zeros(chunk), [np.zeros(chunk) for _ in range(M)])
+    chunk = bufs[0].size
     for j0 in range(0, n, chunk):
         oracle.center_pull(p, beta, pull, off, j0, min(n, j0 + chunk), out=bufs)
+
+
+def oracle_timing(cfg, variant, p, g, budget_s, steps_wanted=1, warmup=1):
+    """The CPU oracle as it stands (plain C, one thread) on the workload.  Whole steps when one step
+    fits the budget; otherwise each step is a prefix of whole layers (all M workers), sized from a
+    warmed probe, and the figure is scaled by elements.  Returns the `cpu_baseline` object and the
+    measured seconds per (sampled) step."""
+    import oracle
+    off = cfg.offsets()
+    chunk = 1 << 18
+    bufs = (np.zeros(chunk), [np.zeros(chunk) for _ in range(cfg.M)])
+    probe_n = int(min(cfg.n, 1 << 20))
+    view = lambda arrs, hi: [a[:hi] for a in arrs]
+    probe_off = np.array([0, probe_n])
+    _oracle_step(oracle, variant, view(p, probe_n), view(g, probe_n), cfg.pull, probe_off, bufs)     # warms pages and caches
+    t0 = time.perf_counter()
+    _oracle_step(oracle, variant, view(p, probe_n), view(g, probe_n), cfg.pull, probe_off, bufs)
+    per_elem = (time.perf_counter() - t0) / probe_n
+    full_estimate = per_elem * cfg.n
+    per_step_budget = budget_s / max(1, steps_wanted + warmup)
+    if full_estimate <= per_step_budget:
+        k_hi, n_s = cfg.K, cfg.n
+    else:
+        want = int(per_step_budget / per_elem)
+        k_hi = max(1, int(np.searchsorted(off, min(want, cfg.n), side="right")) - 1)
+        while k_hi < cfg.K and off[k_hi] == 0:
+            k_hi += 1
+        n_s = int(off[k_hi])
+    soff = off[:k_hi + 1]
+    ps, gs = view(p, n_s), view(g, n_s)
+    times = []
+    for i in range(warmup + steps_wanted):
+        t0 = time.perf_counter()
+        _oracle_step(oracle, variant, ps, gs, cfg.pull, soff, bufs)
+        if i >= warmup:
+            times.append(time.perf_counter() - t0)
+    sec = float(np.mean(times))
+    whole = n_s == cfg.n
+    sample = (f"{len(times)} whole step(s): all {cfg.K} layers, {cfg.n} elements, {cfg.M} workers" if whole else
+              f"{len(times)} step(s) of the first {k_hi} of {cfg.K} layers ({n_s} of {cfg.n} elements, all {cfg.M} workers), "
+              f"scaled by elements to a full step")
+    full = sec * cfg.n / n_s
+    return {"value": 1.0 / full, "unit": "steps/s", "cores": 1, "kind": "oracle", "sample": sample,
+            "seconds_per_sampled_step": sec, "whole_steps": whole}, full
 
 
 def max_over_ranks(values, world, device):
     """Element-wise maximum of per-rank timings (the slowest rank defines the step time)."""
     import torch
-    t = torch.tensor(list(values), dtype=torch.float64, device=device)
     import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
     if world > 1 or (dist.is_available() and dist.is_initialized()):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return [float(v) for v in t]
@@ -215,48 +327,46 @@ def whole_job_steps_per_s(world, ms_per_step_max):
     return world * 1e3 / ms_per_step_max
 
 
-# DRAM traffic of one centre+pull launch, from the ncu capture summarised in
-# profiles/center_pull_kernel_vit_b16_28layers.md (M = 16; 1916.46 MB for 14 918 400 elements),
-# scaled to a full launch by the number of elements.  Only valid for the kernel source it was taken
-# from: the hash below is that of the centre+pull kernel's text in csrc/kernels.cuh (from its
-# heading comment to the next kernel's) at capture time; anything else reports null.
-TRAFFIC_CAPTURE = {"M": 16, "dram_bytes_per_element": (955.077376e6 + 961.380608e6) / 14918400,
-                   "kernels_sha256": "e63e74aaf440bb7584d4f7c4bf30a29a04d4fe74544ad2ec2a8e2d6753ce5a49"}
+# DRAM bytes per element of one launch, from stored ncu captures of a smaller case of the same kernel
+# (first 28 layers of the ViT-B/16 table, 14 918 400 elements, M = 16), scaled to a full launch by the
+# number of elements.  A capture is only quoted for the kernel source and launch code it was taken
+# from (hashes of the kernel's text in csrc/kernels.cuh and of csrc/grawa.cu) and with every tuning
+# knob at its default; anything else reports null.
+CAPTURE_ELEMENTS = 14918400
+STORED_CAPTURES = {
+    "center_pull": {"M": 16, "dram_bytes": None, "begin": "// Steps 4-5, register variant", "end": "// Steps 4-5 for any M up to",
+                    "kernel_sha256": None, "host_sha256": None},
+    "sumsq": {"M": 16, "dram_bytes": None, "begin": "// Step 1 (Eq. 3 / Eq. 5): partial", "end": "// Steps 4-5, register variant",
+              "kernel_sha256": None, "host_sha256": None},
+}
+DEFAULT_KNOBS = {"sumsq_tile": 8192, "pull_tile": 0, "pull_variant": 0, "bulk_tile": 0, "sumsq_ctas_per_sm": 0,
+                 "pull_ctas_per_sm": 0, "dependent_launch": 1, "pull_preload": 1}
 
 
-# Same for the sum-of-squares kernel (profiles/sumsq_kernel_vit_b16_28layers.md: 954.82 MB read +
-# 4.35 MB written for 14 918 400 elements at M = 16).
-SUMSQ_TRAFFIC_CAPTURE = {"M": 16, "dram_bytes_per_element": (954.82112e6 + 4.346368e6) / 14918400,
-                         "kernels_sha256": "3cad663f1177f4a514a5233796ed3df1eeae9242aa4c7b3b5f6ff7623fd66d56"}
-
-
-def sumsq_traffic(cfg):
-    import hashlib
-    path = os.path.join(ROOT, "paper_2403_04206_b200", "csrc", "kernels.cuh")
+def source_hashes(which):
+    cap = STORED_CAPTURES[which]
     try:
-        text = open(path).read()
-        region = text[text.index("// Step 1 (Eq. 3 / Eq. 5): partial[m][s]"):text.index("// Steps 1b-3: one CTA per layer reduces")]
-        digest = hashlib.sha256(region.encode()).hexdigest()
+        text = open(os.path.join(ROOT, "paper_2403_04206_b200", "csrc", "kernels.cuh")).read()
+        region = text[text.index(cap["begin"]):text.index(cap["end"])]
+        host = open(os.path.join(ROOT, "paper_2403_04206_b200", "csrc", "grawa.cu")).read()
     except (OSError, ValueError):
-        return None
-    if digest != SUMSQ_TRAFFIC_CAPTURE["kernels_sha256"] or cfg.M != SUMSQ_TRAFFIC_CAPTURE["M"]:
-        return None
-    return SUMSQ_TRAFFIC_CAPTURE["dram_bytes_per_element"] * cfg.n
+        return None, None
+    return hashlib.sha256(region.encode()).hexdigest(), hashlib.sha256(host.encode()).hexdigest()
 
 
-def center_pull_traffic(cfg):
-    import hashlib
-    path = os.path.join(ROOT, "paper_2403_04206_b200", "csrc", "kernels.cuh")
-    try:
-        text = open(path).read()
-        region = text[text.index("// Steps 4-5, register variant"):text.index("// Steps 4-5 for any M up to")]
-        digest = hashlib.sha256(region.encode()).hexdigest()
-    except (OSError, ValueError):
+def stored_traffic(grawa, which, cfg):
+    """DRAM bytes of one full launch scaled from the stored capture, or None when it does not apply."""
+    cap = STORED_CAPTURES[which]
+    if cap["dram_bytes"] is None or cfg.M != cap["M"]:
         return None
-    if digest != TRAFFIC_CAPTURE["kernels_sha256"] or cfg.M != TRAFFIC_CAPTURE["M"]:
+    if any(grawa.grawa_get_option(k) != v for k, v in DEFAULT_KNOBS.items()):
         return None
-    return TRAFFIC_CAPTURE["dram_bytes_per_element"] * cfg.n
+    if source_hashes(which) != (cap["kernel_sha256"], cap["host_sha256"]):
+        return None
+    return cap["dram_bytes"] / CAPTURE_ELEMENTS * cfg.n
 
+
+# ------------------------------------------------------------------ the CUDA arm
 
 def run_cuda(args):
     import torch
@@ -272,121 +382,250 @@ def run_cuda(args):
 
     import paper_2403_04206_b200 as grawa
     grawa.library()
-
-    cfg = workload_config(args)
-    variant = args.variant
     for kv in args.option:
         name, value = kv.split("=")
         grawa.grawa_set_option(name, int(value))
-    hp, hg = pinned_inputs(cfg)
-    x = [t.cuda(non_blocking=True) for t in hp]
-    g = [t.cuda(non_blocking=True) for t in hg]
-    center = torch.empty(cfg.n, device="cuda")
-    torch.cuda.synchronize()
 
     def barrier():
         if use_dist:
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- timed region: exactly K steps, device-resident inputs
+    peak, peak_src = measured_peak_gbs()
+    cfg = workload_config(args)
+    variant, op, dtype = args.variant, args.op, args.dtype
     sampler = ClockSampler(local_rank)
-    barrier()
     sampler.start()
-    ms, launches, _ = time_device_steps(grawa, cfg, variant, x, g, center, args.steps, args.warmup, False)
-    clocks = sampler.stop()
+
+    # ---- headline: device-resident inputs, exactly K calls
+    hp, hg = pinned_inputs(cfg)
+    x = [t.cuda(non_blocking=True) for t in hp]
+    g = [t.cuda(non_blocking=True) for t in hg]
+    center = torch.zeros(cfg.n, device="cuda")
+    torch.cuda.synchronize()
+    call = Call(grawa, cfg, variant, op, dtype, x, g, center)
     barrier()
-    # ---- same region again with the library's per-phase events (for the kernel-level roofline)
-    ms_k, _, phases = time_device_steps(grawa, cfg, variant, x, g, center, args.steps, 1, True)
-    status = grawa.grawa_last_step_status()
-    # ---- the other variant of the metric (MGRAWA when the headline is LGRAWA, and the reverse), same workload
-    other = "mgrawa" if variant == "lgrawa" else "lgrawa"
-    other_ms, _, _ = time_device_steps(grawa, cfg, other, x, g, center, max(20, args.steps // 4), 3, False)
+    ms, launches, _ = call.time(args.steps, args.warmup)
+    barrier()
+    line = None
+    alg_bytes = op_bytes(cfg, op, dtype)
+    if op == "prox":
+        kernels, ms_k = None, ms
+    else:
+        # the same region again with the library's events around each kernel (for the kernel-level roofline)
+        ms_k, _, phases = call.time(args.steps, 1, phases=True)
+        kernels = kernel_table(cfg, dtype, phases, peak, with_sumsq=(op == "step"))
+    status = grawa.grawa_last_step_status() if op != "prox" else 0
 
-    # ---- end to end through the host-buffer entry point
-    hc = torch.empty(cfg.n, dtype=torch.float32).pin_memory()
-    e2e_steps = max(1, min(args.steps, args.e2e_steps))
-    e2e_ms = time_e2e_steps(grawa, cfg, variant, hp, hg, hc, e2e_steps, 1)
+    other = None
+    if op == "step" and dtype == "f32":
+        ov = "mgrawa" if variant == "lgrawa" else "lgrawa"
+        o_ms, _, _ = Call(grawa, cfg, ov, "step", "f32", x, g, center).time(max(20, args.steps // 4), 3)
+        other = dict(variant=ov, **rates(alg_bytes, o_ms, peak))
 
-    ms_max, e2e_ms_max = max_over_ranks([ms, e2e_ms], world, "cuda")
+    # ---- end to end through the host-buffer entry point (fp32 step only)
+    e2e_ms, e2e_steps = None, 0
+    if op == "step" and dtype == "f32":
+        hc = torch.empty(cfg.n, dtype=torch.float32).pin_memory()
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        e2e_ms = time_e2e_steps(grawa, cfg, variant, hp, hg, hc, e2e_steps, 1)
+        del hc
+
+    # ---- one problem cut by element range over the ranks (with one rank: the same step through the sharded path)
+    sharded_out = None
+    if args.sharded and op == "step" and dtype == "f32":
+        sharded_out = run_sharded(grawa, cfg, variant, args, world, rank, peak, barrier, x, g, center)
+
+    ms_max, e2e_ms_max = max_over_ranks([ms, e2e_ms if e2e_ms is not None else 0.0], world, "cuda")
+    ops = targets = small = None
+    if world == 1 and not args.headline_only:
+        ops = side_ops(grawa, cfg, variant, x, g, center, args, peak)
+    del call, x, g, center
+    torch.cuda.empty_cache()
+    hp_np, hg_np = [t.numpy() for t in hp], [t.numpy() for t in hg]
+    if world == 1 and not args.headline_only:
+        targets = target_runs(grawa, args, peak, have=(cfg, hp, hg))
+        small = small_runs(grawa, args)
+    clocks = sampler.stop()
 
     if rank == 0:
-        peak, peak_src = measured_peak_gbs()
-        alg_bytes = cfg.algorithmic_bytes()
-        pull_bytes = (2 * cfg.M + 1) * 4 * cfg.n
-        sumsq_bytes = cfg.M * 4 * cfg.n
-        pull_ms = phases["center_pull_ms"] / phases["steps"]
-        sumsq_ms = phases["sumsq_ms"] / phases["steps"]
-        fin_ms = phases["finalize_ms"] / phases["steps"]
-        achieved = pull_bytes / (pull_ms * 1e-3) / 1e9
-        step_gbs = alg_bytes / (ms_max * 1e-3) / 1e9
+        step_rates = rates(alg_bytes, ms_max, peak)
+        dominant = "center_pull" if kernels else "prox"
+        if kernels:
+            kd = kernels["center_pull"]
+            roof = {"bound": "hbm", "kernel": dominant, "achieved": kd["achieved_gbs"], "peak": peak, "peak_source": peak_src,
+                    "unit": "GB/s", "frac": kd["frac_of_measured_peak"], "frac_of_nominal_8TBs": kd["achieved_gbs"] / NOMINAL_HBM_GBS,
+                    "traffic": stored_traffic(grawa, "center_pull", cfg) if dtype == "f32" else None,
+                    "traffic_source": "stored ncu capture (dram bytes read + written) of a launch over "
+                                      f"{CAPTURE_ELEMENTS} elements at the same M, scaled by elements; null when the kernel, its launch "
+                                      "code or a tuning knob differs from the capture's",
+                    "traffic_scaled_from_n": CAPTURE_ELEMENTS,
+                    "algorithmic_bytes_per_launch": kd["algorithmic_bytes_per_launch"], "kernel_ms": kd["kernel_ms"],
+                    "timed_with": "library CUDA events around each kernel in a second K-step region (dependent launch off there)",
+                    "other_kernels": {k: v for k, v in kernels.items() if k != "center_pull"},
+                    "ms_per_step_with_events": ms_k}
+            if "sumsq" in roof["other_kernels"]:
+                roof["other_kernels"]["sumsq"]["traffic"] = stored_traffic(grawa, "sumsq", cfg) if dtype == "f32" else None
+        else:
+            roof = {"bound": "hbm", "kernel": "prox", "achieved": step_rates["achieved_gbs"], "peak": peak, "peak_source": peak_src,
+                    "unit": "GB/s", "frac": step_rates["frac_of_measured_peak"], "frac_of_nominal_8TBs": step_rates["frac_of_nominal_8TBs"],
+                    "traffic": None, "algorithmic_bytes_per_launch": alg_bytes, "kernel_ms": ms_max,
+                    "timed_with": "CUDA events around K back-to-back launches (the call is one kernel)"}
         line = {
             "metric": METRIC, "value": whole_job_steps_per_s(world, ms_max), "unit": "steps/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms_max, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": f"{cfg.name} layer table, M={cfg.M} workers, n={cfg.n}, K={cfg.K} layers, "
-                                   f"{variant.upper()} step, pull={cfg.pull}, seed={cfg.seed}",
-                       "variant": variant, "M": cfg.M, "n": cfg.n, "n_layers": cfg.K,
-                       "parallelism": "replicas only" if world > 1 else "single GPU",
-                       "l2": "inputs larger than L2 (no flush needed)" if alg_bytes > 4 * 126e6 else "L2-resident workload",
-                       "algorithmic_bytes_per_step": alg_bytes},
-            "step_hbm": {"achieved_gbs": step_gbs, "frac_of_measured_peak": step_gbs / peak,
-                         "frac_of_nominal_8TBs": step_gbs / NOMINAL_HBM_GBS},
-            "roofline": {"bound": "hbm", "kernel": "center_pull", "achieved": achieved, "peak": peak,
-                         "peak_source": peak_src, "unit": "GB/s", "frac": achieved / peak,
-                         "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS, "traffic": center_pull_traffic(cfg),
-                         "traffic_source": "ncu dram bytes of a 14.9M-element capture at the same M, scaled by elements",
-                         "algorithmic_bytes_per_launch": pull_bytes, "kernel_ms": pull_ms,
-                         "timed_with": "library CUDA events around each kernel in a second K-step region",
-                         "other_kernels": {
-                             "sumsq": {"algorithmic_bytes_per_launch": sumsq_bytes, "kernel_ms": sumsq_ms,
-                                       "achieved": sumsq_bytes / (sumsq_ms * 1e-3) / 1e9,
-                                       "frac": sumsq_bytes / (sumsq_ms * 1e-3) / 1e9 / peak,
-                                       "traffic": sumsq_traffic(cfg)},
-                             "finalize": {"kernel_ms": fin_ms}},
-                         "ms_per_step_with_events": ms_k},
-            "e2e": {"value": whole_job_steps_per_s(world, e2e_ms_max), "unit": "steps/s", "steps": e2e_steps,
-                    "h2d_bytes_per_step": 2 * cfg.M * 4 * cfg.n, "d2h_bytes_per_step": (cfg.M + 1) * 4 * cfg.n,
-                    "entry_point": "grawa_step_host (pinned host buffers)"},
-            "other_variant": {"variant": other, "ms_per_step": other_ms, "steps_per_s": 1e3 / other_ms,
-                              "achieved_gbs": alg_bytes / (other_ms * 1e-3) / 1e9,
-                              "frac_of_measured_peak": alg_bytes / (other_ms * 1e-3) / 1e9 / peak,
-                              "frac_of_nominal_8TBs": alg_bytes / (other_ms * 1e-3) / 1e9 / NOMINAL_HBM_GBS},
+            "scaling": "weak", "vs_baseline": None, "dtype": dtype, "data": "synthetic",
+            "config": describe(cfg, variant, op, dtype, world),
+            "step_hbm": {k: step_rates[k] for k in ("achieved_gbs", "frac_of_measured_peak", "frac_of_nominal_8TBs")},
+            "roofline": roof,
             "gpu_launches": launches, "clocks": clocks, "last_step_status": status,
         }
-        if world == 1 and not args.no_cpu_baseline:
-            line["cpu_baseline"] = oracle_baseline(cfg, variant, [t.numpy() for t in hp], [t.numpy() for t in hg])
-        if world == 1 and args.also:
-            line["also"] = also_runs(grawa, args, exclude=(args.workload, variant))
+        if e2e_ms is not None:
+            line["e2e"] = {"value": whole_job_steps_per_s(world, e2e_ms_max), "unit": "steps/s", "steps": e2e_steps,
+                           "h2d_bytes_per_step": 2 * cfg.M * 4 * cfg.n, "d2h_bytes_per_step": (cfg.M + 1) * 4 * cfg.n,
+                           "entry_point": "grawa_step_host (pinned host buffers)"}
+        if other:
+            line["other_variant"] = other
+        if targets is not None:
+            line["targets"] = targets
+        if ops is not None:
+            line["ops"] = ops
+        if small is not None:
+            line["small"] = small
+        if sharded_out is not None:
+            line["sharded"] = sharded_out
+        if world == 1 and not args.no_cpu_baseline and op == "step":
+            line["cpu_baseline"], _ = oracle_timing(cfg, variant, hp_np, hg_np, budget_s=20.0)
         print(json.dumps(line), flush=True)
     if use_dist:
         dist.barrier()
         dist.destroy_process_group()
 
 
-def also_runs(grawa, args, exclude):
-    """Short secondary measurements of the other large workloads and variants (not the headline)."""
+def side_ops(grawa, cfg, variant, x, g, center, args, peak):
+    """Short runs of the other calls on the headline workload's buffers: the proximity step (runs every
+    local iteration), the step from given layer norms (no gradient pass) and the step on bfloat16 storage."""
+    import torch
+    steps = max(20, min(args.steps, 60))
+    out = []
+    ms, _, _ = Call(grawa, cfg, variant, "prox", "f32", x, g, center).time(steps, 3)
+    out.append(dict(op="prox", storage="f32", workload=cfg.name, steps=steps, algorithmic_bytes=op_bytes(cfg, "prox"),
+                    **rates(op_bytes(cfg, "prox"), ms, peak)))
+    c = Call(grawa, cfg, variant, "from_norms", "f32", x, g, center)
+    ms, _, _ = c.time(steps, 3)
+    _, _, ph = c.time(steps, 1, phases=True)
+    out.append(dict(op="from_norms", variant=variant, storage="f32", workload=cfg.name, steps=steps,
+                    algorithmic_bytes=op_bytes(cfg, "from_norms"), kernels=kernel_table(cfg, "f32", ph, peak, with_sumsq=False),
+                    **rates(op_bytes(cfg, "from_norms"), ms, peak)))
+    del c
+    c = Call(grawa, cfg, variant, "step", "bf16", x, g, center)
+    ms, _, _ = c.time(steps, 3)
+    _, _, ph = c.time(steps, 1, phases=True)
+    out.append(dict(op="step", variant=variant, storage="bf16", workload=cfg.name, steps=steps,
+                    algorithmic_bytes=op_bytes(cfg, "step", "bf16"), kernels=kernel_table(cfg, "bf16", ph, peak),
+                    **rates(op_bytes(cfg, "step", "bf16"), ms, peak)))
+    del c
+    torch.cuda.empty_cache()
+    return out
+
+
+def target_runs(grawa, args, peak, have=None):
+    """Every workload of at least 10 M parameters, MGRAWA and LGRAWA: at least 50 steps after 3 warm-up
+    steps, with the three kernels' times; buffers are freed between workloads."""
     import torch
     out = []
-    peak, _ = measured_peak_gbs()
-    for name in ("resnet18_imagenet", "vgg16", "vit_b16"):
+    steps = max(50, min(args.steps, 200))
+    for name in TARGET_WORKLOADS:
         cfg = gen.CONFIGS[name]
-        hp, hg = pinned_inputs(cfg)
-        x = [t.cuda() for t in hp]
-        g = [t.cuda() for t in hg]
-        center = torch.empty(cfg.n, device="cuda")
-        del hp, hg
+        if have is not None and have[0].name == name:
+            x, g = [t.cuda() for t in have[1]], [t.cuda() for t in have[2]]
+        else:
+            x, g = device_inputs(cfg)
+        center = torch.zeros(cfg.n, device="cuda")
         for variant in ("mgrawa", "lgrawa"):
-            if (name, variant) == exclude:
-                continue
-            steps = max(10, min(args.steps, 50))
-            ms, _, _ = time_device_steps(grawa, cfg, variant, x, g, center, steps, 3, False)
-            gbs = cfg.algorithmic_bytes() / (ms * 1e-3) / 1e9
-            out.append({"workload": name, "variant": variant, "M": cfg.M, "n": cfg.n, "steps": steps,
-                        "ms_per_step": ms, "steps_per_s": 1e3 / ms, "achieved_gbs": gbs,
-                        "frac_of_measured_peak": gbs / peak, "frac_of_nominal_8TBs": gbs / NOMINAL_HBM_GBS})
-        del x, g, center
+            c = Call(grawa, cfg, variant, "step", "f32", x, g, center)
+            ms, _, _ = c.time(steps, 3)
+            _, _, ph = c.time(steps, 1, phases=True)
+            out.append(dict(workload=name, variant=variant, M=cfg.M, n=cfg.n, n_layers=cfg.K, steps=steps,
+                            algorithmic_bytes=op_bytes(cfg, "step"), kernels=kernel_table(cfg, "f32", ph, peak),
+                            **rates(op_bytes(cfg, "step"), ms, peak)))
+            if name == "vgg16" and variant == "lgrawa":
+                cb = Call(grawa, cfg, variant, "step", "bf16", x, g, center)
+                ms, _, _ = cb.time(steps, 3)
+                out.append(dict(workload=name, variant=variant, storage="bf16", M=cfg.M, n=cfg.n, steps=steps,
+                                algorithmic_bytes=op_bytes(cfg, "step", "bf16"), **rates(op_bytes(cfg, "step", "bf16"), ms, peak)))
+                del cb
+        del c, x, g, center
         torch.cuda.empty_cache()
+    return out
+
+
+def small_runs(grawa, args):
+    """The two L2-resident workloads: launch-bound, no roofline target; eager calls and CUDA-graph replays."""
+    import torch
+    out = []
+    for name in SMALL_WORKLOADS:
+        cfg = gen.CONFIGS[name]
+        x, g = device_inputs(cfg)
+        center = torch.zeros(cfg.n, device="cuda")
+        off = cfg.offsets()
+        for variant in ("mgrawa", "lgrawa"):
+            c = Call(grawa, cfg, variant, "step", "f32", x, g, center)
+            eager_ms, _, _ = c.time(1000, 20)
+            stream = torch.cuda.Stream()
+            with torch.cuda.stream(stream):
+                c.fn()                                             # builds the plan for this stream
+                stream.synchronize()
+                graph = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph, stream=stream):
+                    c.fn()
+                for _ in range(20):
+                    graph.replay()
+                e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                e0.record()
+                for _ in range(1000):
+                    graph.replay()
+                e1.record()
+                stream.synchronize()
+            out.append({"workload": name, "variant": variant, "M": cfg.M, "n": cfg.n, "eager_us": eager_ms * 1e3,
+                        "graph_replay_us": e0.elapsed_time(e1), "traffic_time_us_at_8TBs": op_bytes(cfg, "step") / 8e12 * 1e6})
+            del graph
+        del x, g, center
+    return out
+
+
+def run_sharded(grawa, cfg, variant, args, world, rank, peak, barrier, x, g, center):
+    """ONE problem cut by element range over the ranks: local sums of squares, one all-gather of a [K, M]
+    table, the step from the gathered sums.  Strong scaling: the value is steps/s of that one problem."""
+    import torch
+    import torch.distributed as dist
+    from paper_2403_04206_b200 import sharded
+    own_group = False
+    if not dist.is_initialized():
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        os.environ.setdefault("MASTER_PORT", "29551")
+        dist.init_process_group("nccl", rank=0, world_size=1, device_id=torch.device("cuda", torch.cuda.current_device()))
+        own_group = True
+    j0, j1 = sharded.shard_range(cfg.n, world, rank)
+    loc = sharded.local_layer_table(cfg.offsets(), j0, j1)
+    xs, gs, cs = [t[j0:j1] for t in x], [t[j0:j1] for t in g], center[j0:j1]
+    fn = lambda: sharded.sharded_step(variant, xs, gs, cfg.pull, loc, cs)
+    steps = max(20, min(args.steps, 100))
+    for _ in range(3):
+        fn()
+    barrier()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    barrier()
+    ms = max_over_ranks([e0.elapsed_time(e1) / steps], world, "cuda")[0]
+    if own_group:
+        dist.destroy_process_group()
+    out = {"parallelism": "element-range sharded", "scaling": "strong", "n_gpus": world, "steps": steps,
+           "collective": "one all-gather of a [K, M] float64 table per step (NCCL)", "value": 1e3 / ms, "unit": "steps/s"}
+    out.update(rates(op_bytes(cfg, "step"), ms, peak * world))
     return out
 
 
@@ -396,46 +635,17 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    import oracle
     cfg = workload_config(args)
     variant = args.variant
-    off = cfg.offsets()
-    total = args.steps + args.warmup
-    budget = 150.0 / max(1, total)                      # whole run within a few minutes
-    # bounded sample: a prefix of layers, all workers, sized from a probe
-    probe_cfg = gen.custom_config([1 << 18], cfg.M, seed=cfg.seed)
-    pp, pg = gen.make_inputs(probe_cfg)
-    t0 = time.perf_counter()
-    _oracle_sample(oracle, variant, pp, pg, cfg.pull, probe_cfg.offsets())
-    per_elem = (time.perf_counter() - t0) / ((1 << 18) * cfg.M)
-    want = max(1, int(budget / (per_elem * cfg.M)))
-    k_hi = max(1, int(np.searchsorted(off, min(want, cfg.n), side="right")) - 1)
-    while k_hi < cfg.K and off[k_hi] == 0:
-        k_hi += 1
-    n_s = int(off[k_hi])
-    # generate only the sampled prefix: a custom workload with the same first layers and recipe
-    sizes = np.diff(off[:k_hi + 1])
-    sample_cfg = gen.custom_config(sizes, cfg.M, seed=cfg.seed, pull=cfg.pull, grad_recipe=cfg.grad_recipe,
-                                   log10_sigma=cfg.log10_sigma, loud_worker_factor=cfg.loud_worker_factor)
-    p_full, g_full = gen.make_inputs(sample_cfg)
-    soff = off[:k_hi + 1]
-    times = []
-    for i in range(total):
-        t0 = time.perf_counter()
-        _oracle_sample(oracle, variant, p_full, g_full, cfg.pull, soff)
-        if i >= args.warmup:
-            times.append(time.perf_counter() - t0)
-    sec = float(np.mean(times)) * cfg.n / n_s
+    p, g = gen.make_inputs(cfg)
+    base, sec = oracle_timing(cfg, variant, p, g, budget_s=150.0, steps_wanted=max(1, args.steps), warmup=max(0, args.warmup))
     value = 1.0 / sec
-    sample = (f"each step = the first {k_hi} of {cfg.K} layers ({n_s} of {cfg.n} elements, all {cfg.M} workers), "
-              f"scaled by elements to a full step")
+    base = {k: base[k] for k in ("value", "unit", "cores", "kind", "sample", "whole_steps")}
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": 1,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": {"workload": f"{cfg.name} layer table, M={cfg.M} workers, n={cfg.n}, K={cfg.K} layers, "
-                                   f"{variant.upper()} step, pull={cfg.pull}, seed={cfg.seed}",
-                       "variant": variant, "M": cfg.M, "n": cfg.n, "n_layers": cfg.K},
-            "cpu_baseline": {"value": value, "unit": "steps/s", "cores": 1, "kind": "oracle", "sample": sample},
+            "config": describe(cfg, variant, "step", "f32", 1),
+            "cpu_baseline": base,
             "e2e": {"value": value, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
 
@@ -443,13 +653,16 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=400)
+    ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", default="cuda", choices=["cuda", "reference"])
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD, choices=list(gen.CONFIGS))
     ap.add_argument("--variant", default=DEFAULT_VARIANT, choices=["lgrawa", "mgrawa", "grawa"])
+    ap.add_argument("--op", default="step", choices=["step", "prox", "from_norms"])
+    ap.add_argument("--dtype", default="f32", choices=["f32", "bf16", "f16"], help="storage of parameters, gradients and centre")
+    ap.add_argument("--sharded", action="store_true", help="also time one problem cut by element range over the ranks")
     ap.add_argument("--e2e-steps", type=int, default=3)
-    ap.add_argument("--also", action="store_true", help="add short runs of the other large workloads/variants")
+    ap.add_argument("--headline-only", action="store_true", help="skip the short runs of the other workloads and calls")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers-limit", type=int, default=0, help="use only the first L layers (small profiling captures)")
     ap.add_argument("--option", action="append", default=[], help="library tuning knob, name=value (repeatable)")

@@ -344,8 +344,14 @@ finalize_kernel(StepScratch sc)
     trace.go();
 
     const unsigned long long* bins = sc.bins;
-    if (sc.given == nullptr && blockIdx.x == 0 && tid == 0) *sc.next_buf = __ldcg(sc.next_buf) ^ 1;
-    if (blockIdx.x == 0 && tid == 0) *sc.work_counter = 0u;
+    // the first thread turns the copies of the digit rows over; the load is issued now, the store
+    // at the very end, so that nothing waits for it
+    const bool keeper = blockIdx.x == 0 && tid == 0;
+    int next = 0;
+    if (keeper) {
+        *sc.work_counter = 0u;
+        if (sc.given == nullptr) next = __ldcg(sc.next_buf) ^ 1;
+    }
 
     if (sc.variant == kLgrawa) {
         int any_flag = 0;
@@ -390,6 +396,7 @@ finalize_kernel(StepScratch sc)
                 if (sc.status_copy) atomicOr(sc.status_copy, kStatusNonFinite);
             }
         }
+        if (keeper && sc.given == nullptr) *sc.next_buf = next;
         trace.done();
         return;
     }
@@ -439,6 +446,7 @@ finalize_kernel(StepScratch sc)
             if (sc.status_copy) *sc.status_copy = flagged ? kStatusNonFinite : 0;
         }
     }
+    if (keeper && sc.given == nullptr) *sc.next_buf = next;
     trace.done();
 }
 
@@ -462,8 +470,12 @@ sumsq_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
     KernelTrace trace(0);
     grid_dependency_sync();
     trace.go();
-    const int buf = __ldcg(sc.next_buf);
-    unsigned long long* bins = sc.bins + static_cast<size_t>(buf) * bins_copy_words(sc);
+    // Which copy of the digit rows to add into: needed only by thread 0 when an item is done, and by
+    // everybody after the last item; thread 0 fetches it now and hands it on through shared memory,
+    // so that no thread waits for it in front of its gradient loads.
+    __shared__ int buf_sm;
+    int buf = 0;
+    if (tid == 0) buf = __ldcg(sc.next_buf);
 
     int parity = 0;
     for (int item = blockIdx.x; item < items; item += gridDim.x, parity ^= 1) {
@@ -510,15 +522,17 @@ sumsq_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) dacc += __shfl_down_sync(0xffffffffu, dacc, d);
         if (lane == 0) warp_part[parity][warp] = dacc;
+        if (tid == 0) buf_sm = buf;
         __syncthreads();
         if (tid == 0) {
             double total = 0.0;
 #pragma unroll
             for (int w = 0; w < kThreads / 32; ++w) total += warp_part[parity][w];
+            unsigned long long* bins = sc.bins + static_cast<size_t>(buf) * bins_copy_words(sc);
             bins_add(bins + static_cast<size_t>(sg.layer) * sc.M + m, static_cast<size_t>(sc.K) * sc.M, total);
         }
     }
-    bins_turnover(sc, buf);
+    bins_turnover(sc, buf_sm);           // every CTA has had at least one item, hence one barrier after the write
     trace.done();
 }
 

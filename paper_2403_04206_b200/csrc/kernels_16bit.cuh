@@ -83,8 +83,12 @@ sumsq16_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
     Segment first_sg = Segment{0, 0, 0};
     if (static_cast<int>(blockIdx.x) < items) first_sg = sc.segs[blockIdx.x % C];
     grid_dependency_sync();
-    const int buf = __ldcg(sc.next_buf);
-    unsigned long long* bins = sc.bins + static_cast<size_t>(buf) * bins_copy_words(sc);
+    // Which copy of the digit rows to add into: needed only by thread 0 when an item is done, and by
+    // everybody after the last item; thread 0 fetches it now and hands it on through shared memory,
+    // so that no thread waits for it in front of its gradient loads.
+    __shared__ int buf_sm;
+    int buf = 0;
+    if (tid == 0) buf = __ldcg(sc.next_buf);
 
     int parity = 0;
     for (int item = blockIdx.x; item < items; item += gridDim.x, parity ^= 1) {
@@ -130,15 +134,17 @@ sumsq16_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
 #pragma unroll
         for (int d = 16; d > 0; d >>= 1) dacc += __shfl_down_sync(0xffffffffu, dacc, d);
         if (lane == 0) warp_part[parity][warp] = dacc;
+        if (tid == 0) buf_sm = buf;
         __syncthreads();
         if (tid == 0) {
             double total = 0.0;
 #pragma unroll
             for (int w = 0; w < kThreads / 32; ++w) total += warp_part[parity][w];
+            unsigned long long* bins = sc.bins + static_cast<size_t>(buf) * bins_copy_words(sc);
             bins_add(bins + static_cast<size_t>(sg.layer) * sc.M + m, static_cast<size_t>(sc.K) * sc.M, total);
         }
     }
-    bins_turnover(sc, buf);
+    bins_turnover(sc, buf_sm);           // every CTA has had at least one item, hence one barrier after the write
 }
 
 // Shape of the 16-bit centre+pull kernel: columns of WORDS 32-bit words (two elements each) kept

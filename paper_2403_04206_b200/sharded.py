@@ -33,20 +33,49 @@ def local_layer_table(layer_offsets, j0: int, j1: int) -> np.ndarray:
     return np.clip(off, j0, j1) - j0
 
 
+def exchange_layer_sums(local, group=None):
+    """The one exchange of the sharded step: all-gather of every rank's [K, M] table of local sums of
+    squares (float64).  Returns the tables of all ranks in rank order, shape [world, K, M], on the
+    device of ``local``.  Works with any torch.distributed backend (NCCL on GPUs, gloo on CPU); on
+    a GPU the collective is ordered against torch's current stream."""
+    import torch
+    import torch.distributed as dist
+
+    world = dist.get_world_size(group)
+    K, M = local.shape
+    gathered = torch.empty(world * K, M, dtype=local.dtype, device=local.device)      # rank-major
+    dist.all_gather_into_tensor(gathered, local.contiguous(), group=group)
+    return gathered.view(world, K, M)
+
+
+def _stream_context(stream):
+    """Makes ``stream`` (None, a torch.cuda.Stream or a raw cudaStream_t) torch's current stream, so
+    that allocations, the library's kernels and the collective are all ordered on it."""
+    import contextlib
+
+    import torch
+    if stream is None:
+        return contextlib.nullcontext()
+    if not isinstance(stream, torch.cuda.Stream):
+        stream = torch.cuda.ExternalStream(int(stream))
+    return torch.cuda.stream(stream)
+
+
 def sharded_step(variant, params, grads, pull, local_offsets, center_out=None, *, group=None, stream=None):
     """One averaging step on this rank's element range.
 
     params, grads: this rank's slices of the M replicas (device float32 tensors of j1-j0 elements);
     local_offsets: local_layer_table(...) of the range.  Collective: every rank of `group` must call it.
+    Everything (the two library calls and the all-gather between them) is enqueued on ``stream``
+    (default: torch's current stream).
     """
     import torch
     import torch.distributed as dist
 
     world = dist.get_world_size(group)
     K, M = len(local_offsets) - 1, len(params)
-    device = params[0].device
-    local = torch.empty(K, M, dtype=torch.float64, device=device)
-    binding.grawa_layer_sumsq(grads, local_offsets, local, stream=stream)
-    gathered = torch.empty(world * K, M, dtype=torch.float64, device=device)      # rank-major: [world][K][M]
-    dist.all_gather_into_tensor(gathered, local, group=group)
-    binding.grawa_step_from_layer_sums(variant, params, gathered, world, pull, local_offsets, center_out, stream=stream)
+    with _stream_context(stream):
+        local = torch.empty(K, M, dtype=torch.float64, device=params[0].device)
+        binding.grawa_layer_sumsq(grads, local_offsets, local)
+        gathered = exchange_layer_sums(local, group)
+        binding.grawa_step_from_layer_sums(variant, params, gathered, world, pull, local_offsets, center_out)

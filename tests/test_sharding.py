@@ -50,11 +50,11 @@ def _gloo_worker(rank, world, port, out):
     off = cfg.offsets()
     j0, j1 = sharded.shard_range(cfg.n, world, rank)
     loc = sharded.local_layer_table(off, j0, j1)
-    # the exchange of the sharded step, with the oracle standing in for the kernels
+    # the exchange of the sharded step (the function sharded_step itself calls), with the oracle
+    # standing in for the kernels on either side of it
     local = torch.from_numpy(oracle.sumsq([a[j0:j1] for a in g], loc))
-    gathered = torch.empty(world * local.shape[0], local.shape[1], dtype=torch.float64)
-    dist.all_gather_into_tensor(gathered, local)
-    gathered = gathered.view(world, *local.shape)
+    gathered = sharded.exchange_layer_sums(local)
+    assert gathered.shape == (world, *local.shape) and bool((gathered[rank] == local).all())
     S = gathered[0].numpy().copy()
     for r in range(1, world):
         S += gathered[r].numpy()
@@ -142,5 +142,25 @@ def test_sharded_step_through_nccl_with_one_rank():
         assert np.abs(centre.cpu().numpy() - ref["center"]).max() <= tol
         for m in range(cfg.M):
             assert np.abs(x[m].cpu().numpy() - ref["workers"][m]).max() <= tol
+        # On a stream that is not the current one, behind work that produces the inputs there: the
+        # step (kernels and all-gather) must queue up behind that work, not beside it.
+        side = torch.cuda.Stream()
+        x2 = [torch.empty(cfg.n, device="cuda") for _ in p]
+        g2 = [torch.empty(cfg.n, device="cuda") for _ in g]
+        centre2 = torch.empty(cfg.n, device="cuda")
+        big = torch.empty(1 << 28, device="cuda")
+        hp = [torch.from_numpy(a).cuda() for a in p]
+        hg = [torch.from_numpy(a).cuda() for a in g]
+        torch.cuda.synchronize()
+        with torch.cuda.stream(side):
+            for _ in range(4):
+                big.mul_(1.0001)                      # keeps `side` busy while the host runs ahead
+            for dst, src in zip(x2 + g2, hp + hg):
+                dst.copy_(src)
+        sharded.sharded_step("lgrawa", x2, g2, 0.5, sharded.local_layer_table(off, j0, j1), centre2, stream=side)
+        side.synchronize()
+        assert bool((centre2 == centre).all())
+        for u, v in zip(x2, x):
+            assert bool((u == v).all())
     finally:
         dist.destroy_process_group()
