@@ -32,6 +32,8 @@ static int64_t g_bulk_tile = 0;           // 0 = chosen from M so that at least 
 static int64_t g_kernel_timing = 0;
 static int64_t g_pdl = 1;
 static int64_t g_pull_preload = 1;
+static int64_t g_pull_prefetch_waves = 3;
+static int64_t g_sumsq_prefetch_waves = 1;
 static int64_t g_sumsq_ctas_per_sm = 0;   // 0 = one CTA per work item
 static int64_t g_pull_ctas_per_sm = 0;    // 0 = one CTA per work item
 static thread_local std::string t_cuda_error;
@@ -308,13 +310,13 @@ struct CenterPullBulkDispatch<1> {
 template <int M>
 static cudaError_t launch_center_pull(bool per_layer, int grid, int item_begin, int item_end, cudaStream_t stream, bool pdl,
                                       const MutPtrs& x, float* center, const float* beta, const Segment* segs, long long n, int tile,
-                                      float pull, int preload)
+                                      float pull, int preload, int prefetch_stride, int prefetch_waves)
 {
     if (per_layer)
         return launch_kernel(center_pull_kernel<M, true>, grid, kThreads, stream, pdl, x, center, beta, segs, item_begin, item_end, n,
-                             tile, pull, 1, preload);
+                             tile, pull, 1, preload, prefetch_stride, prefetch_waves);
     return launch_kernel(center_pull_kernel<M, false>, grid, kThreads, stream, pdl, x, center, beta, segs, item_begin, item_end, n, tile,
-                         pull, 1, preload);
+                         pull, 1, preload, prefetch_stride, prefetch_waves);
 }
 
 template <int M>
@@ -423,6 +425,7 @@ static grawa_status make_context(int variant, float* const* params, const float*
     StepScratch& sc = ctx->sc;
     sc.segs = plan->d_segs1;
     sc.C = plan->C1; sc.K = K; sc.M = M; sc.variant = variant; sc.n = n;
+    sc.prefetch_stride = 0; sc.prefetch_waves = 0;
     sc.bins = reinterpret_cast<unsigned long long*>(ws + plan->ws.bins);
     sc.next_buf = reinterpret_cast<int*>(ws + plan->ws.words);
     sc.S = reinterpret_cast<double*>(ws + plan->ws.S);
@@ -476,6 +479,8 @@ static grawa_status enqueue_weights_launches(StepContext& c)
     const int grid1 = g_sumsq_ctas_per_sm > 0
                           ? static_cast<int>(std::min<int64_t>(items1, g_sumsq_ctas_per_sm * plan->sm_count)) : items1;
     const int vg = c.vec_g ? 1 : 0;
+    c.sc.prefetch_stride = 6 * plan->sm_count;           // CTAs resident at the start of the kernel
+    c.sc.prefetch_waves = (c.dtype == 0 && grid1 <= 64 * c.sc.prefetch_stride) ? static_cast<int>(g_sumsq_prefetch_waves) : 0;
     if (c.dtype == 1)
         GRAWA_CUDA_TRY(launch_kernel(sumsq16_kernel<__nv_bfloat16, 8>, grid1, kThreads, c.stream, c.pdl, c.gp, c.sc, items1, vg));
     else if (c.dtype == 2)
@@ -534,11 +539,15 @@ static grawa_status enqueue_center_pull(StepContext& c, int item_begin, int item
                                                                    stage_bytes * stages, c.stream, c.pdl, c.xp, c.center, beta,
                                                                    plan->d_segs2, c.n, tile, stages, M, c.pull, c.counter, c.status));
     } else if (c.vec_x && M <= kMaxRegWorkers) {
+        // L2 prefetch of later items during the weights' finalisation: pays on short steps only (a few
+        // dozen waves of CTAs); on long ones the window it fills is negligible and the hint costs a little
+        const int stride = 2 * plan->sm_count;
+        const int waves = (grid <= 64 * stride) ? static_cast<int>(g_pull_prefetch_waves) : 0;
         const int grid2 = g_pull_ctas_per_sm > 0
                               ? static_cast<int>(std::min<int64_t>(grid, g_pull_ctas_per_sm * plan->sm_count)) : grid;
         GRAWA_CUDA_TRY(CenterPullDispatch<kMaxRegWorkers>::run(M, per_layer, grid2, item_begin, item_end, c.stream, c.pdl, c.xp,
                                                                c.center, beta, plan->d_segs2, c.n, tile, c.pull,
-                                                               (c.preload && g_pull_preload) ? 1 : 0));
+                                                               (c.preload && g_pull_preload) ? 1 : 0, stride, waves));
     } else {
         GRAWA_CUDA_TRY(launch_kernel(center_pull_generic_kernel, grid, kThreads, c.stream, c.pdl, c.xp, c.center, beta, plan->d_segs2,
                                      per_layer ? 1 : 0, item_begin, c.n, tile, c.pull, M));
@@ -1096,6 +1105,11 @@ grawa_status grawa_set_option(const char* name, int64_t value)
         g_pdl = value;
         return GRAWA_OK;
     }
+    if (std::strcmp(name, "pull_prefetch_waves") == 0 || std::strcmp(name, "sumsq_prefetch_waves") == 0) {
+        if (value < 0 || value > 8) return GRAWA_ERR_INVALID_ARG;
+        (name[0] == 'p' ? g_pull_prefetch_waves : g_sumsq_prefetch_waves) = value;
+        return GRAWA_OK;
+    }
     if (std::strcmp(name, "pull_preload") == 0) {
         if (value < 0 || value > 1) return GRAWA_ERR_INVALID_ARG;
         g_pull_preload = value;
@@ -1120,6 +1134,8 @@ int64_t grawa_get_option(const char* name)
     if (std::strcmp(name, "kernel_timing") == 0) return g_kernel_timing;
     if (std::strcmp(name, "dependent_launch") == 0) return g_pdl;
     if (std::strcmp(name, "pull_preload") == 0) return g_pull_preload;
+    if (std::strcmp(name, "pull_prefetch_waves") == 0) return g_pull_prefetch_waves;
+    if (std::strcmp(name, "sumsq_prefetch_waves") == 0) return g_sumsq_prefetch_waves;
     if (std::strcmp(name, "sumsq_ctas_per_sm") == 0) return g_sumsq_ctas_per_sm;
     if (std::strcmp(name, "pull_ctas_per_sm") == 0) return g_pull_ctas_per_sm;
     return -1;

@@ -118,6 +118,13 @@ __device__ __forceinline__ float ld_stream1(const float* p) { return __ldcs(p); 
 __device__ __forceinline__ void st_stream4(float4* p, float4 v) { __stcs(p, v); }
 __device__ __forceinline__ void st_stream1(float* p, float v) { __stcs(p, v); }
 
+// Hint: bring `bytes` (a multiple of 16) from the 16-byte aligned address p into L2.  No architectural
+// effect; L2 is the GPU's point of coherence, so a prefetched line can never be stale.
+__device__ __forceinline__ void prefetch_l2(const void* p, unsigned bytes)
+{
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(p), "r"(bytes) : "memory");
+}
+
 // Splits [b, e) into scalar head [b, hb), 16-byte aligned body [hb, te), scalar tail [te, e).
 // With vec_ok == 0 (a base pointer that is not 16-byte aligned) everything is head.
 __device__ __forceinline__ void split_range(long long b, long long e, int vec_ok, long long& hb, long long& te)
@@ -226,6 +233,7 @@ struct StepScratch {
     const Segment* segs;           // sum-of-squares work items of one worker, C of them
     int C, K, M, variant;
     long long n;                   // elements per worker (bounds checks of the debug build)
+    int prefetch_stride, prefetch_waves;   // sum-of-squares kernel: L2 prefetch of later items by the first CTAs (0 = none)
     unsigned long long* bins;      // [2][kRowWords][K][M]
     int* next_buf;                 // copy the next sum-of-squares kernel adds into
     double* S;                     // [K][M]
@@ -459,7 +467,7 @@ finalize_kernel(StepScratch sc)
 // Six CTAs per SM (at most 42 registers): measured 1.4x faster than four on the large workloads.
 template <int UNROLL>
 __global__ void __launch_bounds__(kThreads, 6)
-sumsq_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
+sumsq_kernel(const __grid_constant__ ConstPtrs grads, StepScratch sc, int items, int vec_ok)
 {
     __shared__ double warp_part[2][kThreads / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -467,6 +475,20 @@ sumsq_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
     // the work list belongs to the plan, not to the kernel before this one: fetch the first item early
     Segment first_sg = Segment{0, 0, 0};
     if (static_cast<int>(blockIdx.x) < items) first_sg = sc.segs[blockIdx.x % C];
+    // On short problems the CTAs that are resident when the kernel starts ask for the gradients of
+    // the items one, two, ... grid-fuls further on to be brought into L2 while they wait for the
+    // kernel in front (whose tail leaves DRAM partly idle).  Hints only; see prefetch_l2.
+    if (static_cast<int>(blockIdx.x) < sc.prefetch_stride && tid < sc.prefetch_waves) {
+        const long long it = blockIdx.x + static_cast<long long>(tid + 1) * sc.prefetch_stride;
+        if (it < items) {
+            const int pm = static_cast<int>(it / C);
+            const Segment sg = sc.segs[it - static_cast<long long>(pm) * C];
+            long long phb, pte;
+            split_range(sg.begin, sg.begin + sg.len, vec_ok, phb, pte);
+            const unsigned bytes = static_cast<unsigned>(pte - phb) * 4u;
+            if (bytes > 0 && in_bounds(phb, pte - phb, sc.n)) prefetch_l2(grads.p[pm] + phb, bytes);
+        }
+    }
     KernelTrace trace(0);
     grid_dependency_sync();
     trace.go();
@@ -583,11 +605,17 @@ template <> struct VecIO<2> {
 // front of this one on the stream are this library's own sum-of-squares / finalisation kernels
 // (they pass their own dependency wait before they let this kernel start, so whatever the caller
 // ran earlier has completed by then).
+//
+// With `prefetch_waves` > 0 the first `prefetch_stride` CTAs (the ones resident when the kernel
+// starts) also ask, before the wait, for the parameters of the items `prefetch_stride`,
+// 2 * `prefetch_stride`, ... further on to be brought into L2: while the weights are being finalised
+// DRAM has nothing else to do, and the CTAs that take those items later find them in L2.  A
+// prefetch is a hint without architectural effect, and L2 is the GPU's point of coherence.
 template <int M, bool PER_LAYER>
 __global__ void __launch_bounds__(kThreads, 2)
 center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restrict__ beta,
                    const Segment* __restrict__ segs, int item_begin, int item_end, long long n, int tile, float lambda,
-                   int vec_ok, int preload)
+                   int vec_ok, int preload, int prefetch_stride, int prefetch_waves)
 {
     constexpr int COLS = pull_cols(M);
     constexpr int VEC = pull_vec(M);
@@ -624,6 +652,29 @@ center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restric
     if (item < item_end) {
         locate(item);
         if (preload) {
+            // (not compiled in for M > 8, where the kernel has no registers to spare and problems are large)
+            if (M <= 8 && static_cast<int>(blockIdx.x) < prefetch_stride && tid < M * prefetch_waves) {
+                const int m = tid % M;
+                const long long it = item + static_cast<long long>(tid / M + 1) * prefetch_stride;
+                if (it < item_end) {
+                    long long pb, pe, phb, pte;
+                    if (PER_LAYER) {
+                        const Segment sg = segs[it];
+                        pb = sg.begin;
+                        pe = pb + sg.len;
+                    } else {
+                        pb = it * tile;
+                        pe = min(n, pb + tile);
+                    }
+                    split_range(pb, pe, vec_ok, phb, pte);
+                    const unsigned bytes = static_cast<unsigned>(pte - phb) * 4u;       // a multiple of 16
+                    const float* base = x.p[0];
+#pragma unroll
+                    for (int mm = 1; mm < M; ++mm)
+                        if (mm == m) base = x.p[mm];                // a select chain: no run-time index into the pointer table
+                    if (bytes > 0 && in_bounds(phb, pte - phb, n)) prefetch_l2(base + phb, bytes);
+                }
+            }
             load_chunk(0);
             loaded = true;
         }
