@@ -28,10 +28,15 @@
  *     returns without synchronising.  The first call with a new (device, stream, n, M, layer
  *     table) builds and caches a plan (device allocations and a small upload); later calls
  *     allocate nothing.
- *   - Arithmetic: fp32 loads; sums of squares accumulated in short fp32 runs combined in fp64
- *     in a fixed order (bitwise reproducible run to run); scores and weights in fp64, rounded
- *     once to fp32; centre as an fp32 fused-multiply-add chain over m = 0..M-1; pull as
- *     fmaf(pull, x_C, (1-pull) * x_m).
+ *   - Arithmetic: fp32 loads; squares accumulated in short fp32 runs, the runs of a work item
+ *     combined in fp64 in a fixed order, the items' sums added exactly as fixed-point integers
+ *     (so S does not depend on the order in which items finish: bitwise reproducible run to
+ *     run); scores and weights in fp64, rounded once to fp32; centre as an fp32
+ *     fused-multiply-add chain over m = 0..M-1; pull as fmaf(pull, x_C, (1-pull) * x_m).
+ *   - Supported gradient magnitudes: the squares are taken in fp32, so |g| below about 1e-19
+ *     contributes zero (a layer of only such values scores exactly 0 and takes the zero-score
+ *     rule below) and |g| above about 1.8e19 squares to infinity (a non-finite score, rule
+ *     below).  Between those bounds the weights meet the 1e-5 relative contract.
  *   - Scores that are exactly zero take the limit of 1/A: inside a normalisation group the Z
  *     workers with zero score get 1/Z each, all others 0.  A non-finite score (NaN/Inf
  *     gradients) gives that worker weight 0, the rest are normalised among themselves (uniform
@@ -77,6 +82,10 @@ typedef struct grawa_options {
     double *sumsq_out;     /* DEVICE, fp64: S, [n_layers][M] (one row when there is no layer table) */
     void   *workspace;     /* DEVICE scratch, 256-byte aligned; NULL = the cached plan owns one     */
     size_t  workspace_bytes; /* size of `workspace`; at least grawa_workspace_bytes(...)            */
+    int    *status_word;   /* DEVICE int, or NULL: receives the step's status bits (0 = clean, bit 0 = a
+                              non-finite score met the fallback of step 3) when the weights are
+                              finalised, so that a caller who replays a captured step can poll it
+                              without the host-synchronising grawa_last_step_status                 */
 } grawa_options;
 
 /* Library version, major*10000 + minor*100 + patch. */
@@ -88,10 +97,11 @@ const char *grawa_status_string(grawa_status status);
 /* Text of the last CUDA error seen by the calling thread ("" if none). */
 const char *grawa_last_cuda_error(void);
 
-/* Bytes of device scratch a step needs for this problem (partial sums, S, A, beta, status), for
- * any storage type (16-bit storage needs no more than fp32).  layer_offsets may be NULL with
- * n_layers = 0 (one layer).  Returns 0 on invalid arguments.  The value depends on the
- * "sumsq_tile" option in force. */
+/* Bytes of device scratch a step needs for this problem (the exact sums, S, A, beta, status): per
+ * (layer, worker) tables only, the same for every storage type and vector length.  layer_offsets
+ * may be NULL with n_layers = 0 (one layer).  Returns 0 on invalid arguments.  A caller's
+ * workspace needs no particular contents: every step that uses it clears the part that has to
+ * start from zero (one small memset in front of the kernels). */
 size_t grawa_workspace_bytes(int64_t n, int M, const int64_t *layer_offsets, int n_layers);
 
 /* MGRAWA step (Eq. 3-4, then centre and pull): one weight per worker from the sum of its
@@ -202,6 +212,46 @@ grawa_status grawa_step_from_layer_sums(grawa_variant variant, float *const *par
                                         int n_layers, float *center_out, const grawa_options *options,
                                         grawa_stream_t stream);
 
+/* The other entry points on 16-bit storage.  Each `_typed` call is the call of the same name above with
+ * parameters, gradients and centre stored in `dtype` (GRAWA_F32 gives exactly that call); pointers to
+ * them are untyped, aligned to the element size, and every stored result is rounded to nearest-even
+ * once, as in grawa_step_typed.  Tables of norms, sums of squares, scores and weights keep their
+ * types (fp64 / fp32).  Together they let a caller who keeps bfloat16 or half replicas run
+ * Algorithm 1 / 2 end to end: the proximity step of every local iteration, the Local variants of
+ * the appendix and the element-range sharded step.
+ *
+ * grawa_prox_step_typed: the "Prox." update of Algorithms 1 and 2; mu_over_tau = 0 leaves the workers'
+ * bits untouched, mu_over_tau = 1 makes them bit-equal to `center`. */
+grawa_status grawa_prox_step_typed(grawa_dtype dtype, void *const *params, const void *center, int64_t n, int M,
+                                   float mu_over_tau, grawa_stream_t stream);
+
+/* grawa_layer_norms_typed / grawa_layer_sumsq_typed: per-layer norms of one gradient, per-layer sums of
+ * squares of M gradients, from 16-bit gradients (widened exactly to fp32 before squaring). */
+grawa_status grawa_layer_norms_typed(grawa_dtype dtype, const void *grad, int64_t n, const int64_t *layer_offsets,
+                                     int n_layers, double *norms_out, grawa_stream_t stream);
+grawa_status grawa_layer_sumsq_typed(grawa_dtype dtype, const void *const *grads, int64_t n, int M,
+                                     const int64_t *layer_offsets, int n_layers, double *sumsq_out,
+                                     grawa_stream_t stream);
+
+/* grawa_step_from_layer_norms_typed / grawa_step_from_layer_sums_typed: the averaging step from given
+ * scores (appendix algorithm of the Local variants; sums of squares added over element-range shards,
+ * Eq. 3 / Eq. 5) on parameters and centre of `dtype`. */
+grawa_status grawa_step_from_layer_norms_typed(grawa_dtype dtype, grawa_variant variant, void *const *params,
+                                               const double *layer_norms, int64_t n, int M, float pull,
+                                               const int64_t *layer_offsets, int n_layers, void *center_out,
+                                               const grawa_options *options, grawa_stream_t stream);
+grawa_status grawa_step_from_layer_sums_typed(grawa_dtype dtype, grawa_variant variant, void *const *params,
+                                              const double *layer_sums, int parts, int64_t n, int M, float pull,
+                                              const int64_t *layer_offsets, int n_layers, void *center_out,
+                                              const grawa_options *options, grawa_stream_t stream);
+
+/* grawa_step_host_typed: grawa_step_host with HOST buffers of `dtype` (Eq. 2-7, centre, pull); the
+ * device staging buffers take (2M+1)*n elements of `dtype`. */
+grawa_status grawa_step_host_typed(grawa_dtype dtype, grawa_variant variant, void *const *params,
+                                   const void *const *grads, int64_t n, int M, float pull,
+                                   const int64_t *layer_offsets, int n_layers, void *center_out,
+                                   grawa_stream_t stream);
+
 /* Largest number of partial sums grawa_sumsq_static can hold: M * ceil(n / 16384) must not
  * exceed it (for example M = 16 workers of up to 134 million elements each). */
 #define GRAWA_STATIC_MAX_PARTIALS 131072
@@ -243,12 +293,13 @@ grawa_status grawa_sumsq_static(const float *const *grads, int64_t n, int M, dou
  * GRAWA_ERR_TIMEOUT with the context still usable.  Touches no caller memory. */
 grawa_status grawa_selftest_bounded_wait(int64_t limit_ns, grawa_stream_t stream);
 
-/* Debug build only (the library compiled with -DGRAWA_DEBUG_BOUNDS, which checks every global access
- * of the streaming kernels against the vector length, counts violations and skips them): returns
- * the number of violations on the current device since the last call and resets it; synchronises
- * the device.  With selfcheck != 0 it first feeds the checker three out-of-range index triples
- * (arithmetic only, no memory access), so a healthy debug build returns exactly 3 more.
- * Returns -1 in the normal build, -2 on a CUDA error. */
+/* Debug build only (the library compiled with -DGRAWA_DEBUG_BOUNDS, in which every global access of
+ * the streaming kernels is first checked against the work item it belongs to and the vector, and
+ * every index into scratch memory against its table; violations are counted and the access
+ * skipped): returns the number of violations on the current device since the last call and resets
+ * it; synchronises the device.  With selfcheck != 0 it first feeds the checker seven planted
+ * violations and two clean probes (arithmetic only, no memory access), so a healthy debug build
+ * returns exactly 7 more.  Returns -1 in the normal build, -2 on a CUDA error. */
 int64_t grawa_debug_bounds_violations(int selfcheck);
 
 /* Trace build only (the library compiled with -DGRAWA_TRACE): the sum-of-squares, finalisation and
@@ -280,6 +331,11 @@ int grawa_trace_read(uint64_t *rows_out, int max_rows);
  *                  stream serialisation, so each one's launch overlaps the tail of the one
  *                  before it on the stream (it still waits for that kernel's results);
  *                  0 = plain stream order.
+ *   "pull_preload"  1 (default) = a device-buffer step's centre+pull kernel loads its first
+ *                  parameters ahead of its wait for the weights; 0 = after it.
+ *   "pull_prefetch_waves", "sumsq_prefetch_waves" (0..8; defaults 3 and 1) on short steps the CTAs
+ *                  that are resident when a kernel starts hint the data of the items that many
+ *                  grid-fuls further on into L2 while they wait for the kernel in front; 0 = off.
  *   "sumsq_ctas_per_sm", "pull_ctas_per_sm" (0..32) CTAs per SM of the grid that streams
  *                  through the work items of the sum-of-squares / centre+pull kernel;
  *                  0 = one CTA per work item.

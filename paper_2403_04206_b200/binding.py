@@ -30,7 +30,7 @@ class GrawaError(RuntimeError):
 
 class _Options(ctypes.Structure):
     _fields_ = [("weights_out", ctypes.c_void_p), ("scores_out", ctypes.c_void_p), ("sumsq_out", ctypes.c_void_p),
-                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
+                ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t), ("status_word", ctypes.c_void_p)]
 
 
 _lib = None
@@ -81,6 +81,18 @@ def library() -> ctypes.CDLL:
     lib.grawa_layer_sumsq.restype = ci
     lib.grawa_step_from_layer_sums.argtypes = [ci, vp, vp, ci, i64, ci, cf, vp, ci, vp, vp, vp]
     lib.grawa_step_from_layer_sums.restype = ci
+    lib.grawa_prox_step_typed.argtypes = [ci, vp, vp, i64, ci, cf, vp]
+    lib.grawa_prox_step_typed.restype = ci
+    lib.grawa_layer_norms_typed.argtypes = [ci, vp, i64, vp, ci, vp, vp]
+    lib.grawa_layer_norms_typed.restype = ci
+    lib.grawa_layer_sumsq_typed.argtypes = [ci, vp, i64, ci, vp, ci, vp, vp]
+    lib.grawa_layer_sumsq_typed.restype = ci
+    lib.grawa_step_from_layer_norms_typed.argtypes = [ci, ci, vp, vp, i64, ci, cf, vp, ci, vp, vp, vp]
+    lib.grawa_step_from_layer_norms_typed.restype = ci
+    lib.grawa_step_from_layer_sums_typed.argtypes = [ci, ci, vp, vp, ci, i64, ci, cf, vp, ci, vp, vp, vp]
+    lib.grawa_step_from_layer_sums_typed.restype = ci
+    lib.grawa_step_host_typed.argtypes = [ci, ci, vp, vp, i64, ci, cf, vp, ci, vp, vp]
+    lib.grawa_step_host_typed.restype = ci
     lib.grawa_sumsq_static.argtypes = [vp, i64, ci, vp, vp]
     lib.grawa_sumsq_static.restype = ci
     lib.grawa_debug_bounds_violations.argtypes = [ci]
@@ -151,8 +163,34 @@ def _raise(status: int, where: str):
         raise GrawaError(status, where)
 
 
+def _options(weights_out=None, scores_out=None, sumsq_out=None, workspace=None, status_word=None):
+    """The optional-arguments struct, or None when every option is at its default."""
+    if all(b is None for b in (weights_out, scores_out, sumsq_out, workspace, status_word)):
+        return None
+    ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    return _Options(_addr(weights_out), _addr(scores_out), _addr(sumsq_out), _addr(workspace), ws_bytes, _addr(status_word))
+
+
+def _byref(opt):
+    return ctypes.byref(opt) if opt is not None else None
+
+
+_DTYPES = {"torch.float32": 0, "torch.bfloat16": 1, "torch.float16": 2, "float32": 0, "float16": 2}
+
+
+def _dtype_of(bufs) -> int:
+    """Storage type code of a list of buffers (all of one type)."""
+    key = str(bufs[0].dtype)
+    if key not in _DTYPES:
+        raise TypeError(f"unsupported storage dtype {key}")
+    for b in bufs:
+        if str(b.dtype) != key:
+            raise TypeError(f"all buffers must be {key}, got {b.dtype}")
+    return _DTYPES[key]
+
+
 def _step(name, params, grads, pull, layer_offsets, center_out, weights_out, scores_out, sumsq_out,
-          workspace, stream, n):
+          workspace, stream, n, status_word=None):
     lib = library()
     if len(params) != len(grads):
         raise ValueError("params and grads must have one entry per worker")
@@ -161,73 +199,70 @@ def _step(name, params, grads, pull, layer_offsets, center_out, weights_out, sco
     if n is None:
         n = _numel(params[0]) if M else 0
     off, K = _offsets(layer_offsets)
-    opt = None
-    if any(b is not None for b in (weights_out, scores_out, sumsq_out, workspace)):
-        ws_bytes = 0
-        if workspace is not None:
-            ws_bytes = workspace.numel() * workspace.element_size()
-        opt = _Options(_addr(weights_out), _addr(scores_out), _addr(sumsq_out), _addr(workspace), ws_bytes)
+    opt = _options(weights_out, scores_out, sumsq_out, workspace, status_word)
     status = getattr(lib, name)(_ptr_array(params), _ptr_array(grads), n, M, float(pull),
                                 off.ctypes.data if off is not None else None, K, _addr(center_out),
-                                ctypes.byref(opt) if opt is not None else None, _stream(stream))
+                                _byref(opt), _stream(stream))
     _raise(status, name)
 
 
 # ------------------------------------------------------------------ entry points (same names as the C ABI)
 
 def grawa_mgrawa_step(params, grads, pull, layer_offsets=None, center_out=None, *, weights_out=None,
-                      scores_out=None, sumsq_out=None, workspace=None, stream=None, n=None) -> None:
+                      scores_out=None, sumsq_out=None, workspace=None, stream=None, n=None, status_word=None) -> None:
     """MGRAWA step (Eq. 3-4, centre, pull) in place on ``params``; see grawa_mgrawa_step in grawa.h."""
     _step("grawa_mgrawa_step", params, grads, pull, layer_offsets, center_out, weights_out, scores_out,
-          sumsq_out, workspace, stream, n)
+          sumsq_out, workspace, stream, n, status_word)
 
 
 def grawa_grawa_step(params, grads, pull, layer_offsets=None, center_out=None, *, weights_out=None,
-                     scores_out=None, sumsq_out=None, workspace=None, stream=None, n=None) -> None:
+                     scores_out=None, sumsq_out=None, workspace=None, stream=None, n=None, status_word=None) -> None:
     """Vanilla GRAWA step (Eq. 2: flat gradient norm); see grawa_grawa_step in grawa.h."""
     _step("grawa_grawa_step", params, grads, pull, layer_offsets, center_out, weights_out, scores_out,
-          sumsq_out, workspace, stream, n)
+          sumsq_out, workspace, stream, n, status_word)
 
 
 def grawa_lgrawa_step(params, grads, pull, layer_offsets, center_out=None, *, weights_out=None,
-                      scores_out=None, sumsq_out=None, workspace=None, stream=None, n=None) -> None:
+                      scores_out=None, sumsq_out=None, workspace=None, stream=None, n=None, status_word=None) -> None:
     """LGRAWA step (Eq. 5-7: per-layer weights); see grawa_lgrawa_step in grawa.h."""
     _step("grawa_lgrawa_step", params, grads, pull, layer_offsets, center_out, weights_out, scores_out,
-          sumsq_out, workspace, stream, n)
-
-
-_DTYPES = {"torch.float32": 0, "torch.bfloat16": 1, "torch.float16": 2}
+          sumsq_out, workspace, stream, n, status_word)
 
 
 def grawa_step_typed(variant, params, grads, pull, layer_offsets=None, center_out=None, *, weights_out=None,
-                     scores_out=None, sumsq_out=None, workspace=None, stream=None, n=None) -> None:
+                     scores_out=None, sumsq_out=None, workspace=None, stream=None, n=None, status_word=None) -> None:
     """The step on parameters / gradients / centre stored as float32, bfloat16 or float16 device tensors
     (all of one dtype, taken from ``params[0]``); arithmetic in fp32/fp64, one rounding per stored value."""
-    lib = library()
     M = len(params)
     if len(grads) != M or M == 0:
         raise ValueError("params and grads must have one entry per worker")
-    key = str(params[0].dtype)
-    if key not in _DTYPES:
-        raise TypeError(f"unsupported storage dtype {key}")
-    for b in list(params) + list(grads) + ([center_out] if center_out is not None else []):
-        if str(b.dtype) != key:
-            raise TypeError(f"all buffers must be {key}, got {b.dtype}")
+    dt = _dtype_of(list(params) + list(grads) + ([center_out] if center_out is not None else []))
     v = _VARIANTS[variant] if isinstance(variant, str) else int(variant)
     if n is None:
         n = _numel(params[0])
     off, K = _offsets(layer_offsets)
-    opt = None
-    if any(b is not None for b in (weights_out, scores_out, sumsq_out, workspace)):
-        ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
-        opt = _Options(_addr(weights_out), _addr(scores_out), _addr(sumsq_out), _addr(workspace), ws_bytes)
-    _raise(lib.grawa_step_typed(_DTYPES[key], v, _ptr_array(params), _ptr_array(grads), n, M, float(pull),
-                                off.ctypes.data if off is not None else None, K, _addr(center_out),
-                                ctypes.byref(opt) if opt is not None else None, _stream(stream)), "grawa_step_typed")
+    opt = _options(weights_out, scores_out, sumsq_out, workspace, status_word)
+    _raise(library().grawa_step_typed(dt, v, _ptr_array(params), _ptr_array(grads), n, M, float(pull),
+                                      off.ctypes.data if off is not None else None, K, _addr(center_out),
+                                      _byref(opt), _stream(stream)), "grawa_step_typed")
+
+
+def grawa_step_host_typed(variant, params, grads, pull, layer_offsets=None, center_out=None, *, stream=None, n=None) -> None:
+    """Whole step with HOST buffers (numpy arrays or pinned CPU tensors) of float32, float16 or bfloat16;
+    synchronises before returning."""
+    v = _VARIANTS[variant] if isinstance(variant, str) else int(variant)
+    M = len(params)
+    dt = _dtype_of(list(params) + list(grads) + ([center_out] if center_out is not None else []))
+    if n is None:
+        n = _numel(params[0]) if M else 0
+    off, K = _offsets(layer_offsets)
+    _raise(library().grawa_step_host_typed(dt, v, _ptr_array(params), _ptr_array(grads), n, M, float(pull),
+                                           off.ctypes.data if off is not None else None, K, _addr(center_out),
+                                           _stream(stream)), "grawa_step_host_typed")
 
 
 def grawa_step_host(variant, params, grads, pull, layer_offsets=None, center_out=None, *, stream=None, n=None) -> None:
-    """Whole step with HOST buffers (numpy arrays or pinned CPU tensors); synchronises before returning."""
+    """Whole step with HOST float32 buffers (numpy arrays or pinned CPU tensors); synchronises before returning."""
     lib = library()
     v = _VARIANTS[variant] if isinstance(variant, str) else int(variant)
     _check_f32(list(params) + list(grads) + ([center_out] if center_out is not None else []))
@@ -240,6 +275,15 @@ def grawa_step_host(variant, params, grads, pull, layer_offsets=None, center_out
     _raise(status, "grawa_step_host")
 
 
+def grawa_prox_step_typed(params, center, mu_over_tau, *, stream=None, n=None) -> None:
+    """Proximity step on float32, bfloat16 or float16 device tensors (dtype taken from the buffers)."""
+    dt = _dtype_of(list(params) + [center])
+    if n is None:
+        n = _numel(center)
+    _raise(library().grawa_prox_step_typed(dt, _ptr_array(params), _addr(center), n, len(params), float(mu_over_tau),
+                                           _stream(stream)), "grawa_prox_step_typed")
+
+
 def grawa_prox_step(params, center, mu_over_tau, *, stream=None, n=None) -> None:
     """Proximity step x_m <- (1 - mu/tau) x_m + (mu/tau) x_C for all workers in one pass."""
     lib = library()
@@ -249,6 +293,16 @@ def grawa_prox_step(params, center, mu_over_tau, *, stream=None, n=None) -> None
         n = _numel(center)
     _raise(lib.grawa_prox_step(_ptr_array(params), _addr(center), n, M, float(mu_over_tau), _stream(stream)),
            "grawa_prox_step")
+
+
+def grawa_layer_norms_typed(grad, layer_offsets, norms_out, *, stream=None, n=None) -> None:
+    """Per-layer L2 norms of one worker's gradient (float32, bfloat16 or float16) into ``norms_out`` (K float64)."""
+    dt = _dtype_of([grad])
+    if n is None:
+        n = _numel(grad)
+    off, K = _offsets(layer_offsets)
+    _raise(library().grawa_layer_norms_typed(dt, _addr(grad), n, off.ctypes.data if off is not None else None, K,
+                                             _addr(norms_out), _stream(stream)), "grawa_layer_norms_typed")
 
 
 def grawa_layer_norms(grad, layer_offsets, norms_out, *, stream=None, n=None) -> None:
@@ -267,25 +321,37 @@ def grawa_norm_ema(g_mvg, g_cur, gamma, t, g_est, *, stream=None) -> None:
                                     _stream(stream)), "grawa_norm_ema")
 
 
-def grawa_step_from_layer_norms(variant, params, layer_norms, pull, layer_offsets=None, center_out=None, *,
-                                weights_out=None, scores_out=None, sumsq_out=None, workspace=None, stream=None,
-                                n=None) -> None:
-    """Averaging step with scores from given per-layer norms ([K, M] device float64) instead of gradients."""
-    lib = library()
+def _from_given(name, typed, variant, params, table, parts, pull, layer_offsets, center_out, weights_out, scores_out,
+                sumsq_out, workspace, stream, n, status_word):
     v = _VARIANTS[variant] if isinstance(variant, str) else int(variant)
-    _check_f32(list(params) + ([center_out] if center_out is not None else []))
+    bufs = list(params) + ([center_out] if center_out is not None else [])
     M = len(params)
     if n is None:
         n = _numel(params[0]) if M else 0
     off, K = _offsets(layer_offsets)
-    opt = None
-    if any(b is not None for b in (weights_out, scores_out, sumsq_out, workspace)):
-        ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
-        opt = _Options(_addr(weights_out), _addr(scores_out), _addr(sumsq_out), _addr(workspace), ws_bytes)
-    _raise(lib.grawa_step_from_layer_norms(v, _ptr_array(params), _addr(layer_norms), n, M, float(pull),
-                                           off.ctypes.data if off is not None else None, K, _addr(center_out),
-                                           ctypes.byref(opt) if opt is not None else None, _stream(stream)),
-           "grawa_step_from_layer_norms")
+    opt = _options(weights_out, scores_out, sumsq_out, workspace, status_word)
+    head = [_dtype_of(bufs), v] if typed else [v]
+    if not typed:
+        _check_f32(bufs)
+    mid = [_ptr_array(params), _addr(table)] + ([int(parts)] if parts is not None else [])
+    tail = [n, M, float(pull), off.ctypes.data if off is not None else None, K, _addr(center_out), _byref(opt), _stream(stream)]
+    _raise(getattr(library(), name)(*(head + mid + tail)), name)
+
+
+def grawa_step_from_layer_norms(variant, params, layer_norms, pull, layer_offsets=None, center_out=None, *,
+                                weights_out=None, scores_out=None, sumsq_out=None, workspace=None, stream=None,
+                                n=None, status_word=None) -> None:
+    """Averaging step with scores from given per-layer norms ([K, M] device float64) instead of gradients."""
+    _from_given("grawa_step_from_layer_norms", False, variant, params, layer_norms, None, pull, layer_offsets, center_out,
+                weights_out, scores_out, sumsq_out, workspace, stream, n, status_word)
+
+
+def grawa_step_from_layer_norms_typed(variant, params, layer_norms, pull, layer_offsets=None, center_out=None, *,
+                                      weights_out=None, scores_out=None, sumsq_out=None, workspace=None, stream=None,
+                                      n=None, status_word=None) -> None:
+    """The same on float32, bfloat16 or float16 parameters and centre."""
+    _from_given("grawa_step_from_layer_norms_typed", True, variant, params, layer_norms, None, pull, layer_offsets,
+                center_out, weights_out, scores_out, sumsq_out, workspace, stream, n, status_word)
 
 
 def grawa_layer_sumsq(grads, layer_offsets, sumsq_out, *, stream=None, n=None) -> None:
@@ -299,25 +365,31 @@ def grawa_layer_sumsq(grads, layer_offsets, sumsq_out, *, stream=None, n=None) -
                                        _addr(sumsq_out), _stream(stream)), "grawa_layer_sumsq")
 
 
+def grawa_layer_sumsq_typed(grads, layer_offsets, sumsq_out, *, stream=None, n=None) -> None:
+    """The same from float32, bfloat16 or float16 gradients."""
+    M = len(grads)
+    dt = _dtype_of(list(grads))
+    if n is None:
+        n = _numel(grads[0]) if M else 0
+    off, K = _offsets(layer_offsets)
+    _raise(library().grawa_layer_sumsq_typed(dt, _ptr_array(grads), n, M, off.ctypes.data if off is not None else None, K,
+                                             _addr(sumsq_out), _stream(stream)), "grawa_layer_sumsq_typed")
+
+
 def grawa_step_from_layer_sums(variant, params, layer_sums, parts, pull, layer_offsets=None, center_out=None, *,
                                weights_out=None, scores_out=None, sumsq_out=None, workspace=None, stream=None,
-                               n=None) -> None:
+                               n=None, status_word=None) -> None:
     """Averaging step on local elements with S = sum over ``parts`` tables of ``layer_sums`` ([parts, K, M])."""
-    lib = library()
-    v = _VARIANTS[variant] if isinstance(variant, str) else int(variant)
-    _check_f32(list(params) + ([center_out] if center_out is not None else []))
-    M = len(params)
-    if n is None:
-        n = _numel(params[0]) if M else 0
-    off, K = _offsets(layer_offsets)
-    opt = None
-    if any(b is not None for b in (weights_out, scores_out, sumsq_out, workspace)):
-        ws_bytes = workspace.numel() * workspace.element_size() if workspace is not None else 0
-        opt = _Options(_addr(weights_out), _addr(scores_out), _addr(sumsq_out), _addr(workspace), ws_bytes)
-    _raise(lib.grawa_step_from_layer_sums(v, _ptr_array(params), _addr(layer_sums), int(parts), n, M, float(pull),
-                                          off.ctypes.data if off is not None else None, K, _addr(center_out),
-                                          ctypes.byref(opt) if opt is not None else None, _stream(stream)),
-           "grawa_step_from_layer_sums")
+    _from_given("grawa_step_from_layer_sums", False, variant, params, layer_sums, parts, pull, layer_offsets, center_out,
+                weights_out, scores_out, sumsq_out, workspace, stream, n, status_word)
+
+
+def grawa_step_from_layer_sums_typed(variant, params, layer_sums, parts, pull, layer_offsets=None, center_out=None, *,
+                                     weights_out=None, scores_out=None, sumsq_out=None, workspace=None, stream=None,
+                                     n=None, status_word=None) -> None:
+    """The same on float32, bfloat16 or float16 parameters and centre."""
+    _from_given("grawa_step_from_layer_sums_typed", True, variant, params, layer_sums, parts, pull, layer_offsets,
+                center_out, weights_out, scores_out, sumsq_out, workspace, stream, n, status_word)
 
 
 def grawa_sumsq_static(grads, sumsq_out, *, stream=None, n=None) -> None:

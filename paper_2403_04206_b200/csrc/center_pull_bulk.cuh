@@ -141,7 +141,7 @@ center_pull_bulk_kernel(MutPtrs x, float* __restrict__ center, const float* __re
             split_range(b, b + len, 1, hb, te);
             bytes = static_cast<unsigned>(te - hb) * 4u;
         }
-        if (bytes > 0 && !in_bounds(hb, bytes / 4, n)) bytes = 0;      // debug build: never copy outside the vector
+        if (bytes > 0 && !in_bounds(hb, bytes / 4, b, b + len, n)) bytes = 0;      // debug build: never copy outside the vector
         if (lane == 0) mbar_arrive_expect_tx(&full_bar[s], bytes * static_cast<unsigned>(M));
         __syncwarp();
         if (bytes > 0) {
@@ -219,9 +219,9 @@ center_pull_bulk_kernel(MutPtrs x, float* __restrict__ center, const float* __re
             }
             // unaligned layer edges: at most 3 elements on each side, straight in global memory
             for (long long i = b + tid; i < hb; i += kThreads)
-                if (in_bounds(i, 1, n)) bulk_edge_element(x, center, bt, M, lambda, oml, i);
+                if (in_bounds(i, 1, b, e, n)) bulk_edge_element(x, center, bt, M, lambda, oml, i);
             for (long long i = te + tid; i < e; i += kThreads)
-                if (in_bounds(i, 1, n)) bulk_edge_element(x, center, bt, M, lambda, oml, i);
+                if (in_bounds(i, 1, b, e, n)) bulk_edge_element(x, center, bt, M, lambda, oml, i);
         }
         fence_async_proxy();                          // this thread's shared-memory writes -> async proxy
         if (__syncthreads_or(ok ? 0 : 1)) { timed_out = true; break; }   // uniform: some thread's wait ran out
@@ -229,7 +229,7 @@ center_pull_bulk_kernel(MutPtrs x, float* __restrict__ center, const float* __re
 
         if (warp == 0) {
             const unsigned bytes = static_cast<unsigned>(te - hb) * 4u;
-            if (bytes > 0 && in_bounds(hb, bytes / 4, n)) {
+            if (bytes > 0 && in_bounds(hb, bytes / 4, si.begin, si.begin + si.len, n)) {
                 for (int m = lane; m < M; m += 32) bulk_store(x.p[m] + hb, st + m * slice_floats, bytes);
                 if (lane == 0 && center) bulk_store(center + hb, st + M * slice_floats, bytes);
             }

@@ -132,7 +132,7 @@ struct Plan {
     bool ws_dirty = false;           // a step failed half-way: the owned scratch is cleared before the next one
     void* d_ws = nullptr;            // owned scratch (used when the caller passes none)
     WorkspaceLayout ws{};
-    float* d_stage = nullptr;        // owned staging for the host-buffer entry point
+    void* d_stage = nullptr;         // owned staging for the host-buffer entry point
     int sm_count = 148;
     std::vector<Segment> h_segs2;    // host copy of the centre+pull items (chunking of the host-buffer path)
     cudaStream_t d2h_stream = nullptr;   // downloads of the host-buffer path
@@ -247,6 +247,12 @@ static grawa_status validate(float* const* params, const float* const* grads, in
 }
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+static inline bool dtype_ok(grawa_dtype d) { return d == GRAWA_F32 || d == GRAWA_BF16 || d == GRAWA_F16; }
+static inline bool variant_ok(grawa_variant v)
+{
+    return v == GRAWA_VARIANT_GRAWA || v == GRAWA_VARIANT_MGRAWA || v == GRAWA_VARIANT_LGRAWA;
+}
+static inline size_t elem_size(int dtype) { return dtype == 0 ? sizeof(float) : size_t{2}; }
 
 // ------------------------------------------------------------------ launches
 // One launch, optionally with programmatic stream serialisation (the kernel may start launching
@@ -431,7 +437,7 @@ static grawa_status make_context(int variant, float* const* params, const float*
     sc.S = reinterpret_cast<double*>(ws + plan->ws.S);
     sc.A = reinterpret_cast<double*>(ws + plan->ws.A);
     sc.beta = reinterpret_cast<float*>(ws + plan->ws.beta);
-    sc.status_copy = nullptr;
+    sc.status_copy = opt ? opt->status_word : nullptr;
     sc.status = ctx->status; sc.work_counter = ctx->counter;
     sc.weights_out = opt ? opt->weights_out : nullptr;
     sc.scores_out = opt ? opt->scores_out : nullptr;
@@ -656,7 +662,7 @@ sumsq_flat_kernel(ConstPtrs grads, long long n, int tiles, int tile, double* __r
 #pragma unroll
         for (int u = 0; u < UNROLL; ++u) {
             const int c = c0 + u * kThreads + tid;
-            v[u] = (c < ncol) ? ld_stream4(g4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+            v[u] = (c < ncol && in_bounds(hb + 4LL * c, 4, b, e, n)) ? ld_stream4(g4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
         float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
@@ -670,15 +676,16 @@ sumsq_flat_kernel(ConstPtrs grads, long long n, int tiles, int tile, double* __r
                 (static_cast<double>(a2) + static_cast<double>(a3));
     }
     for (long long i = b + tid; i < hb; i += kThreads) {
-        const double v = static_cast<double>(ld_stream1(g + i));
+        const double v = in_bounds(i, 1, b, e, n) ? static_cast<double>(ld_stream1(g + i)) : 0.0;
         dacc += v * v;
     }
     for (long long i = te + tid; i < e; i += kThreads) {
-        const double v = static_cast<double>(ld_stream1(g + i));
+        const double v = in_bounds(i, 1, b, e, n) ? static_cast<double>(ld_stream1(g + i)) : 0.0;
         dacc += v * v;
     }
     const double total = block_sum_fixed_order<kThreads>(dacc);
-    if (tid == 0) partials[static_cast<size_t>(m) * tiles + t] = total;
+    if (tid == 0 && scratch_ok(static_cast<long long>(m) * tiles + t, GRAWA_STATIC_MAX_PARTIALS))
+        partials[static_cast<size_t>(m) * tiles + t] = total;
 }
 
 // One CTA per worker adds that worker's `tiles` partial sums in a fixed order.
@@ -687,7 +694,8 @@ sum_partials_kernel(const double* __restrict__ partials, int tiles, double* __re
 {
     const double* __restrict__ row = partials + static_cast<size_t>(blockIdx.x) * tiles;
     double acc = 0.0;
-    for (int s = threadIdx.x; s < tiles; s += kFinalizeThreads) acc += row[s];
+    for (int s = threadIdx.x; s < tiles; s += kFinalizeThreads)
+        if (scratch_ok(static_cast<long long>(blockIdx.x) * tiles + s, GRAWA_STATIC_MAX_PARTIALS)) acc += row[s];
     const double total = block_sum_fixed_order<kFinalizeThreads>(acc);
     if (threadIdx.x == 0) out[blockIdx.x] = total;
 }
@@ -766,39 +774,55 @@ grawa_status grawa_step_typed(grawa_dtype dtype, grawa_variant variant, void* co
                       static_cast<float*>(center_out), options, stream, static_cast<int>(dtype));
 }
 
+grawa_status grawa_step_from_layer_norms_typed(grawa_dtype dtype, grawa_variant variant, void* const* params,
+                                               const double* layer_norms, int64_t n, int M, float pull,
+                                               const int64_t* layer_offsets, int n_layers, void* center_out,
+                                               const grawa_options* options, grawa_stream_t stream)
+{
+    if (!variant_ok(variant) || !dtype_ok(dtype)) return GRAWA_ERR_INVALID_ARG;
+    GivenScores given;
+    given.data = layer_norms;
+    return step_entry(static_cast<int>(variant), reinterpret_cast<float* const*>(params), nullptr, given, n, M, pull, layer_offsets,
+                      n_layers, static_cast<float*>(center_out), options, stream, static_cast<int>(dtype));
+}
+
 grawa_status grawa_step_from_layer_norms(grawa_variant variant, float* const* params, const double* layer_norms, int64_t n,
                                          int M, float pull, const int64_t* layer_offsets, int n_layers, float* center_out,
                                          const grawa_options* options, grawa_stream_t stream)
 {
-    if (variant != GRAWA_VARIANT_GRAWA && variant != GRAWA_VARIANT_MGRAWA && variant != GRAWA_VARIANT_LGRAWA)
-        return GRAWA_ERR_INVALID_ARG;
+    return grawa_step_from_layer_norms_typed(GRAWA_F32, variant, reinterpret_cast<void* const*>(params), layer_norms, n, M, pull,
+                                             layer_offsets, n_layers, center_out, options, stream);
+}
+
+grawa_status grawa_step_from_layer_sums_typed(grawa_dtype dtype, grawa_variant variant, void* const* params,
+                                              const double* layer_sums, int parts, int64_t n, int M, float pull,
+                                              const int64_t* layer_offsets, int n_layers, void* center_out,
+                                              const grawa_options* options, grawa_stream_t stream)
+{
+    if (!variant_ok(variant) || !dtype_ok(dtype)) return GRAWA_ERR_INVALID_ARG;
     GivenScores given;
-    given.data = layer_norms;
-    return step_entry(static_cast<int>(variant), params, nullptr, given, n, M, pull, layer_offsets, n_layers, center_out,
-                      options, stream);
+    given.data = layer_sums; given.parts = parts; given.sums = 1;
+    return step_entry(static_cast<int>(variant), reinterpret_cast<float* const*>(params), nullptr, given, n, M, pull, layer_offsets,
+                      n_layers, static_cast<float*>(center_out), options, stream, static_cast<int>(dtype));
 }
 
 grawa_status grawa_step_from_layer_sums(grawa_variant variant, float* const* params, const double* layer_sums, int parts,
                                         int64_t n, int M, float pull, const int64_t* layer_offsets, int n_layers,
                                         float* center_out, const grawa_options* options, grawa_stream_t stream)
 {
-    if (variant != GRAWA_VARIANT_GRAWA && variant != GRAWA_VARIANT_MGRAWA && variant != GRAWA_VARIANT_LGRAWA)
-        return GRAWA_ERR_INVALID_ARG;
-    GivenScores given;
-    given.data = layer_sums; given.parts = parts; given.sums = 1;
-    return step_entry(static_cast<int>(variant), params, nullptr, given, n, M, pull, layer_offsets, n_layers, center_out,
-                      options, stream);
+    return grawa_step_from_layer_sums_typed(GRAWA_F32, variant, reinterpret_cast<void* const*>(params), layer_sums, parts, n, M,
+                                            pull, layer_offsets, n_layers, center_out, options, stream);
 }
 
-grawa_status grawa_layer_sumsq(const float* const* grads, int64_t n, int M, const int64_t* layer_offsets, int n_layers,
-                               double* sumsq_out, grawa_stream_t stream)
+grawa_status grawa_layer_sumsq_typed(grawa_dtype dtype, const void* const* grads, int64_t n, int M,
+                                     const int64_t* layer_offsets, int n_layers, double* sumsq_out, grawa_stream_t stream)
 {
-    if (grads == nullptr || sumsq_out == nullptr || M < 1 || M > GRAWA_MAX_WORKERS) return GRAWA_ERR_INVALID_ARG;
+    if (grads == nullptr || sumsq_out == nullptr || M < 1 || M > GRAWA_MAX_WORKERS || !dtype_ok(dtype)) return GRAWA_ERR_INVALID_ARG;
     // validate() wants parameter vectors; the gradients stand in (nothing is written through them)
     std::vector<float*> fake(M);
-    for (int m = 0; m < M; ++m) fake[m] = const_cast<float*>(grads[m]);
+    for (int m = 0; m < M; ++m) fake[m] = static_cast<float*>(const_cast<void*>(grads[m]));
     std::vector<int64_t> off;
-    grawa_status st = validate(fake.data(), nullptr, n, M, 0.0f, layer_offsets, n_layers, nullptr, &off);
+    grawa_status st = validate(fake.data(), nullptr, n, M, 0.0f, layer_offsets, n_layers, nullptr, &off, elem_size(dtype));
     if (st != GRAWA_OK) return st;
     std::lock_guard<std::mutex> lock(g_mutex);
     if (n == 0) {                                    // nothing to add up: every sum is zero
@@ -806,36 +830,51 @@ grawa_status grawa_layer_sumsq(const float* const* grads, int64_t n, int M, cons
         return GRAWA_OK;
     }
     Plan* plan = nullptr;
-    st = get_plan(n, M, off, stream, &plan);
+    st = get_plan(n, M, off, stream, &plan, dtype == GRAWA_F32 ? 4 : 2);
     if (st != GRAWA_OK) return st;
     grawa_options opt{};
     opt.sumsq_out = sumsq_out;
     StepContext c;
-    st = make_context(kLgrawa, fake.data(), grads, n, M, 0.0f, nullptr, &opt, stream, plan, &c);
+    st = make_context(kLgrawa, fake.data(), reinterpret_cast<const float* const*>(grads), n, M, 0.0f, nullptr, &opt, stream, plan, &c);
     if (st != GRAWA_OK) return st;
+    c.dtype = static_cast<int>(dtype);
+    return enqueue_weights(c);
+}
+
+grawa_status grawa_layer_sumsq(const float* const* grads, int64_t n, int M, const int64_t* layer_offsets, int n_layers,
+                               double* sumsq_out, grawa_stream_t stream)
+{
+    return grawa_layer_sumsq_typed(GRAWA_F32, reinterpret_cast<const void* const*>(grads), n, M, layer_offsets, n_layers, sumsq_out,
+                                   stream);
+}
+
+grawa_status grawa_layer_norms_typed(grawa_dtype dtype, const void* grad, int64_t n, const int64_t* layer_offsets, int n_layers,
+                                     double* norms_out, grawa_stream_t stream)
+{
+    if (grad == nullptr || norms_out == nullptr || n < 0 || !dtype_ok(dtype)) return GRAWA_ERR_INVALID_ARG;
+    // validate() wants a parameter vector; the gradient stands in (nothing is written through it)
+    float* fake_params[1] = {static_cast<float*>(const_cast<void*>(grad))};
+    std::vector<int64_t> off;
+    grawa_status st = validate(fake_params, nullptr, n, 1, 0.0f, layer_offsets, n_layers, nullptr, &off, elem_size(dtype));
+    if (st != GRAWA_OK || n == 0) return st;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    Plan* plan = nullptr;
+    st = get_plan(n, 1, off, stream, &plan, dtype == GRAWA_F32 ? 4 : 2);
+    if (st != GRAWA_OK) return st;
+    grawa_options opt{};
+    opt.scores_out = norms_out;
+    const float* grads[1] = {static_cast<const float*>(grad)};
+    StepContext c;
+    st = make_context(kLgrawa, fake_params, grads, n, 1, 0.0f, nullptr, &opt, stream, plan, &c);
+    if (st != GRAWA_OK) return st;
+    c.dtype = static_cast<int>(dtype);
     return enqueue_weights(c);
 }
 
 grawa_status grawa_layer_norms(const float* grad, int64_t n, const int64_t* layer_offsets, int n_layers, double* norms_out,
                                grawa_stream_t stream)
 {
-    if (grad == nullptr || norms_out == nullptr || n < 0 || (reinterpret_cast<uintptr_t>(grad) & 3u)) return GRAWA_ERR_INVALID_ARG;
-    // validate() wants a parameter vector; the gradient stands in (nothing is written through it)
-    float* fake_params[1] = {const_cast<float*>(grad)};
-    std::vector<int64_t> off;
-    grawa_status st = validate(fake_params, nullptr, n, 1, 0.0f, layer_offsets, n_layers, nullptr, &off);
-    if (st != GRAWA_OK || n == 0) return st;
-    std::lock_guard<std::mutex> lock(g_mutex);
-    Plan* plan = nullptr;
-    st = get_plan(n, 1, off, stream, &plan);
-    if (st != GRAWA_OK) return st;
-    grawa_options opt{};
-    opt.scores_out = norms_out;
-    const float* grads[1] = {grad};
-    StepContext c;
-    st = make_context(kLgrawa, fake_params, grads, n, 1, 0.0f, nullptr, &opt, stream, plan, &c);
-    if (st != GRAWA_OK) return st;
-    return enqueue_weights(c);
+    return grawa_layer_norms_typed(GRAWA_F32, grad, n, layer_offsets, n_layers, norms_out, stream);
 }
 
 grawa_status grawa_norm_ema(double* g_mvg, const double* g_cur, int n_layers, double gamma, int64_t t, double* g_est,
@@ -850,35 +889,38 @@ grawa_status grawa_norm_ema(double* g_mvg, const double* g_cur, int n_layers, do
     return GRAWA_OK;
 }
 
-grawa_status grawa_step_host(grawa_variant variant, float* const* params, const float* const* grads, int64_t n, int M,
-                             float pull, const int64_t* layer_offsets, int n_layers, float* center_out,
-                             grawa_stream_t stream)
+grawa_status grawa_step_host_typed(grawa_dtype dtype, grawa_variant variant, void* const* params, const void* const* grads,
+                                   int64_t n, int M, float pull, const int64_t* layer_offsets, int n_layers, void* center_out,
+                                   grawa_stream_t stream)
 {
-    if (variant != GRAWA_VARIANT_GRAWA && variant != GRAWA_VARIANT_MGRAWA && variant != GRAWA_VARIANT_LGRAWA)
-        return GRAWA_ERR_INVALID_ARG;
-    if (grads == nullptr) return GRAWA_ERR_INVALID_ARG;
+    if (!variant_ok(variant) || !dtype_ok(dtype) || grads == nullptr) return GRAWA_ERR_INVALID_ARG;
+    const size_t es = elem_size(dtype);
     std::vector<int64_t> off;
-    grawa_status st = validate(params, grads, n, M, pull, layer_offsets, n_layers, center_out, &off);
+    grawa_status st = validate(reinterpret_cast<float* const*>(params), reinterpret_cast<const float* const*>(grads), n, M, pull,
+                               layer_offsets, n_layers, static_cast<const float*>(center_out), &off, es);
     if (st != GRAWA_OK || n == 0) return st;
     std::lock_guard<std::mutex> lock(g_mutex);
     Plan* plan = nullptr;
-    st = get_plan(n, M, off, stream, &plan);
+    st = get_plan(n, M, off, stream, &plan, dtype == GRAWA_F32 ? 4 : 2);
     if (st != GRAWA_OK) return st;
-    const size_t nn = align_up(static_cast<size_t>(n), 64);      // keeps every staged vector 256-byte aligned
-    if (!plan->d_stage) GRAWA_CUDA_TRY(cudaMalloc(&plan->d_stage, sizeof(float) * nn * (2 * static_cast<size_t>(M) + 1)));
+    const size_t nn = align_up(static_cast<size_t>(n), 128);     // keeps every staged vector 256-byte aligned
+    if (!plan->d_stage) GRAWA_CUDA_TRY(cudaMalloc(&plan->d_stage, es * nn * (2 * static_cast<size_t>(M) + 1)));
     if (!plan->d2h_stream) GRAWA_CUDA_TRY(cudaStreamCreateWithFlags(&plan->d2h_stream, cudaStreamNonBlocking));
-    std::vector<float*> dx(M);
+    char* stage = reinterpret_cast<char*>(plan->d_stage);
+    std::vector<float*> dx(M);                        // untyped device addresses; the kernels of `dtype` type them
     std::vector<const float*> dg(M);
-    float* dc = plan->d_stage + nn * 2 * M;
-    const size_t bytes = sizeof(float) * static_cast<size_t>(n);
+    char* dc = stage + es * nn * 2 * M;
+    const size_t bytes = es * static_cast<size_t>(n);
     for (int m = 0; m < M; ++m) {
-        dg[m] = plan->d_stage + nn * m;
-        dx[m] = plan->d_stage + nn * (M + m);
-        GRAWA_CUDA_TRY(cudaMemcpyAsync(plan->d_stage + nn * m, grads[m], bytes, cudaMemcpyHostToDevice, stream));
+        dg[m] = reinterpret_cast<const float*>(stage + es * nn * m);
+        dx[m] = reinterpret_cast<float*>(stage + es * nn * (M + m));
+        GRAWA_CUDA_TRY(cudaMemcpyAsync(stage + es * nn * m, grads[m], bytes, cudaMemcpyHostToDevice, stream));
     }
     StepContext c;
-    st = make_context(variant, dx.data(), dg.data(), n, M, pull, center_out ? dc : nullptr, nullptr, stream, plan, &c);
+    st = make_context(variant, dx.data(), dg.data(), n, M, pull, center_out ? reinterpret_cast<float*>(dc) : nullptr, nullptr, stream,
+                      plan, &c);
     if (st != GRAWA_OK) return st;
+    c.dtype = static_cast<int>(dtype);
     st = enqueue_weights(c);                          // runs while the parameters are still arriving
     if (st != GRAWA_OK) return st;
     if (M == 1) {
@@ -890,7 +932,7 @@ grawa_status grawa_step_host(grawa_variant variant, float* const* params, const 
     // Centre+pull in chunks of work items: upload the chunk of all M workers, run it, and download
     // its results on a second stream while the next chunk is being uploaded (the two directions of
     // the host link work at the same time).
-    const bool per_layer = variant == kLgrawa;
+    const bool per_layer = static_cast<int>(variant) == kLgrawa;
     const int items = c.pull_items;
     const int64_t chunk_elems = std::max<int64_t>(int64_t{1} << 20, (n + 15) / 16);
     auto item_begin_elem = [&](int i) -> int64_t {
@@ -904,9 +946,10 @@ grawa_status grawa_step_host(grawa_variant variant, float* const* params, const 
         const int64_t e0 = item_begin_elem(i0);
         while (i1 < items && item_begin_elem(i1) - e0 < chunk_elems) ++i1;
         const int64_t e1 = item_begin_elem(i1);
-        const size_t cb = sizeof(float) * static_cast<size_t>(e1 - e0);
+        const size_t cb = es * static_cast<size_t>(e1 - e0), o0 = es * static_cast<size_t>(e0);
         for (int m = 0; m < M; ++m)
-            GRAWA_CUDA_TRY(cudaMemcpyAsync(dx[m] + e0, params[m] + e0, cb, cudaMemcpyHostToDevice, stream));
+            GRAWA_CUDA_TRY(cudaMemcpyAsync(reinterpret_cast<char*>(dx[m]) + o0, static_cast<const char*>(params[m]) + o0, cb,
+                                           cudaMemcpyHostToDevice, stream));
         if (plan->bulk) GRAWA_CUDA_TRY(cudaMemsetAsync(c.counter, 0, sizeof(unsigned), stream));
         st = enqueue_center_pull(c, i0, i1);
         if (st != GRAWA_OK) return st;
@@ -919,13 +962,23 @@ grawa_status grawa_step_host(grawa_variant variant, float* const* params, const 
         GRAWA_CUDA_TRY(cudaEventRecord(ev, stream));
         GRAWA_CUDA_TRY(cudaStreamWaitEvent(plan->d2h_stream, ev, 0));
         for (int m = 0; m < M; ++m)
-            GRAWA_CUDA_TRY(cudaMemcpyAsync(params[m] + e0, dx[m] + e0, cb, cudaMemcpyDeviceToHost, plan->d2h_stream));
-        if (center_out) GRAWA_CUDA_TRY(cudaMemcpyAsync(center_out + e0, dc + e0, cb, cudaMemcpyDeviceToHost, plan->d2h_stream));
+            GRAWA_CUDA_TRY(cudaMemcpyAsync(static_cast<char*>(params[m]) + o0, reinterpret_cast<char*>(dx[m]) + o0, cb,
+                                           cudaMemcpyDeviceToHost, plan->d2h_stream));
+        if (center_out)
+            GRAWA_CUDA_TRY(cudaMemcpyAsync(static_cast<char*>(center_out) + o0, dc + o0, cb, cudaMemcpyDeviceToHost, plan->d2h_stream));
         i0 = i1;
     }
     GRAWA_CUDA_TRY(cudaStreamSynchronize(plan->d2h_stream));
     GRAWA_CUDA_TRY(cudaStreamSynchronize(stream));
     return GRAWA_OK;
+}
+
+grawa_status grawa_step_host(grawa_variant variant, float* const* params, const float* const* grads, int64_t n, int M,
+                             float pull, const int64_t* layer_offsets, int n_layers, float* center_out,
+                             grawa_stream_t stream)
+{
+    return grawa_step_host_typed(GRAWA_F32, variant, reinterpret_cast<void* const*>(params),
+                                 reinterpret_cast<const void* const*>(grads), n, M, pull, layer_offsets, n_layers, center_out, stream);
 }
 
 grawa_status grawa_last_step_status(grawa_stream_t stream)
@@ -947,27 +1000,41 @@ grawa_status grawa_last_step_status(grawa_stream_t stream)
     return GRAWA_OK;
 }
 
-grawa_status grawa_prox_step(float* const* params, const float* center, int64_t n, int M, float mu_over_tau,
-                             grawa_stream_t stream)
+grawa_status grawa_prox_step_typed(grawa_dtype dtype, void* const* params, const void* center, int64_t n, int M,
+                                   float mu_over_tau, grawa_stream_t stream)
 {
-    if (center == nullptr && n > 0) return GRAWA_ERR_INVALID_ARG;
+    if (!dtype_ok(dtype) || (center == nullptr && n > 0)) return GRAWA_ERR_INVALID_ARG;
     std::vector<int64_t> off;
-    grawa_status st = validate(params, nullptr, n, M, mu_over_tau, nullptr, 0, center, &off);
+    grawa_status st = validate(reinterpret_cast<float* const*>(params), nullptr, n, M, mu_over_tau, nullptr, 0,
+                               static_cast<const float*>(center), &off, elem_size(dtype));
     if (st != GRAWA_OK || n == 0) return st;
     MutPtrs xp{};
     bool vec = aligned16(center);
-    for (int m = 0; m < M; ++m) { xp.p[m] = params[m]; vec = vec && aligned16(params[m]); }
+    for (int m = 0; m < M; ++m) { xp.p[m] = static_cast<float*>(params[m]); vec = vec && aligned16(params[m]); }
     int64_t tile;
     {
         std::lock_guard<std::mutex> lock(g_mutex);
-        tile = g_pull_tile > 0 ? g_pull_tile : 1024;   // one vector column per thread: measured best (6.6-6.9 TB/s)
+        // one vector column per thread (measured best): 1024 fp32 or 2048 16-bit elements per CTA
+        tile = g_pull_tile > 0 ? g_pull_tile : (dtype == GRAWA_F32 ? 1024 : 2048);
     }
     const int64_t tiles = (n + tile - 1) / tile;
     if (tiles > 0x7fffffffll) return GRAWA_ERR_INVALID_ARG;
-    prox_kernel<<<static_cast<int>(tiles), kThreads, 0, stream>>>(xp, center, n, static_cast<int>(tile), mu_over_tau, M, vec ? 1 : 0);
+    const int grid = static_cast<int>(tiles), t = static_cast<int>(tile), v = vec ? 1 : 0;
+    if (dtype == GRAWA_BF16)
+        prox16_kernel<__nv_bfloat16><<<grid, kThreads, 0, stream>>>(xp, static_cast<const __nv_bfloat16*>(center), n, t, mu_over_tau, M, v);
+    else if (dtype == GRAWA_F16)
+        prox16_kernel<__half><<<grid, kThreads, 0, stream>>>(xp, static_cast<const __half*>(center), n, t, mu_over_tau, M, v);
+    else
+        prox_kernel<<<grid, kThreads, 0, stream>>>(xp, static_cast<const float*>(center), n, t, mu_over_tau, M, v);
     ++g_launches;
     GRAWA_CUDA_TRY(cudaGetLastError());
     return GRAWA_OK;
+}
+
+grawa_status grawa_prox_step(float* const* params, const float* center, int64_t n, int M, float mu_over_tau,
+                             grawa_stream_t stream)
+{
+    return grawa_prox_step_typed(GRAWA_F32, reinterpret_cast<void* const*>(params), center, n, M, mu_over_tau, stream);
 }
 
 grawa_status grawa_sumsq_static(const float* const* grads, int64_t n, int M, double* sumsq_out, grawa_stream_t stream)

@@ -86,28 +86,44 @@ struct KernelTrace {
 #endif
 
 // Debug build (-DGRAWA_DEBUG_BOUNDS): every global access of the streaming kernels is first checked
-// against the vector's length; a violation is counted and the access skipped (nothing traps).
-// In the normal build the check is the constant `true` and costs nothing.
+// against the work item it belongs to, [lo, hi), which itself must lie inside the vector [0, total);
+// every index into scratch memory is checked against the size of its table.  A violation is counted
+// and the access skipped (nothing traps).  In the normal build the checks are the constant `true`
+// and cost nothing.
 #ifdef GRAWA_DEBUG_BOUNDS
 __device__ int g_bounds_violations = 0;
-__device__ __forceinline__ bool in_bounds(long long first, long long count, long long total)
+__device__ __forceinline__ bool in_bounds(long long first, long long count, long long lo, long long hi, long long total)
 {
-    if (first >= 0 && count >= 0 && first + count <= total) return true;
+    if (count >= 0 && lo >= 0 && hi <= total && first >= lo && first + count <= hi) return true;
     atomicAdd(&g_bounds_violations, 1);
     return false;
 }
-// Arithmetic-only check of the checker itself: three ranges that are out of bounds, one that is not.
+__device__ __forceinline__ bool scratch_ok(long long index, long long limit)
+{
+    if (index >= 0 && index < limit) return true;
+    atomicAdd(&g_bounds_violations, 1);
+    return false;
+}
+// Arithmetic-only check of the checker itself: six triples that must be counted (outside the vector,
+// inside the vector but outside the item, an item that sticks out of the vector, a scratch index at
+// its limit), two that must not.
 __global__ void bounds_selfcheck_kernel()
 {
     if (threadIdx.x == 0) {
-        (void)in_bounds(-1, 1, 10);
-        (void)in_bounds(8, 4, 10);
-        (void)in_bounds(10, 1, 10);
-        (void)in_bounds(6, 4, 10);
+        (void)in_bounds(-1, 1, 0, 10, 10);
+        (void)in_bounds(8, 4, 0, 10, 10);
+        (void)in_bounds(10, 1, 0, 10, 10);
+        (void)in_bounds(6, 4, 0, 8, 10);        // in the vector, past the end of the item
+        (void)in_bounds(2, 1, 3, 8, 10);        // in the vector, in front of the item
+        (void)in_bounds(6, 2, 4, 12, 10);       // the item itself leaves the vector
+        (void)scratch_ok(5, 5);
+        (void)in_bounds(6, 4, 4, 10, 10);
+        (void)scratch_ok(4, 5);
     }
 }
 #else
-__device__ __forceinline__ bool in_bounds(long long, long long, long long) { return true; }
+__device__ __forceinline__ bool in_bounds(long long, long long, long long, long long, long long) { return true; }
+__device__ __forceinline__ bool scratch_ok(long long, long long) { return true; }
 #endif
 
 // Streaming accesses: every byte is touched once per step, so keep it out of the way in L1/L2
@@ -196,6 +212,7 @@ __device__ __forceinline__ void bins_add(unsigned long long* __restrict__ row, s
     const unsigned long long lo = man << r;             // bits 0..63 of man * 2^r
     const unsigned long long hi = r ? (man >> (64 - r)) : 0ull;    // bits 64..84
     const unsigned long long d0 = lo & 0xffffffffull, d1 = lo >> 32;
+    if (!scratch_ok(b0 + (hi ? 2 : d1 ? 1 : 0), kBinWords)) return;       // debug build: the digits stay inside the row
     if (d0) atomicAdd(row + b0 * stride, d0);
     if (d1) atomicAdd(row + (b0 + 1) * stride, d1);
     if (hi) atomicAdd(row + (b0 + 2) * stride, hi);     // b0 + 2 <= 9 because v < 2^170
@@ -325,6 +342,7 @@ __device__ __forceinline__ double row_term(const StepScratch& sc, size_t idx, do
 
 __device__ __forceinline__ void store_row(const StepScratch& sc, size_t idx, double s, double term)
 {
+    if (!scratch_ok(static_cast<long long>(idx), static_cast<long long>(sc.K) * sc.M)) return;
     sc.S[idx] = s;
     sc.A[idx] = term;
     if (sc.sumsq_out) sc.sumsq_out[idx] = s;
@@ -486,7 +504,7 @@ sumsq_kernel(const __grid_constant__ ConstPtrs grads, StepScratch sc, int items,
             long long phb, pte;
             split_range(sg.begin, sg.begin + sg.len, vec_ok, phb, pte);
             const unsigned bytes = static_cast<unsigned>(pte - phb) * 4u;
-            if (bytes > 0 && in_bounds(phb, pte - phb, sc.n)) prefetch_l2(grads.p[pm] + phb, bytes);
+            if (bytes > 0 && in_bounds(phb, pte - phb, sg.begin, sg.begin + sg.len, sc.n)) prefetch_l2(grads.p[pm] + phb, bytes);
         }
     }
     KernelTrace trace(0);
@@ -517,7 +535,7 @@ sumsq_kernel(const __grid_constant__ ConstPtrs grads, StepScratch sc, int items,
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const int c = c0 + u * kThreads + tid;
-                v[u] = (c < ncol && in_bounds(hb + 4LL * c, 4, sc.n)) ? ld_stream4(g4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
+                v[u] = (c < ncol && in_bounds(hb + 4LL * c, 4, b, e, sc.n)) ? ld_stream4(g4 + c) : make_float4(0.f, 0.f, 0.f, 0.f);
             }
             float a0 = 0.f, a1 = 0.f, a2 = 0.f, a3 = 0.f;
 #pragma unroll
@@ -531,11 +549,11 @@ sumsq_kernel(const __grid_constant__ ConstPtrs grads, StepScratch sc, int items,
                     (static_cast<double>(a2) + static_cast<double>(a3));
         }
         for (long long i = b + tid; i < hb; i += kThreads) {
-            const double v = in_bounds(i, 1, sc.n) ? static_cast<double>(ld_stream1(g + i)) : 0.0;
+            const double v = in_bounds(i, 1, b, e, sc.n) ? static_cast<double>(ld_stream1(g + i)) : 0.0;
             dacc += v * v;
         }
         for (long long i = te + tid; i < e; i += kThreads) {
-            const double v = in_bounds(i, 1, sc.n) ? static_cast<double>(ld_stream1(g + i)) : 0.0;
+            const double v = in_bounds(i, 1, b, e, sc.n) ? static_cast<double>(ld_stream1(g + i)) : 0.0;
             dacc += v * v;
         }
         // Fixed-order block sum.  Two alternating buffers need only one barrier per item: a warp
@@ -551,7 +569,8 @@ sumsq_kernel(const __grid_constant__ ConstPtrs grads, StepScratch sc, int items,
 #pragma unroll
             for (int w = 0; w < kThreads / 32; ++w) total += warp_part[parity][w];
             unsigned long long* bins = sc.bins + static_cast<size_t>(buf) * bins_copy_words(sc);
-            bins_add(bins + static_cast<size_t>(sg.layer) * sc.M + m, static_cast<size_t>(sc.K) * sc.M, total);
+            if (scratch_ok(buf, 2) && scratch_ok(static_cast<long long>(sg.layer) * sc.M + m, static_cast<long long>(sc.K) * sc.M))
+                bins_add(bins + static_cast<size_t>(sg.layer) * sc.M + m, static_cast<size_t>(sc.K) * sc.M, total);
         }
     }
     bins_turnover(sc, buf_sm);           // every CTA has had at least one item, hence one barrier after the write
@@ -642,7 +661,7 @@ center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restric
 #pragma unroll
         for (int q = 0; q < COLS; ++q) {
             const int c = c0 + q * kThreads + tid;
-            if (c < ncol && in_bounds(hb + static_cast<long long>(c) * VEC, VEC, n)) {
+            if (c < ncol && in_bounds(hb + static_cast<long long>(c) * VEC, VEC, b, e, n)) {
 #pragma unroll
                 for (int m = 0; m < M; ++m) VecIO<VEC>::ld(x.p[m] + hb + static_cast<long long>(c) * VEC, v[q][m]);
             }
@@ -672,7 +691,7 @@ center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restric
 #pragma unroll
                     for (int mm = 1; mm < M; ++mm)
                         if (mm == m) base = x.p[mm];                // a select chain: no run-time index into the pointer table
-                    if (bytes > 0 && in_bounds(phb, pte - phb, n)) prefetch_l2(base + phb, bytes);
+                    if (bytes > 0 && in_bounds(phb, pte - phb, pb, pe, n)) prefetch_l2(base + phb, bytes);
                 }
             }
             load_chunk(0);
@@ -700,7 +719,7 @@ center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restric
 #pragma unroll
             for (int q = 0; q < COLS; ++q) {
                 const int c = c0 + q * kThreads + tid;
-                if (c < ncol && in_bounds(hb + static_cast<long long>(c) * VEC, VEC, n)) {
+                if (c < ncol && in_bounds(hb + static_cast<long long>(c) * VEC, VEC, b, e, n)) {
                     float cc[VEC];
 #pragma unroll
                     for (int t = 0; t < VEC; ++t) cc[t] = w[0] * v[q][0][t];
@@ -722,9 +741,9 @@ center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restric
         }
         loaded = false;                                  // an item without a vector body used nothing
         for (long long i = b + tid; i < hb; i += kThreads)
-            if (in_bounds(i, 1, n)) pull_scalar<M>(x, center, w, lambda, oml, i);
+            if (in_bounds(i, 1, b, e, n)) pull_scalar<M>(x, center, w, lambda, oml, i);
         for (long long i = te + tid; i < e; i += kThreads)
-            if (in_bounds(i, 1, n)) pull_scalar<M>(x, center, w, lambda, oml, i);
+            if (in_bounds(i, 1, b, e, n)) pull_scalar<M>(x, center, w, lambda, oml, i);
         item += gridDim.x;
         if (item < item_end) locate(item);
     }
@@ -755,7 +774,7 @@ center_pull_generic_kernel(MutPtrs x, float* __restrict__ center, const float* _
     __syncthreads();
     const float oml = 1.0f - lambda;
     for (long long i = b + threadIdx.x; i < e; i += kThreads) {
-        if (!in_bounds(i, 1, n)) continue;
+        if (!in_bounds(i, 1, b, e, n)) continue;
         float c = w[0] * x.p[0][i];
         for (int m = 1; m < M; ++m) c = fmaf(w[m], x.p[m][i], c);
         if (center) center[i] = c;
@@ -787,8 +806,9 @@ copy_kernel(const float* __restrict__ src, float* __restrict__ dst, long long n,
     const long long t = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x;
     const long long n4 = vec_ok ? (n >> 2) : 0;
     for (long long c = t; c < n4; c += stride)
-        st_stream4(reinterpret_cast<float4*>(dst) + c, ld_stream4(reinterpret_cast<const float4*>(src) + c));
-    for (long long i = (n4 << 2) + t; i < n; i += stride) dst[i] = src[i];
+        if (in_bounds(4 * c, 4, 0, n, n)) st_stream4(reinterpret_cast<float4*>(dst) + c, ld_stream4(reinterpret_cast<const float4*>(src) + c));
+    for (long long i = (n4 << 2) + t; i < n; i += stride)
+        if (in_bounds(i, 1, 0, n, n)) dst[i] = src[i];
 }
 
 // Proximity step (the "Prox." update of Algorithms 1-2): x_m <- fmaf(a, x_C, (1-a) x_m), a = mu/tau.
@@ -804,7 +824,7 @@ prox_kernel(MutPtrs x, const float* __restrict__ center, long long n, int tile, 
     split_range(b, e, vec_ok, hb, te);
     const int ncol = static_cast<int>((te - hb) >> 2);
     for (int c = threadIdx.x; c < ncol; c += kThreads) {
-        if (!in_bounds(hb + 4LL * c, 4, n)) continue;
+        if (!in_bounds(hb + 4LL * c, 4, b, e, n)) continue;
         const float4 cc = ld_stream4(reinterpret_cast<const float4*>(center + hb) + c);
         int m = 0;
         for (; m + 4 <= M; m += 4) {
@@ -830,7 +850,7 @@ prox_kernel(MutPtrs x, const float* __restrict__ center, long long n, int tile, 
     for (int pass = 0; pass < 2; ++pass) {
         const long long lo = pass ? te : b, hi = pass ? e : hb;
         for (long long i = lo + threadIdx.x; i < hi; i += kThreads) {
-            if (!in_bounds(i, 1, n)) continue;
+            if (!in_bounds(i, 1, b, e, n)) continue;
             const float c = center[i];
             for (int m = 0; m < M; ++m) x.p[m][i] = fmaf(a, c, oma * x.p[m][i]);
         }

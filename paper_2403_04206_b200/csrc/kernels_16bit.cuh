@@ -108,7 +108,7 @@ sumsq16_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
                 const int c = c0 + u * kThreads + tid;
-                raw[u] = (c < ncol && in_bounds(hb + 8LL * c, 8, sc.n)) ? __ldcs(g8 + c) : make_uint4(0u, 0u, 0u, 0u);      // all-zero bits are 0.0 in both types
+                raw[u] = (c < ncol && in_bounds(hb + 8LL * c, 8, b, e, sc.n)) ? __ldcs(g8 + c) : make_uint4(0u, 0u, 0u, 0u);      // all-zero bits are 0.0 in both types
             }
             float a[8];
 #pragma unroll
@@ -124,11 +124,11 @@ sumsq16_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
                     ((static_cast<double>(a[4]) + static_cast<double>(a[5])) + (static_cast<double>(a[6]) + static_cast<double>(a[7])));
         }
         for (long long i = b + tid; i < hb; i += kThreads) {
-            const double v = in_bounds(i, 1, sc.n) ? static_cast<double>(Pair16<T>::load1(g + i)) : 0.0;
+            const double v = in_bounds(i, 1, b, e, sc.n) ? static_cast<double>(Pair16<T>::load1(g + i)) : 0.0;
             dacc += v * v;
         }
         for (long long i = te + tid; i < e; i += kThreads) {
-            const double v = in_bounds(i, 1, sc.n) ? static_cast<double>(Pair16<T>::load1(g + i)) : 0.0;
+            const double v = in_bounds(i, 1, b, e, sc.n) ? static_cast<double>(Pair16<T>::load1(g + i)) : 0.0;
             dacc += v * v;
         }
 #pragma unroll
@@ -141,7 +141,8 @@ sumsq16_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
 #pragma unroll
             for (int w = 0; w < kThreads / 32; ++w) total += warp_part[parity][w];
             unsigned long long* bins = sc.bins + static_cast<size_t>(buf) * bins_copy_words(sc);
-            bins_add(bins + static_cast<size_t>(sg.layer) * sc.M + m, static_cast<size_t>(sc.K) * sc.M, total);
+            if (scratch_ok(buf, 2) && scratch_ok(static_cast<long long>(sg.layer) * sc.M + m, static_cast<long long>(sc.K) * sc.M))
+                bins_add(bins + static_cast<size_t>(sg.layer) * sc.M + m, static_cast<size_t>(sc.K) * sc.M, total);
         }
     }
     bins_turnover(sc, buf_sm);           // every CTA has had at least one item, hence one barrier after the write
@@ -232,7 +233,7 @@ center_pull16_kernel(MutPtrs x, T* __restrict__ center, const float* __restrict_
 #pragma unroll
             for (int q = 0; q < COLS; ++q) {
                 const int c = c0 + q * kThreads + tid;
-                if (c < ncol && in_bounds(hb + static_cast<long long>(c) * VEC, VEC, n)) {
+                if (c < ncol && in_bounds(hb + static_cast<long long>(c) * VEC, VEC, b, e, n)) {
 #pragma unroll
                     for (int m = 0; m < M; ++m)
                         Words<WORDS>::ld(reinterpret_cast<const T*>(x.p[m]) + hb + static_cast<long long>(c) * VEC, raw[q][m]);
@@ -241,7 +242,7 @@ center_pull16_kernel(MutPtrs x, T* __restrict__ center, const float* __restrict_
 #pragma unroll
             for (int q = 0; q < COLS; ++q) {
                 const int c = c0 + q * kThreads + tid;
-                if (c < ncol && in_bounds(hb + static_cast<long long>(c) * VEC, VEC, n)) {
+                if (c < ncol && in_bounds(hb + static_cast<long long>(c) * VEC, VEC, b, e, n)) {
                     // centre of the column's elements (fp32 FMA chain over the workers)
                     float cc[VEC];
 #pragma unroll
@@ -282,9 +283,9 @@ center_pull16_kernel(MutPtrs x, T* __restrict__ center, const float* __restrict_
             }
         }
         for (long long i = b + tid; i < hb; i += kThreads)
-            if (in_bounds(i, 1, n)) pull16_scalar<T, M>(x, center, w, lambda, oml, i);
+            if (in_bounds(i, 1, b, e, n)) pull16_scalar<T, M>(x, center, w, lambda, oml, i);
         for (long long i = te + tid; i < e; i += kThreads)
-            if (in_bounds(i, 1, n)) pull16_scalar<T, M>(x, center, w, lambda, oml, i);
+            if (in_bounds(i, 1, b, e, n)) pull16_scalar<T, M>(x, center, w, lambda, oml, i);
         item += gridDim.x;
         if (PER_LAYER && item < item_end) first_sg = segs[item];
     }
@@ -314,13 +315,67 @@ center_pull16_generic_kernel(MutPtrs x, T* __restrict__ center, const float* __r
     __syncthreads();
     const float oml = 1.0f - lambda;
     for (long long i = b + threadIdx.x; i < e; i += kThreads) {
-        if (!in_bounds(i, 1, n)) continue;
+        if (!in_bounds(i, 1, b, e, n)) continue;
         float c = w[0] * Pair16<T>::load1(reinterpret_cast<const T*>(x.p[0]) + i);
         for (int m = 1; m < M; ++m) c = fmaf(w[m], Pair16<T>::load1(reinterpret_cast<const T*>(x.p[m]) + i), c);
         if (center) Pair16<T>::store1(center + i, c);
         for (int m = 0; m < M; ++m) {
             T* p = reinterpret_cast<T*>(x.p[m]) + i;
             Pair16<T>::store1(p, fmaf(lambda, c, oml * Pair16<T>::load1(p)));
+        }
+    }
+}
+
+// Proximity step on 16-bit parameters and centre: x_m <- round(fmaf(a, x_C, (1-a) x_m)), fp32 arithmetic on
+// the widened values, one rounding per stored value (a = 0 leaves the workers' bits untouched,
+// a = 1 makes them bit-equal to the centre).  One CTA per flat tile; the centre column (eight
+// elements, 16 bytes) is loaded once and reused for all M workers.
+template <typename T>
+__global__ void __launch_bounds__(kThreads)
+prox16_kernel(MutPtrs x, const T* __restrict__ center, long long n, int tile, float a, int M, int vec_ok)
+{
+    grid_dependency_sync();
+    const long long b = static_cast<long long>(blockIdx.x) * tile;
+    const long long e = min(n, b + tile);
+    const float oma = 1.0f - a;
+    long long hb, te;
+    split_range16(b, e, vec_ok, hb, te);
+    const int ncol = static_cast<int>((te - hb) >> 3);
+    for (int c = threadIdx.x; c < ncol; c += kThreads) {
+        if (!in_bounds(hb + 8LL * c, 8, b, e, n)) continue;
+        float cc[8];
+        unpack8<T>(__ldcs(reinterpret_cast<const uint4*>(center + hb) + c), cc);
+        int m = 0;
+        for (; m + 4 <= M; m += 4) {
+            uint4 raw[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) raw[q] = __ldcs(reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(x.p[m + q]) + hb) + c);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                float v[8];
+                unpack8<T>(raw[q], v);
+#pragma unroll
+                for (int t = 0; t < 8; ++t) v[t] = fmaf(a, cc[t], oma * v[t]);
+                __stcs(reinterpret_cast<uint4*>(reinterpret_cast<T*>(x.p[m + q]) + hb) + c, pack8<T>(v));
+            }
+        }
+        for (; m < M; ++m) {
+            float v[8];
+            unpack8<T>(__ldcs(reinterpret_cast<const uint4*>(reinterpret_cast<const T*>(x.p[m]) + hb) + c), v);
+#pragma unroll
+            for (int t = 0; t < 8; ++t) v[t] = fmaf(a, cc[t], oma * v[t]);
+            __stcs(reinterpret_cast<uint4*>(reinterpret_cast<T*>(x.p[m]) + hb) + c, pack8<T>(v));
+        }
+    }
+    for (int pass = 0; pass < 2; ++pass) {
+        const long long lo = pass ? te : b, hi = pass ? e : hb;
+        for (long long i = lo + threadIdx.x; i < hi; i += kThreads) {
+            if (!in_bounds(i, 1, b, e, n)) continue;
+            const float c = Pair16<T>::load1(center + i);
+            for (int m = 0; m < M; ++m) {
+                T* p = reinterpret_cast<T*>(x.p[m]) + i;
+                Pair16<T>::store1(p, fmaf(a, c, oma * Pair16<T>::load1(p)));
+            }
         }
     }
 }
@@ -332,7 +387,8 @@ copy16_kernel(const T* __restrict__ src, T* __restrict__ dst, long long n)
 {
     grid_dependency_sync();
     const long long stride = static_cast<long long>(gridDim.x) * kThreads;
-    for (long long i = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x; i < n; i += stride) dst[i] = src[i];
+    for (long long i = static_cast<long long>(blockIdx.x) * kThreads + threadIdx.x; i < n; i += stride)
+        if (in_bounds(i, 1, 0, n, n)) dst[i] = src[i];
 }
 
 }  // namespace grawa

@@ -38,9 +38,12 @@ def main():
                 c = torch.empty(cfg.n, dtype=dt, device="cuda")
                 grawa.grawa_step_typed("lgrawa", x, gr, 0.5, cfg.offsets(), c)
                 out["cases"] += 1
-            xs32 = [torch.from_numpy(a).cuda() for a in p]         # proximity step
+            xs32 = [torch.from_numpy(a).cuda() for a in p]         # proximity step, fp32 and 16-bit
             grawa.grawa_prox_step(xs32, torch.from_numpy(g[0]).cuda(), 0.01)
-            out["cases"] += 1
+            grawa.grawa_prox_step_typed([t.bfloat16() for t in xs32], torch.from_numpy(g[0]).cuda().bfloat16(), 0.01)
+            sq = torch.empty(M, dtype=torch.float64, device="cuda")  # the sums of squares on built-in scratch
+            grawa.grawa_sumsq_static([torch.from_numpy(a).cuda() for a in g], sq)
+            out["cases"] += 3
             if M > 1 and cfg.n < 100000:                           # bulk-copy kernel and the host-buffer path
                 grawa.grawa_set_option("pull_variant", 2)
                 gpu_step(grawa, "lgrawa", p, g, 0.5, cfg.offsets())

@@ -1,6 +1,7 @@
 """The bounds-checking debug build of the library (every global access of the streaming kernels
-checked against the vector length, violations counted and skipped) on ragged problems: the
-kernels must not attempt a single out-of-range access.  This stands in for a memory checker."""
+checked against the work item it belongs to and the vector, every scratch index against its
+table; violations counted and skipped) on ragged problems: the kernels must not attempt a single
+access outside their own item.  This stands in for a memory checker."""
 import json
 import os
 import subprocess
@@ -18,7 +19,7 @@ def test_no_out_of_range_access_on_ragged_problems():
                          capture_output=True, text=True, timeout=1200)
     assert res.returncode == 0, res.stdout[-2000:] + res.stderr[-4000:]
     out = json.loads(res.stdout.strip().splitlines()[-1])
-    assert out["selfcheck"] == 3          # the checker itself counts (three planted out-of-range triples)
+    assert out["selfcheck"] == 7          # the checker itself counts (seven planted violations, two clean probes)
     assert out["cases"] > 300
     assert out["violations"] == 0
 
