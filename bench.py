@@ -573,6 +573,9 @@ def small_runs(grawa, args):
         for variant in ("mgrawa", "lgrawa"):
             c = Call(grawa, cfg, variant, "step", "f32", x, g, center)
             eager_ms, _, _ = c.time(1000, 20)
+            # the same C call with its arguments marshalled once (what a C caller pays per step)
+            c.fn = grawa.PreparedStep(variant, x, g, cfg.pull, off, center)
+            prepared_ms, _, _ = c.time(1000, 20)
             stream = torch.cuda.Stream()
             with torch.cuda.stream(stream):
                 c.fn()                                             # builds the plan for this stream
@@ -588,7 +591,7 @@ def small_runs(grawa, args):
                     graph.replay()
                 e1.record()
                 stream.synchronize()
-            out.append({"workload": name, "variant": variant, "M": cfg.M, "n": cfg.n, "eager_us": eager_ms * 1e3,
+            out.append({"workload": name, "variant": variant, "M": cfg.M, "n": cfg.n, "eager_us": eager_ms * 1e3, "eager_prepared_args_us": prepared_ms * 1e3,
                         "graph_replay_us": e0.elapsed_time(e1), "traffic_time_us_at_8TBs": op_bytes(cfg, "step") / 8e12 * 1e6})
             del graph
         del x, g, center

@@ -33,10 +33,11 @@
  *     (so S does not depend on the order in which items finish: bitwise reproducible run to
  *     run); scores and weights in fp64, rounded once to fp32; centre as an fp32
  *     fused-multiply-add chain over m = 0..M-1; pull as fmaf(pull, x_C, (1-pull) * x_m).
- *   - Supported gradient magnitudes: the squares are taken in fp32, so |g| below about 1e-19
- *     contributes zero (a layer of only such values scores exactly 0 and takes the zero-score
- *     rule below) and |g| above about 1.8e19 squares to infinity (a non-finite score, rule
- *     below).  Between those bounds the weights meet the 1e-5 relative contract.
+ *   - Supported gradient magnitudes: the squares are taken in fp32, so the square of |g| below
+ *     about 1e-19 is subnormal (it loses digits) and of |g| below about 3.7e-23 exactly zero (a
+ *     layer of only such values scores 0 and takes the zero-score rule below), and |g| above
+ *     about 1.8e19 squares to infinity (a non-finite score, rule below).  Between 1e-19 and
+ *     1.8e19 the weights meet the 1e-5 relative contract.
  *   - Scores that are exactly zero take the limit of 1/A: inside a normalisation group the Z
  *     workers with zero score get 1/Z each, all others 0.  A non-finite score (NaN/Inf
  *     gradients) gives that worker weight 0, the rest are normalised among themselves (uniform

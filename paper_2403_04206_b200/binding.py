@@ -392,6 +392,31 @@ def grawa_step_from_layer_sums_typed(variant, params, layer_sums, parts, pull, l
                 center_out, weights_out, scores_out, sumsq_out, workspace, stream, n, status_word)
 
 
+class PreparedStep:
+    """A device-buffer step with its arguments marshalled once: calling the object makes the same C call
+    (grawa_step_typed) again on the stream that is current at that moment.  For loops over small models,
+    where building the pointer tables in Python costs as much as the update.  Holds references to the
+    buffers; marshals only, like every function of this module."""
+
+    def __init__(self, variant, params, grads, pull, layer_offsets=None, center_out=None, *, status_word=None):
+        self._keep = (list(params), list(grads), center_out, status_word)
+        self._dt = _dtype_of(list(params) + list(grads) + ([center_out] if center_out is not None else []))
+        self._v = _VARIANTS[variant] if isinstance(variant, str) else int(variant)
+        self._params, self._grads = _ptr_array(params), _ptr_array(grads)
+        self._n, self._M, self._pull = _numel(params[0]), len(params), float(pull)
+        self._off, self._K = _offsets(layer_offsets)
+        self._off_ptr = self._off.ctypes.data if self._off is not None else None
+        self._center = _addr(center_out)
+        self._opt = _options(status_word=status_word)
+        self._fn = library().grawa_step_typed
+
+    def __call__(self, stream=None) -> None:
+        status = self._fn(self._dt, self._v, self._params, self._grads, self._n, self._M, self._pull, self._off_ptr, self._K,
+                          self._center, _byref(self._opt), _stream(stream))
+        if status < 0:
+            raise GrawaError(status, "grawa_step_typed")
+
+
 def grawa_sumsq_static(grads, sumsq_out, *, stream=None, n=None) -> None:
     """Squared gradient norms of the M workers into ``sumsq_out`` (device, M float64) using only
     the scratch array built into the library: for callers whose device memory belongs to another

@@ -130,6 +130,8 @@ struct Plan {
     Segment* d_segs1 = nullptr;      // sum-of-squares items
     Segment* d_segs2 = nullptr;      // per-layer centre+pull items
     bool ws_dirty = false;           // a step failed half-way: the owned scratch is cleared before the next one
+    int elem = 4;                    // bytes per stored element the work lists were cut for
+    std::vector<const void*> seen_ptrs;   // the last pointer table that passed validation (params, grads, centre)
     void* d_ws = nullptr;            // owned scratch (used when the caller passes none)
     WorkspaceLayout ws{};
     void* d_stage = nullptr;         // owned staging for the host-buffer entry point
@@ -166,6 +168,7 @@ static size_t g_timed_used = 0;
 
 // Heap-allocated and never destroyed: at process exit the CUDA runtime may already be gone.
 static auto& g_plans = *new std::map<PlanKey, std::unique_ptr<Plan>>;
+static Plan* g_recent_plan = nullptr;      // plan of the most recent step (fast path of step_entry)
 static auto& g_last_status = *new std::map<std::pair<int, cudaStream_t>, int*>;   // (device, stream) -> status word
 
 // `elem`: bytes per stored element (4, or 2 for 16-bit storage, whose kernels cover twice the
@@ -179,7 +182,7 @@ static grawa_status get_plan(int64_t n, int M, const std::vector<int64_t>& off, 
     if (it != g_plans.end()) { *out = it->second.get(); return GRAWA_OK; }
 
     std::unique_ptr<Plan> p(new Plan);
-    p->device = device; p->stream = stream; p->n = n; p->M = M; p->off = off;
+    p->device = device; p->stream = stream; p->n = n; p->M = M; p->off = off; p->elem = elem;
     p->K = static_cast<int>(off.size()) - 1;
     p->bulk = elem == 4 && wants_bulk(M);
     p->tile1 = g_sumsq_tile * (4 / elem);
@@ -208,23 +211,10 @@ static bool ranges_overlap(const void* a, const void* b, size_t bytes)
     return x < y + bytes && y < x + bytes;
 }
 
-static grawa_status validate(float* const* params, const float* const* grads, int64_t n, int M, float pull,
-                             const int64_t* layer_offsets, int n_layers, const float* center_out,
-                             std::vector<int64_t>* off, size_t elem_size = sizeof(float))
+// Buffers: non-NULL, aligned to their element size, and no overlap visible from the pointer ranges.
+static grawa_status validate_pointers(float* const* params, const float* const* grads, int64_t n, int M,
+                                      const float* center_out, size_t elem_size)
 {
-    if (M < 1 || M > GRAWA_MAX_WORKERS || n < 0 || n_layers < 0) return GRAWA_ERR_INVALID_ARG;
-    if (!(pull >= 0.0f && pull <= 1.0f)) return GRAWA_ERR_INVALID_ARG;   // also rejects NaN
-    if (params == nullptr) return GRAWA_ERR_INVALID_ARG;
-    if ((layer_offsets == nullptr) != (n_layers == 0)) return GRAWA_ERR_INVALID_ARG;
-    if (layer_offsets) {
-        if (layer_offsets[0] != 0 || layer_offsets[n_layers] != n) return GRAWA_ERR_INVALID_ARG;
-        for (int k = 0; k < n_layers; ++k)
-            if (layer_offsets[k + 1] < layer_offsets[k]) return GRAWA_ERR_INVALID_ARG;
-        off->assign(layer_offsets, layer_offsets + n_layers + 1);
-    } else {
-        off->assign({0, n});
-    }
-    if (n == 0) return GRAWA_OK;
     const size_t bytes = static_cast<size_t>(n) * elem_size;
     const uintptr_t amask = elem_size - 1;          // buffers must be aligned to their element size
     for (int m = 0; m < M; ++m) {
@@ -244,6 +234,34 @@ static grawa_status validate(float* const* params, const float* const* grads, in
         }
     }
     return GRAWA_OK;
+}
+
+// Sizes, pull strength and the shape of the layer table (not its contents).
+static grawa_status validate_scalars(const void* params, int64_t n, int M, float pull, const int64_t* layer_offsets, int n_layers)
+{
+    if (M < 1 || M > GRAWA_MAX_WORKERS || n < 0 || n_layers < 0) return GRAWA_ERR_INVALID_ARG;
+    if (!(pull >= 0.0f && pull <= 1.0f)) return GRAWA_ERR_INVALID_ARG;   // also rejects NaN
+    if (params == nullptr) return GRAWA_ERR_INVALID_ARG;
+    if ((layer_offsets == nullptr) != (n_layers == 0)) return GRAWA_ERR_INVALID_ARG;
+    return GRAWA_OK;
+}
+
+static grawa_status validate(float* const* params, const float* const* grads, int64_t n, int M, float pull,
+                             const int64_t* layer_offsets, int n_layers, const float* center_out,
+                             std::vector<int64_t>* off, size_t elem_size = sizeof(float))
+{
+    const grawa_status st = validate_scalars(params, n, M, pull, layer_offsets, n_layers);
+    if (st != GRAWA_OK) return st;
+    if (layer_offsets) {
+        if (layer_offsets[0] != 0 || layer_offsets[n_layers] != n) return GRAWA_ERR_INVALID_ARG;
+        for (int k = 0; k < n_layers; ++k)
+            if (layer_offsets[k + 1] < layer_offsets[k]) return GRAWA_ERR_INVALID_ARG;
+        off->assign(layer_offsets, layer_offsets + n_layers + 1);
+    } else {
+        off->assign({0, n});
+    }
+    if (n == 0) return GRAWA_OK;
+    return validate_pointers(params, grads, n, M, center_out, elem_size);
 }
 
 static inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
@@ -618,14 +636,42 @@ static grawa_status step_entry(int variant, float* const* params, const float* c
 {
     if ((grads == nullptr) == (given.data == nullptr)) return GRAWA_ERR_INVALID_ARG;   // exactly one source of scores
     if (given.parts < 1) return GRAWA_ERR_INVALID_ARG;
-    std::vector<int64_t> off;
-    grawa_status st = validate(params, grads, n, M, pull, layer_offsets, n_layers, center_out, &off,
-                               dtype == 0 ? sizeof(float) : size_t{2});
-    if (st != GRAWA_OK || n == 0) return st;
-    std::lock_guard<std::mutex> lock(g_mutex);
-    Plan* plan = nullptr;
-    st = get_plan(n, M, off, stream, &plan, dtype == 0 ? 4 : 2);
+    const int elem = dtype == 0 ? 4 : 2;
+    grawa_status st = validate_scalars(params, n, M, pull, layer_offsets, n_layers);
     if (st != GRAWA_OK) return st;
+    std::lock_guard<std::mutex> lock(g_mutex);
+    // Fast path of a training loop: the same problem as the call before (device, stream, sizes and a
+    // byte-identical layer table), usually with the same buffers.  The table was validated when the
+    // plan was built and the buffers when they were first seen, so neither is walked again.
+    Plan* plan = g_recent_plan;
+    bool same_problem =
+        n > 0 && plan != nullptr && plan->stream == stream && plan->n == n && plan->M == M && plan->elem == elem &&
+        (layer_offsets ? (plan->K == n_layers && std::memcmp(plan->off.data(), layer_offsets, sizeof(int64_t) * (static_cast<size_t>(n_layers) + 1)) == 0)
+                       : plan->K == 1);
+    if (same_problem) {
+        int device = 0;
+        GRAWA_CUDA_TRY(cudaGetDevice(&device));
+        same_problem = plan->device == device;
+    }
+    if (!same_problem) {
+        std::vector<int64_t> off;
+        st = validate(params, grads, n, M, pull, layer_offsets, n_layers, center_out, &off, static_cast<size_t>(elem));
+        if (st != GRAWA_OK || n == 0) return st;
+        st = get_plan(n, M, off, stream, &plan, elem);
+        if (st != GRAWA_OK) return st;
+        plan->seen_ptrs.clear();
+        g_recent_plan = plan;
+    }
+    // the pointer table: 2M + 1 addresses; byte-identical to the last validated one = nothing to check
+    const void* ptrs[2 * GRAWA_MAX_WORKERS + 1];
+    for (int m = 0; m < M; ++m) { ptrs[m] = params[m]; ptrs[M + m] = grads ? grads[m] : nullptr; }
+    ptrs[2 * M] = center_out;
+    const size_t np = 2 * static_cast<size_t>(M) + 1;
+    if (plan->seen_ptrs.size() != np || std::memcmp(plan->seen_ptrs.data(), ptrs, sizeof(void*) * np) != 0) {
+        st = validate_pointers(params, grads, n, M, center_out, static_cast<size_t>(elem));
+        if (st != GRAWA_OK) return st;
+        plan->seen_ptrs.assign(ptrs, ptrs + np);
+    }
     return enqueue_step(variant, params, grads, given, n, M, pull, center_out, opt, stream, plan, dtype);
 }
 
@@ -1133,6 +1179,7 @@ int grawa_trace_read(uint64_t* rows_out, int max_rows)
 static void clear_plans_locked()
 {
     cudaDeviceSynchronize();
+    g_recent_plan = nullptr;
     g_plans.clear();
     g_last_status.clear();
 }

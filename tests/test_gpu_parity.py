@@ -266,6 +266,32 @@ def test_zero_and_nonfinite_scores_follow_the_stated_policy(grawa):
     assert grawa.grawa_last_step_status() == 0
 
 
+def test_gradient_magnitudes_outside_the_supported_range_take_the_stated_rules(grawa):
+    """The squares are taken in fp32: below |g| of about 1e-19 they are subnormal (fewer and fewer
+    digits), below about 3.7e-23 exactly zero, so a layer of only such gradients sums to zero and takes
+    the zero-score rule (where the float64 oracle still sees norms); a gradient above about 1.8e19
+    squares to infinity and takes the non-finite rule.  The other layers are unaffected and match
+    the oracle."""
+    sizes = [3000, 5000, 7000]
+    off = np.concatenate([[0], np.cumsum(sizes)])
+    cfg = gen.custom_config(sizes, 4, seed=31, log10_sigma=(-2.0, 0.0))
+    p, g = gen.make_inputs(cfg)
+    for m in range(4):
+        g[m][off[1]:off[2]] *= np.float32(1e-25) * (m + 1)       # layer 1: tiny, different per worker
+    res = gpu_step(grawa, "lgrawa", p, g, 0.5, off)
+    ref_beta, _ = oracle.weights(oracle.scores(oracle.sumsq(g, off), "lgrawa"))
+    assert np.all(res["S"][1] == 0) and np.array_equal(res["beta"][1], [0.25] * 4)     # zero-score rule, not the oracle's weights
+    assert not np.allclose(ref_beta[1], 0.25, rtol=0.1)
+    for k in (0, 2):
+        assert np.abs(res["beta"][k] / ref_beta[k] - 1).max() <= 1e-5
+    assert grawa.grawa_last_step_status() == 0
+    g[3][off[2] + 5] = np.float32(3e19)                          # squares to +inf in fp32, finite in float64
+    res = gpu_step(grawa, "lgrawa", p, g, 0.5, off)
+    assert grawa.grawa_last_step_status() == -3
+    assert res["beta"][2][3] == 0 and abs(res["beta"][2][:3].sum() - 1) < 1e-6
+    assert np.isfinite(res["center"].cpu().numpy()).all()
+
+
 # ------------------------------------------------------------------ optional arguments and the other entry points
 
 def test_caller_workspace_and_no_centre(grawa):
