@@ -104,6 +104,13 @@ class ClockSampler:
                         reasons.add(name)
             except Exception:
                 continue
+        if not sm:                                   # a run too short to catch a sample under load: use them all
+            for r in rows:
+                try:
+                    sm.append(float(r[0]))
+                    power.append(float(r[2]))
+                except Exception:
+                    continue
         if sm:
             out["sm_mhz"] = float(np.median(sm))
             out["samples"] = len(sm)
@@ -334,10 +341,14 @@ def whole_job_steps_per_s(world, ms_per_step_max):
 # knob at its default; anything else reports null.
 CAPTURE_ELEMENTS = 14918400
 STORED_CAPTURES = {
-    "center_pull": {"M": 16, "dram_bytes": None, "begin": "// Steps 4-5, register variant", "end": "// Steps 4-5 for any M up to",
-                    "kernel_sha256": None, "host_sha256": None},
-    "sumsq": {"M": 16, "dram_bytes": None, "begin": "// Step 1 (Eq. 3 / Eq. 5): partial", "end": "// Steps 4-5, register variant",
-              "kernel_sha256": None, "host_sha256": None},
+    "center_pull": {"M": 16, "dram_bytes": 955045376 + 958240256, "begin": "// Steps 4-5, register variant",
+                    "end": "// Steps 4-5 for any M up to",
+                    "kernel_sha256": "42e74cf8fd0856f1e1ae61a6b7fcca1c753822a71e1e49fbc04314ba07a2d2df",
+                    "host_sha256": "976696af3f7aa30debde58418a25f3dbeda935d85aad1067614168e0d9f80fcf"},
+    "sumsq": {"M": 16, "dram_bytes": 954845952 + 3118336, "begin": "// Step 1 (Eq. 3 / Eq. 5): partial",
+              "end": "// Steps 4-5, register variant",
+              "kernel_sha256": "993469fab3fdeaec9810faa2aeba3fd6a0af16733b1ebf4da2409a515b82814f",
+              "host_sha256": "976696af3f7aa30debde58418a25f3dbeda935d85aad1067614168e0d9f80fcf"},
 }
 DEFAULT_KNOBS = {"sumsq_tile": 8192, "pull_tile": 0, "pull_variant": 0, "bulk_tile": 0, "sumsq_ctas_per_sm": 0,
                  "pull_prefetch_waves": 3, "sumsq_prefetch_waves": 1,
@@ -670,7 +681,12 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--layers-limit", type=int, default=0, help="use only the first L layers (small profiling captures)")
     ap.add_argument("--option", action="append", default=[], help="library tuning knob, name=value (repeatable)")
+    ap.add_argument("--print-source-hashes", action="store_true",
+                    help="print the hashes that tie a stored ncu capture to the kernel source, and exit")
     args = ap.parse_args()
+    if args.print_source_hashes:
+        print(json.dumps({k: source_hashes(k) for k in STORED_CAPTURES}))
+        return
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
     if args.impl == "reference":
         run_reference(args)
