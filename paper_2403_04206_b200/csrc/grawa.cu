@@ -477,7 +477,10 @@ static cudaError_t launch_finalize(const StepContext& c)
     const bool layered = c.variant == kLgrawa && c.sc.given == nullptr;
     const int warps = kFinThreadsLayered / 32;
     const int grid = layered ? std::max(1, std::min((plan->K + warps - 1) / warps, 4 * plan->sm_count)) : 1;
-    const int block = layered ? kFinThreadsLayered : kFinThreadsFlat;
+    // the one CTA of the other cases: a thread per (layer, worker) row when that fits
+    const int64_t rows = static_cast<int64_t>(plan->K) * c.M;
+    const int flat = static_cast<int>(std::max<int64_t>(128, std::min<int64_t>(kFinThreadsFlat, (rows + 31) / 32 * 32)));
+    const int block = layered ? kFinThreadsLayered : flat;
     return launch_kernel(finalize_kernel, grid, block, c.stream, c.pdl, c.sc);
 }
 

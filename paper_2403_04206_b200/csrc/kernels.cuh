@@ -351,17 +351,20 @@ __device__ __forceinline__ void store_row(const StepScratch& sc, size_t idx, dou
 // ---------------------------------------------------------------------------------------------
 // Steps 2-3: S -> scores -> weights.
 // LGRAWA: one warp per layer, any number of CTAs, no CTA depends on another (Eq. 5-7).
-// MGRAWA / GRAWA: one CTA; thread (p, m) adds worker m's terms of a contiguous run of layers in
-// layer order, thread m adds the runs in order (Eq. 3 / Eq. 2), one warp normalises (Eq. 4).
+// MGRAWA / GRAWA: one CTA; thread (p, m) adds worker m's terms of a contiguous run of layers (one
+// layer when the CTA has a thread per row) in layer order, the runs are added in run order in two
+// levels (Eq. 3 / Eq. 2), one warp normalises (Eq. 4).
 // Every sum has a fixed order.  The status word is rewritten by every launch.
 // ---------------------------------------------------------------------------------------------
 constexpr int kFinThreadsLayered = 256;     // LGRAWA: 8 layers per CTA
-constexpr int kFinThreadsFlat = 1024;       // MGRAWA / GRAWA: the one CTA
+constexpr int kFinThreadsFlat = 1024;       // MGRAWA / GRAWA: the one CTA (at most)
+constexpr int kFinGroupSlots = 512;         // >= ceil(sqrt(P)) * M for every P * M <= 1024, M <= 64
 
 __global__ void __launch_bounds__(kFinThreadsFlat, 1)
 finalize_kernel(StepScratch sc)
 {
     __shared__ double part_sm[kFinThreadsFlat];
+    __shared__ double group_sm[kFinGroupSlots];
     __shared__ double score_sm[kMaxWorkers];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int M = sc.M, K = sc.K;
@@ -428,7 +431,7 @@ finalize_kernel(StepScratch sc)
     }
 
     // MGRAWA / GRAWA (launched as one CTA)
-    const int P = max(1, min((K + 1) / 2, static_cast<int>(blockDim.x) / M));
+    const int P = max(1, min(K, static_cast<int>(blockDim.x) / M));
     const int run = (K + P - 1) / P;
     if (tid < P * M) {
         const int p = tid / M, m = tid - p * M;
@@ -444,9 +447,21 @@ finalize_kernel(StepScratch sc)
         part_sm[tid] = a;
     }
     __syncthreads();
+    // the P runs of a worker are added in two levels, both in run order: G groups of L consecutive runs
+    int G = 1;
+    while (G * G < P) ++G;
+    const int L = (P + G - 1) / G;
+    if (tid < G * M) {
+        const int j = tid / M, m = tid - j * M;
+        const int p1 = min(P, (j + 1) * L);
+        double a = 0.0;
+        for (int p = j * L; p < p1; ++p) a += part_sm[p * M + m];
+        group_sm[tid] = a;
+    }
+    __syncthreads();
     if (tid < M) {
         double a = 0.0;
-        for (int p = 0; p < P; ++p) a += part_sm[p * M + tid];
+        for (int j = 0; j < G; ++j) a += group_sm[j * M + tid];
         if (sc.variant == kGrawa) a = sqrt(a);
         sc.A[static_cast<size_t>(K) * M + tid] = a;
         if (sc.scores_out) sc.scores_out[tid] = a;
