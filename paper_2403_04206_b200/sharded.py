@@ -64,7 +64,8 @@ def _stream_context(stream):
 def sharded_step(variant, params, grads, pull, local_offsets, center_out=None, *, group=None, stream=None):
     """One averaging step on this rank's element range.
 
-    params, grads: this rank's slices of the M replicas (device float32 tensors of j1-j0 elements);
+    params, grads: this rank's slices of the M replicas (device float32, bfloat16 or float16 tensors of
+    j1-j0 elements, all of one type);
     local_offsets: local_layer_table(...) of the range.  Collective: every rank of `group` must call it.
     Everything (the two library calls and the all-gather between them) is enqueued on ``stream``
     (default: torch's current stream).
@@ -76,6 +77,6 @@ def sharded_step(variant, params, grads, pull, local_offsets, center_out=None, *
     K, M = len(local_offsets) - 1, len(params)
     with _stream_context(stream):
         local = torch.empty(K, M, dtype=torch.float64, device=params[0].device)
-        binding.grawa_layer_sumsq(grads, local_offsets, local)
+        binding.grawa_layer_sumsq_typed(grads, local_offsets, local)          # storage type taken from the tensors
         gathered = exchange_layer_sums(local, group)
-        binding.grawa_step_from_layer_sums(variant, params, gathered, world, pull, local_offsets, center_out)
+        binding.grawa_step_from_layer_sums_typed(variant, params, gathered, world, pull, local_offsets, center_out)

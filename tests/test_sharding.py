@@ -142,6 +142,17 @@ def test_sharded_step_through_nccl_with_one_rank():
         assert np.abs(centre.cpu().numpy() - ref["center"]).max() <= tol
         for m in range(cfg.M):
             assert np.abs(x[m].cpu().numpy() - ref["workers"][m]).max() <= tol
+        # bfloat16 replicas through the same call: bit-identical to the unsharded typed step
+        xb = [torch.from_numpy(a).cuda().bfloat16() for a in p]
+        xr = [t.clone() for t in xb]
+        gb = [torch.from_numpy(a).cuda().bfloat16() for a in g]
+        cb, cr = torch.zeros(cfg.n, dtype=torch.bfloat16, device="cuda"), torch.zeros(cfg.n, dtype=torch.bfloat16, device="cuda")
+        sharded.sharded_step("lgrawa", xb, gb, 0.5, sharded.local_layer_table(off, j0, j1), cb)
+        grawa.grawa_step_typed("lgrawa", xr, gb, 0.5, off, cr)
+        torch.cuda.synchronize()
+        assert bool((cb.view(torch.int16) == cr.view(torch.int16)).all())
+        for u, v in zip(xb, xr):
+            assert bool((u.view(torch.int16) == v.view(torch.int16)).all())
         # On a stream that is not the current one, behind work that produces the inputs there: the
         # step (kernels and all-gather) must queue up behind that work, not beside it.
         side = torch.cuda.Stream()
