@@ -186,7 +186,9 @@ static grawa_status get_plan(int64_t n, int M, const std::vector<int64_t>& off, 
     p->K = static_cast<int>(off.size()) - 1;
     p->bulk = elem == 4 && wants_bulk(M);
     p->tile1 = g_sumsq_tile * (4 / elem);
-    p->tile2 = p->bulk ? bulk_tile_for(M) : (g_pull_tile > 0 ? g_pull_tile : pull_pass_elems(std::min(M, kMaxRegWorkers)));
+    p->tile2 = p->bulk ? bulk_tile_for(M)
+               : (g_pull_tile > 0 ? g_pull_tile
+                  : (elem == 2 ? pull16_pass_elems(std::min(M, kMaxRegWorkers)) : pull_pass_elems(std::min(M, kMaxRegWorkers))));
     GRAWA_CUDA_TRY(cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, device));
     std::vector<Segment> s1, s2;
     build_segments(off, p->tile1, kMaxSumsqItemsPerLayer, &s1);
