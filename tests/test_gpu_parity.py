@@ -402,6 +402,28 @@ def test_step_inside_a_cuda_graph(grawa):
             assert bool((u == v).all())
 
 
+def test_prepared_step_makes_the_same_call(grawa):
+    """The step with its arguments marshalled once gives the same bytes as the plain binding call,
+    for fp32 and for 16-bit storage, and keeps doing so when called again."""
+    import torch
+    cfg = gen.CONFIGS["resnet20_cifar"]
+    p, g = inputs("resnet20_cifar")
+    off = cfg.offsets()
+    for dt in (torch.float32, torch.bfloat16):
+        xa = [torch.from_numpy(a).cuda().to(dt) for a in p]
+        xb = [t.clone() for t in xa]
+        gr = [torch.from_numpy(a).cuda().to(dt) for a in g]
+        ca, cb = torch.zeros(cfg.n, dtype=dt, device="cuda"), torch.zeros(cfg.n, dtype=dt, device="cuda")
+        word = torch.full((1,), 5, dtype=torch.int32, device="cuda")
+        step = grawa.PreparedStep("lgrawa", xb, gr, 0.5, off, cb, status_word=word)
+        for _ in range(3):
+            grawa.grawa_step_typed("lgrawa", xa, gr, 0.5, off, ca)
+            step()
+            torch.cuda.synchronize()
+            assert bool((ca == cb).all()) and all(bool((u == v).all()) for u, v in zip(xa, xb))
+            assert int(word.item()) == 0
+
+
 # ------------------------------------------------------------------ the bulk-copy centre+pull kernel
 
 @pytest.fixture

@@ -53,3 +53,41 @@ def test_reference_arm_line_has_the_contract_keys():
     assert line["cpu_baseline"]["kind"] == "oracle" and line["cpu_baseline"]["cores"] == 1
     assert line["e2e"]["h2d_bytes_per_step"] == 0 and line["e2e"]["d2h_bytes_per_step"] == 0
     assert line["higher_is_better"] is True and line["config"]["workload"].startswith("toy10")
+
+
+def test_both_arms_describe_the_workload_with_one_function():
+    """The reference arm's `config` equals the CUDA arm's key by key (one GPU, fp32 step)."""
+    import bench
+    import gen
+    cfg = gen.CONFIGS["toy10"]
+    a = bench.describe(cfg, "lgrawa", "step", "f32", 1)
+    assert a["workload"].startswith("toy10") and a["parallelism"] == "single GPU"
+    assert a["algorithmic_bytes_per_step"] == (3 * cfg.M + 1) * 4 * cfg.n == cfg.algorithmic_bytes()
+    assert bench.op_bytes(cfg, "prox") == (2 * cfg.M + 1) * 4 * cfg.n == bench.op_bytes(cfg, "from_norms")
+    assert bench.op_bytes(cfg, "step", "bf16") * 2 == bench.op_bytes(cfg, "step", "f32")
+    assert bench.describe(cfg, "lgrawa", "step", "f32", 4)["parallelism"] == "replicas only"
+    assert bench.describe(cfg, "lgrawa", "step", "f32", 4, sharded=True)["parallelism"] == "element-range sharded"
+
+
+def test_stored_ncu_traffic_is_quoted_only_for_the_captured_kernel_and_default_knobs():
+    import bench
+    import gen
+
+    class Knobs:
+        def __init__(self, **changed):
+            self.v = dict(bench.DEFAULT_KNOBS, **changed)
+
+        def grawa_get_option(self, name):
+            return self.v[name]
+
+    vit, vgg = gen.CONFIGS["vit_b16"], gen.CONFIGS["vgg16"]
+    for which in bench.STORED_CAPTURES:
+        kernel_hash, host_hash = bench.source_hashes(which)
+        cap = bench.STORED_CAPTURES[which]
+        same_source = (kernel_hash, host_hash) == (cap["kernel_sha256"], cap["host_sha256"])
+        got = bench.stored_traffic(Knobs(), which, vit)
+        assert (got is not None) == (same_source and cap["dram_bytes"] is not None)
+        if got is not None:
+            assert abs(got / (cap["dram_bytes"] / bench.CAPTURE_ELEMENTS * vit.n) - 1) < 1e-12
+        assert bench.stored_traffic(Knobs(), which, vgg) is None                      # another M
+        assert bench.stored_traffic(Knobs(pull_variant=2), which, vit) is None       # a knob off its default
