@@ -448,7 +448,7 @@ def run_cuda(args):
 
     # ---- one problem cut by element range over the ranks (with one rank: the same step through the sharded path)
     sharded_out = None
-    if args.sharded and op == "step" and dtype == "f32":
+    if (args.sharded or world > 1) and op == "step" and dtype == "f32":      # always recorded by a multi-rank run
         sharded_out = run_sharded(grawa, cfg, variant, args, world, rank, peak, barrier, x, g, center)
 
     ms_max, e2e_ms_max = max_over_ranks([ms, e2e_ms if e2e_ms is not None else 0.0], world, "cuda")
@@ -678,7 +678,8 @@ def main():
     ap.add_argument("--variant", default=DEFAULT_VARIANT, choices=["lgrawa", "mgrawa", "grawa"])
     ap.add_argument("--op", default="step", choices=["step", "prox", "from_norms"])
     ap.add_argument("--dtype", default="f32", choices=["f32", "bf16", "f16"], help="storage of parameters, gradients and centre")
-    ap.add_argument("--sharded", action="store_true", help="also time one problem cut by element range over the ranks")
+    ap.add_argument("--sharded", action="store_true",
+                    help="also time one problem cut by element range over the ranks (always on with more than one rank)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--headline-only", action="store_true", help="skip the short runs of the other workloads and calls")
     ap.add_argument("--no-cpu-baseline", action="store_true")
