@@ -402,6 +402,49 @@ def test_step_inside_a_cuda_graph(grawa):
             assert bool((u == v).all())
 
 
+def test_captured_step_with_a_callers_workspace_and_status_word(grawa):
+    """A caller's scratch buffer and status word inside a captured step: the part of the scratch that
+    carries state is cleared by a node of the graph, so replays start clean whatever the buffer held,
+    and the status word is rewritten by every replay."""
+    import torch
+    cfg = gen.custom_config([10, 50000, 0, 3, 120000, 777], 6, seed=77, log10_sigma=(-2.0, 0.0))
+    p, g = gen.make_inputs(cfg)
+    off = cfg.offsets()
+    ref = {v: gpu_step(grawa, v, p, g, 0.5, off) for v in ("lgrawa", "mgrawa")}
+    need = grawa.grawa_workspace_bytes(cfg.n, cfg.M, off)
+    ws = torch.empty(need, dtype=torch.uint8, device="cuda")
+    word = torch.zeros(1, dtype=torch.int32, device="cuda")
+    stream = torch.cuda.Stream()
+    for variant, fn in (("lgrawa", grawa.grawa_lgrawa_step), ("mgrawa", grawa.grawa_mgrawa_step)):
+        x, gr = to_device(p), to_device(g)
+        center = torch.empty(cfg.n, device="cuda")
+        with torch.cuda.stream(stream):
+            fn(x, gr, 0.5, off, center, workspace=ws, status_word=word)        # builds the plan for this stream
+            stream.synchronize()
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph, stream=stream):
+                fn(x, gr, 0.5, off, center, workspace=ws, status_word=word, stream=torch.cuda.current_stream())
+        for rep in range(4):
+            for t, a in zip(x, p):
+                t.copy_(torch.from_numpy(a))
+            ws.fill_(0xFF if rep % 2 else 0x5A)          # whatever the caller did with its buffer in between
+            word.fill_(9)
+            if rep == 2:
+                gr[1][off[1] + 3] = float("nan")         # this replay meets a non-finite score
+            torch.cuda.synchronize()
+            graph.replay()
+            torch.cuda.synchronize()
+            if rep == 2:
+                assert int(word.item()) == 1
+                gr[1].copy_(torch.from_numpy(g[1]))
+                continue
+            assert int(word.item()) == 0
+            assert bool((center == ref[variant]["center"]).all())
+            for u, v in zip(x, ref[variant]["workers"]):
+                assert bool((u == v).all())
+        del graph
+
+
 def test_prepared_step_makes_the_same_call(grawa):
     """The step with its arguments marshalled once gives the same bytes as the plain binding call,
     for fp32 and for 16-bit storage, and keeps doing so when called again."""
