@@ -337,24 +337,31 @@ def whole_job_steps_per_s(world, ms_per_step_max):
 # DRAM bytes per element of one launch, from stored ncu captures of a smaller case of the same kernel
 # (first 28 layers of the ViT-B/16 table, 14 918 400 elements, M = 16), scaled to a full launch by the
 # number of elements.  A capture is only quoted for the kernel source and launch code it was taken
-# from (hashes of the kernel's text in csrc/kernels.cuh and of the function that launches it in csrc/grawa.cu) and with every tuning
+# from (hashes of the kernel's code in csrc/kernels.cuh and of the function that launches it in csrc/grawa.cu,
+# comments and blank lines left out) and with every tuning
 # knob at its default; anything else reports null.
 CAPTURE_ELEMENTS = 14918400
 STORED_CAPTURES = {
     "center_pull": {"M": 16, "dram_bytes": 955045376 + 958240256, "begin": "// Steps 4-5, register variant",
                     "end": "// Steps 4-5 for any M up to",
                     "host_begin": "static grawa_status enqueue_center_pull(StepContext", "host_end": "// Given scores of a step",
-                    "kernel_sha256": "42e74cf8fd0856f1e1ae61a6b7fcca1c753822a71e1e49fbc04314ba07a2d2df",
-                    "host_sha256": "3033d59ca0bf5efadef8458dde4ff4d33b566e9bc50fde50ae50cea2d99e7047"},
-    "sumsq": {"M": 16, "dram_bytes": 954845952 + 3118336, "begin": "// Step 1 (Eq. 3 / Eq. 5): partial",
+                    "kernel_sha256": "9aa1cd15bd94e316e2a45778645f33881e36eaed5ee35a7f1b272d01f6475272",
+                    "host_sha256": "3da8ac05f8a7f1338e0f94cc8aaec33818f4bbe64ec93fb725b53e58e6c35fda"},
+    "sumsq": {"M": 16, "dram_bytes": 954845952 + 3118336, "begin": "// Step 1 (Eq. 3 / Eq. 5):",
               "end": "// Steps 4-5, register variant",
               "host_begin": "static grawa_status enqueue_weights_launches(StepContext& c)\n", "host_end": "// Steps 4-5 on 16-bit storage",
-              "kernel_sha256": "993469fab3fdeaec9810faa2aeba3fd6a0af16733b1ebf4da2409a515b82814f",
-              "host_sha256": "1f1bcbced245b07e7d2ae229eee47a9e71a3b977fc88321a3f678f941486c622"},
+              "kernel_sha256": "6c8fcdcd2927db90fe40fdbb204bf18a7a4757f76906c7670ab4625309856fa1",
+              "host_sha256": "d4e501bd1b39f7af71d29a7670c0fa21c05eabf6517be8608e100ac96bc95406"},
 }
 DEFAULT_KNOBS = {"sumsq_tile": 8192, "pull_tile": 0, "pull_variant": 0, "bulk_tile": 0, "sumsq_ctas_per_sm": 0,
                  "pull_prefetch_waves": 3, "sumsq_prefetch_waves": 1,
                  "pull_ctas_per_sm": 0, "dependent_launch": 1, "pull_preload": 1}
+
+
+def code_only(text):
+    """Source text without `//` comments, blank lines and indentation: what a hash of the code should see."""
+    lines = (line.split("//")[0].strip() for line in text.splitlines())
+    return "\n".join(line for line in lines if line)
 
 
 def source_hashes(which):
@@ -366,7 +373,7 @@ def source_hashes(which):
         host = host[host.index(cap["host_begin"]):host.index(cap["host_end"])]      # the code that launches this kernel
     except (OSError, ValueError):
         return None, None
-    return hashlib.sha256(region.encode()).hexdigest(), hashlib.sha256(host.encode()).hexdigest()
+    return hashlib.sha256(code_only(region).encode()).hexdigest(), hashlib.sha256(code_only(host).encode()).hexdigest()
 
 
 def stored_traffic(grawa, which, cfg):

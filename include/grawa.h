@@ -349,8 +349,8 @@ int64_t grawa_get_option(const char *name);
 /* Number of kernels this library has launched in the calling process since it was loaded. */
 int64_t grawa_launch_count(void);
 
-/* Sums, in milliseconds, of the device time of the three phases (sum-of-squares kernel; partial
- * reduction + scores + weights kernel; centre+pull kernel) over the steps enqueued while
+/* Sums, in milliseconds, of the device time of the three phases (sum-of-squares kernel; scores +
+ * weights kernel; centre+pull kernel) over the steps enqueued while
  * "kernel_timing" was 1 since the previous call, and the number of those steps.  Any output
  * pointer may be NULL.  Synchronises the device. */
 grawa_status grawa_collect_kernel_times(double *sumsq_ms, double *finalize_ms, double *center_pull_ms,

@@ -71,8 +71,8 @@ static int64_t bulk_tile_for(int M)
 
 // ------------------------------------------------------------------ work list
 // Tile used inside one layer: `tile`, doubled until the layer has at most `max_items` items (0 =
-// no limit).  Keeps the number of partial sums of a huge layer small enough for the one CTA that
-// adds them up, without giving up the fine grain that balances the many small layers.
+// no limit).  Bounds the number of atomic additions that meet on one row of exact sums for a huge
+// layer, without giving up the fine grain that balances the many small layers.
 static int64_t layer_tile(int64_t layer_elems, int64_t tile, int64_t max_items)
 {
     int64_t t = tile;

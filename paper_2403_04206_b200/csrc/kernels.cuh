@@ -492,10 +492,11 @@ finalize_kernel(StepScratch sc)
 }
 
 // ---------------------------------------------------------------------------------------------
-// Step 1 (Eq. 3 / Eq. 5): partial[m][s] = sum of g_m[j]^2 over segment s.  Work items are the
+// Step 1 (Eq. 3 / Eq. 5): S[k][m] += sum of g_m[j]^2 over segment s of layer k.  Work items are the
 // (worker, segment) pairs, worker-major; CTA b takes items b, b + gridDim.x, ...  fp32 squares
-// are accumulated in runs of UNROLL terms per accumulator and the runs are combined in fp64; the
-// order depends only on the item, never on the grid, so results are reproducible.
+// are accumulated in runs of UNROLL terms per accumulator, the runs are combined in fp64 in an order
+// that depends only on the item, and the item's sum is added exactly (integer digits) to its row:
+// the result does not depend on the grid or on the order in which items finish.
 // ---------------------------------------------------------------------------------------------
 // Six CTAs per SM (at most 42 registers): measured 1.4x faster than four on the large workloads.
 template <int UNROLL>
