@@ -337,6 +337,9 @@ int grawa_trace_read(uint64_t *rows_out, int max_rows);
  *   "pull_prefetch_waves", "sumsq_prefetch_waves" (0..8; defaults 3 and 1) on short steps the CTAs
  *                  that are resident when a kernel starts hint the data of the items that many
  *                  grid-fuls further on into L2 while they wait for the kernel in front; 0 = off.
+ *   "pull16_staged" 1 (default) = on 16-bit storage with 5..16 workers the centre+pull kernel stages
+ *                  its columns through shared memory (per-thread asynchronous 16-byte copies);
+ *                  0 = the register kernel for every worker count.  Drops the cached plans.
  *   "sumsq_ctas_per_sm", "pull_ctas_per_sm" (0..32) CTAs per SM of the grid that streams
  *                  through the work items of the sum-of-squares / centre+pull kernel;
  *                  0 = one CTA per work item.

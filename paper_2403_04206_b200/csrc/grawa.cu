@@ -32,6 +32,7 @@ static int64_t g_bulk_tile = 0;           // 0 = chosen from M so that at least 
 static int64_t g_kernel_timing = 0;
 static int64_t g_pdl = 1;
 static int64_t g_pull_preload = 1;
+static int64_t g_pull16_staged = 1;         // 16-bit storage, 5..16 workers: shared-memory staged kernel (1) or register kernel (0)
 static int64_t g_pull_prefetch_waves = 3;
 static int64_t g_sumsq_prefetch_waves = 1;
 static int64_t g_sumsq_ctas_per_sm = 0;   // 0 = one CTA per work item
@@ -188,7 +189,8 @@ static grawa_status get_plan(int64_t n, int M, const std::vector<int64_t>& off, 
     p->tile1 = g_sumsq_tile * (4 / elem);
     p->tile2 = p->bulk ? bulk_tile_for(M)
                : (g_pull_tile > 0 ? g_pull_tile
-                  : (elem == 2 ? pull16_pass_elems(std::min(M, kMaxRegWorkers)) : pull_pass_elems(std::min(M, kMaxRegWorkers))));
+                  : (elem == 2 ? ((M > 4 && g_pull16_staged) ? pull16s_pass_elems(std::min(M, kMaxRegWorkers)) : pull16_pass_elems(std::min(M, kMaxRegWorkers)))
+                               : pull_pass_elems(std::min(M, kMaxRegWorkers))));
     GRAWA_CUDA_TRY(cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, device));
     std::vector<Segment> s1, s2;
     build_segments(off, p->tile1, kMaxSumsqItemsPerLayer, &s1);
@@ -394,6 +396,38 @@ struct CenterPull16Dispatch<T, 1> {
     }
 };
 
+// 16-bit storage, 5..16 aligned workers: columns staged through shared memory by per-thread asynchronous copies.
+template <typename T, int M>
+static cudaError_t launch_center_pull16_staged(bool per_layer, int grid, int item_begin, int item_end, cudaStream_t stream, bool pdl,
+                                               const MutPtrs& x, T* center, const float* beta, const Segment* segs, long long n,
+                                               int tile, float pull, int preload)
+{
+    const size_t smem = sizeof(uint4) * static_cast<size_t>(M) * kThreads * pull16s_cols(M);
+    auto kernel = per_layer ? center_pull16_staged_kernel<T, M, true> : center_pull16_staged_kernel<T, M, false>;
+    const cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem));
+    if (err != cudaSuccess) return err;
+    return launch_kernel_smem(kernel, grid, kThreads, smem, stream, pdl, x, center, beta, segs, item_begin, item_end, n, tile, pull,
+                              preload);
+}
+
+template <typename T, int M>
+struct CenterPull16StagedDispatch {
+    template <typename... A>
+    static cudaError_t run(int m, A&&... a)
+    {
+        if (m == M) return launch_center_pull16_staged<T, M>(static_cast<A&&>(a)...);
+        return CenterPull16StagedDispatch<T, M - 1>::run(m, static_cast<A&&>(a)...);
+    }
+};
+template <typename T>
+struct CenterPull16StagedDispatch<T, 4> {
+    template <typename... A>
+    static cudaError_t run(int, A&&...)
+    {
+        return cudaErrorInvalidValue;
+    }
+};
+
 // Device pointers and launch facts of one step, resolved once from the plan and the options.
 struct StepContext {
     Plan* plan = nullptr;
@@ -508,8 +542,8 @@ static grawa_status enqueue_weights_launches(StepContext& c)
     const int grid1 = g_sumsq_ctas_per_sm > 0
                           ? static_cast<int>(std::min<int64_t>(items1, g_sumsq_ctas_per_sm * plan->sm_count)) : items1;
     const int vg = c.vec_g ? 1 : 0;
-    c.sc.prefetch_stride = 6 * plan->sm_count;           // CTAs resident at the start of the kernel
-    c.sc.prefetch_waves = (c.dtype == 0 && grid1 <= 64 * c.sc.prefetch_stride) ? static_cast<int>(g_sumsq_prefetch_waves) : 0;
+    c.sc.prefetch_stride = (c.dtype == 0 ? 6 : 5) * plan->sm_count;           // CTAs resident at the start of the kernel
+    c.sc.prefetch_waves = (grid1 <= 64 * c.sc.prefetch_stride) ? static_cast<int>(g_sumsq_prefetch_waves) : 0;
     if (c.dtype == 1)
         GRAWA_CUDA_TRY(launch_kernel(sumsq16_kernel<__nv_bfloat16, 8>, grid1, kThreads, c.stream, c.pdl, c.gp, c.sc, items1, vg));
     else if (c.dtype == 2)
@@ -532,7 +566,11 @@ static grawa_status enqueue_center_pull16_t(StepContext& c, int item_begin, int 
     const int grid = item_end - item_begin;
     const int tile = static_cast<int>(plan->tile2);
     T* center = reinterpret_cast<T*>(c.center);
-    if (c.vec_x && M <= kMaxRegWorkers) {
+    if (c.vec_x && M > 4 && M <= kMaxRegWorkers && g_pull16_staged) {
+        GRAWA_CUDA_TRY((CenterPull16StagedDispatch<T, kMaxRegWorkers>::run(M, per_layer, grid, item_begin, item_end, c.stream, c.pdl,
+                                                                           c.xp, center, c.sc.beta, plan->d_segs2, c.n, tile, c.pull,
+                                                                           (c.preload && g_pull_preload) ? 1 : 0)));
+    } else if (c.vec_x && M <= kMaxRegWorkers) {
         GRAWA_CUDA_TRY((CenterPull16Dispatch<T, kMaxRegWorkers>::run(M, per_layer, grid, item_begin, item_end, c.stream, c.pdl, c.xp,
                                                                      center, c.sc.beta, plan->d_segs2, c.n, tile, c.pull)));
     } else {
@@ -1234,6 +1272,11 @@ grawa_status grawa_set_option(const char* name, int64_t value)
         g_pull_preload = value;
         return GRAWA_OK;
     }
+    if (std::strcmp(name, "pull16_staged") == 0) {
+        if (value < 0 || value > 1) return GRAWA_ERR_INVALID_ARG;
+        if (value != g_pull16_staged) { g_pull16_staged = value; clear_plans_locked(); }
+        return GRAWA_OK;
+    }
     if (std::strcmp(name, "sumsq_ctas_per_sm") == 0 || std::strcmp(name, "pull_ctas_per_sm") == 0) {
         if (value < 0 || value > 32) return GRAWA_ERR_INVALID_ARG;
         (name[0] == 's' ? g_sumsq_ctas_per_sm : g_pull_ctas_per_sm) = value;
@@ -1253,6 +1296,7 @@ int64_t grawa_get_option(const char* name)
     if (std::strcmp(name, "kernel_timing") == 0) return g_kernel_timing;
     if (std::strcmp(name, "dependent_launch") == 0) return g_pdl;
     if (std::strcmp(name, "pull_preload") == 0) return g_pull_preload;
+    if (std::strcmp(name, "pull16_staged") == 0) return g_pull16_staged;
     if (std::strcmp(name, "pull_prefetch_waves") == 0) return g_pull_prefetch_waves;
     if (std::strcmp(name, "sumsq_prefetch_waves") == 0) return g_sumsq_prefetch_waves;
     if (std::strcmp(name, "sumsq_ctas_per_sm") == 0) return g_sumsq_ctas_per_sm;

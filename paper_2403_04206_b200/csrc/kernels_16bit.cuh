@@ -74,7 +74,7 @@ __device__ __forceinline__ void split_range16(long long b, long long e, int vec_
 // a thread's 16-byte load carries 8 elements, each with its own fp32 accumulator.
 template <typename T, int UNROLL>
 __global__ void __launch_bounds__(kThreads, 5)
-sumsq16_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
+sumsq16_kernel(const __grid_constant__ ConstPtrs grads, StepScratch sc, int items, int vec_ok)
 {
     __shared__ double warp_part[2][kThreads / 32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -82,6 +82,19 @@ sumsq16_kernel(ConstPtrs grads, StepScratch sc, int items, int vec_ok)
     // the work list belongs to the plan, not to the kernel before this one: fetch the first item early
     Segment first_sg = Segment{0, 0, 0};
     if (static_cast<int>(blockIdx.x) < items) first_sg = sc.segs[blockIdx.x % C];
+    // L2 hints for the items further on, on short problems (see sumsq_kernel)
+    if (static_cast<int>(blockIdx.x) < sc.prefetch_stride && tid < sc.prefetch_waves) {
+        const long long it = blockIdx.x + static_cast<long long>(tid + 1) * sc.prefetch_stride;
+        if (it < items) {
+            const int pm = static_cast<int>(it / C);
+            const Segment sg = sc.segs[it - static_cast<long long>(pm) * C];
+            long long phb, pte;
+            split_range16(sg.begin, sg.begin + sg.len, vec_ok, phb, pte);
+            const unsigned bytes = static_cast<unsigned>(pte - phb) * 2u;         // a multiple of 16
+            if (bytes > 0 && in_bounds(phb, pte - phb, sg.begin, sg.begin + sg.len, sc.n))
+                prefetch_l2(reinterpret_cast<const T*>(grads.p[pm]) + phb, bytes);
+        }
+    }
     grid_dependency_sync();
     // Which copy of the digit rows to add into: needed only by thread 0 when an item is done, and by
     // everybody after the last item; thread 0 fetches it now and hands it on through shared memory,
@@ -177,7 +190,7 @@ template <> struct Words<2> {
 };
 
 template <typename T, int M>
-__device__ __forceinline__ void pull16_scalar(const MutPtrs& x, T* center, const float (&w)[M], float lambda, float oml,
+__device__ __forceinline__ void pull16_scalar(const MutPtrs& x, T* center, const float* w, float lambda, float oml,
                                               long long i)
 {
     float v[M];
@@ -287,6 +300,123 @@ center_pull16_kernel(MutPtrs x, T* __restrict__ center, const float* __restrict_
             if (in_bounds(i, 1, b, e, n)) pull16_scalar<T, M>(x, center, w, lambda, oml, i);
         item += gridDim.x;
         if (PER_LAYER && item < item_end) first_sg = segs[item];
+    }
+}
+
+// Steps 4-5 on 16-bit parameters for 5..16 workers.  Sixteen 16-byte columns (the same bytes in flight
+// as the fp32 kernel; two columns of up to eight workers) do not fit in registers next to their
+// arithmetic, so every thread copies its columns of each worker straight from global to its own slots
+// of shared memory with asynchronous
+// 16-byte copies (`cp.async`, no registers held while they fly, L1 bypassed), waits for its own
+// copies only (no CTA barrier: a thread reads nothing but what it copied), and then walks the
+// workers twice from shared memory: the fp32 FMA chain of the centre, then the pull and one
+// 16-byte store per worker.  Same arithmetic and rounding as center_pull16_kernel.  Shared memory:
+// COLS x M x 256 x 16 bytes (64 KB at M = 16 and at M = 8), three CTAs per SM.
+__host__ __device__ constexpr int pull16s_cols(int M) { return (M <= 8) ? 2 : 1; }     // 16-byte columns per thread in flight
+__host__ __device__ constexpr int pull16s_pass_elems(int M) { return kThreads * 8 * pull16s_cols(M); }
+
+__device__ __forceinline__ void cp_async16(void* smem_dst, const void* gsrc)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(static_cast<unsigned>(__cvta_generic_to_shared(smem_dst))), "l"(gsrc)
+                 : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all()
+{
+    asm volatile("cp.async.commit_group;\n\tcp.async.wait_group 0;" ::: "memory");
+}
+
+template <typename T, int M, bool PER_LAYER>
+__global__ void __launch_bounds__(kThreads, 3)
+center_pull16_staged_kernel(MutPtrs x, T* __restrict__ center, const float* __restrict__ beta, const Segment* __restrict__ segs,
+                            int item_begin, int item_end, long long n, int tile, float lambda, int preload)
+{
+    extern __shared__ __align__(16) uint4 stage16[];          // [COLS][M][kThreads]
+    constexpr int COLS = pull16s_cols(M);
+    const int tid = threadIdx.x;
+    int item = item_begin + blockIdx.x;
+    int layer = 0, ncol = 0;
+    long long b = 0, e = 0, hb = 0, te = 0;
+    auto locate = [&](int it) {
+        if (PER_LAYER) {
+            const Segment sg = segs[it];
+            b = sg.begin;
+            e = b + sg.len;
+            layer = sg.layer;
+        } else {
+            b = static_cast<long long>(it) * tile;
+            e = min(n, b + tile);
+        }
+        split_range16(b, e, 1, hb, te);
+        ncol = static_cast<int>((te - hb) >> 3);
+    };
+    auto fetch = [&](int c0) {                                  // this thread's columns of every worker -> shared memory
+#pragma unroll
+        for (int q = 0; q < COLS; ++q) {
+            const int c = c0 + q * kThreads + tid;
+            if (c < ncol && in_bounds(hb + 8LL * c, 8, b, e, n)) {
+#pragma unroll
+                for (int m = 0; m < M; ++m)
+                    cp_async16(&stage16[(q * M + m) * kThreads + tid], reinterpret_cast<const T*>(x.p[m]) + hb + 8LL * c);
+            }
+        }
+    };
+    bool fetched = false;
+    if (item < item_end) {
+        locate(item);
+        if (preload) {                                          // see center_pull_kernel for when this is valid
+            fetch(0);
+            fetched = true;
+        }
+    }
+    grid_dependency_sync();
+    const float oml = 1.0f - lambda;
+    __shared__ float w[M];                                      // the item's weights, read where they are used
+    while (item < item_end) {
+        __syncthreads();                                        // nobody still reads the previous item's weights
+        if (tid < M) w[tid] = PER_LAYER ? beta[static_cast<size_t>(layer) * M + tid] : beta[tid];
+        __syncthreads();
+        for (int c0 = 0; c0 < ncol; c0 += kThreads * COLS) {
+            if (!fetched) fetch(c0);
+            fetched = false;
+            cp_async_wait_all();
+#pragma unroll
+            for (int q = 0; q < COLS; ++q) {
+                const int c = c0 + q * kThreads + tid;
+                if (c >= ncol || !in_bounds(hb + 8LL * c, 8, b, e, n)) continue;
+                const uint4* col = stage16 + q * M * kThreads + tid;
+                float cc[8];
+                {
+                    float v[8];
+                    unpack8<T>(col[0], v);
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) cc[t] = w[0] * v[t];
+                }
+#pragma unroll 4
+                for (int m = 1; m < M; ++m) {
+                    float v[8];
+                    unpack8<T>(col[m * kThreads], v);
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) cc[t] = fmaf(w[m], v[t], cc[t]);
+                }
+                if (center) __stcs(reinterpret_cast<uint4*>(center + hb) + c, pack8<T>(cc));
+#pragma unroll 4
+                for (int m = 0; m < M; ++m) {
+                    float v[8];
+                    unpack8<T>(col[m * kThreads], v);
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) v[t] = fmaf(lambda, cc[t], oml * v[t]);
+                    __stcs(reinterpret_cast<uint4*>(reinterpret_cast<T*>(x.p[m]) + hb) + c, pack8<T>(v));
+                }
+            }
+        }
+        fetched = false;
+        cp_async_wait_all();                                    // an early fetch of an item without a vector body
+        for (long long i = b + tid; i < hb; i += kThreads)
+            if (in_bounds(i, 1, b, e, n)) pull16_scalar<T, M>(x, center, w, lambda, oml, i);
+        for (long long i = te + tid; i < e; i += kThreads)
+            if (in_bounds(i, 1, b, e, n)) pull16_scalar<T, M>(x, center, w, lambda, oml, i);
+        item += gridDim.x;
+        if (item < item_end) locate(item);
     }
 }
 
