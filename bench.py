@@ -185,18 +185,13 @@ class Call:
             x, g, center = [t.to(tdt) for t in x], [t.to(tdt) for t in g], center.to(tdt)
         self.x, self.g, self.center = x, g, center
         if op == "prox":
-            if dtype != "f32":
-                raise SystemExit("the proximity step runs on fp32 storage")
-            self.fn = lambda: grawa.grawa_prox_step(x, center, 0.05 / 16)        # mu / tau of the paper's grid
+            self.fn = lambda: grawa.grawa_prox_step_typed(x, center, 0.05 / 16)  # mu / tau of the paper's grid
         elif op == "from_norms":
-            if dtype != "f32":
-                raise SystemExit("the step from given norms runs on fp32 storage")
-            K, G = cfg.K, (cfg.K if variant == "lgrawa" else 1)
-            norms = torch.empty(K * cfg.M, dtype=torch.float64, device="cuda")
-            grawa.grawa_lgrawa_step(x, g, 0.0, off, None, scores_out=norms)      # per-layer norms, workers untouched
+            norms = torch.empty(cfg.K * cfg.M, dtype=torch.float64, device="cuda")
+            grawa.grawa_step_typed("lgrawa", x, g, 0.0, off, None, scores_out=norms)   # per-layer norms, workers untouched
             torch.cuda.synchronize()
             self.norms = norms
-            self.fn = lambda: grawa.grawa_step_from_layer_norms(variant, x, norms, cfg.pull, off, center)
+            self.fn = lambda: grawa.grawa_step_from_layer_norms_typed(variant, x, norms, cfg.pull, off, center)
         elif dtype == "f32":
             step = {"lgrawa": grawa.grawa_lgrawa_step, "mgrawa": grawa.grawa_mgrawa_step, "grawa": grawa.grawa_grawa_step}[variant]
             self.fn = lambda: step(x, g, cfg.pull, off, center)
@@ -546,6 +541,10 @@ def side_ops(grawa, cfg, variant, x, g, center, args, peak):
     out.append(dict(op="step", variant=variant, storage="bf16", workload=cfg.name, steps=steps,
                     algorithmic_bytes=op_bytes(cfg, "step", "bf16"), kernels=kernel_table(cfg, "bf16", ph, peak),
                     **rates(op_bytes(cfg, "step", "bf16"), ms, peak)))
+    c.op, c.fn = "prox", (lambda xs=c.x, cc=c.center: grawa.grawa_prox_step_typed(xs, cc, 0.05 / 16))   # same bf16 buffers
+    ms, _, _ = c.time(steps, 3)
+    out.append(dict(op="prox", storage="bf16", workload=cfg.name, steps=steps, algorithmic_bytes=op_bytes(cfg, "prox", "bf16"),
+                    **rates(op_bytes(cfg, "prox", "bf16"), ms, peak)))
     del c
     torch.cuda.empty_cache()
     return out
