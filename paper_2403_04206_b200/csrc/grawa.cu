@@ -542,7 +542,7 @@ static grawa_status enqueue_weights_launches(StepContext& c)
     const int grid1 = g_sumsq_ctas_per_sm > 0
                           ? static_cast<int>(std::min<int64_t>(items1, g_sumsq_ctas_per_sm * plan->sm_count)) : items1;
     const int vg = c.vec_g ? 1 : 0;
-    c.sc.prefetch_stride = (c.dtype == 0 ? 6 : 5) * plan->sm_count;           // CTAs resident at the start of the kernel
+    c.sc.prefetch_stride = 6 * plan->sm_count;           // CTAs resident at the start of the kernel
     c.sc.prefetch_waves = (grid1 <= 64 * c.sc.prefetch_stride) ? static_cast<int>(g_sumsq_prefetch_waves) : 0;
     if (c.dtype == 1)
         GRAWA_CUDA_TRY(launch_kernel(sumsq16_kernel<__nv_bfloat16, 8>, grid1, kThreads, c.stream, c.pdl, c.gp, c.sc, items1, vg));

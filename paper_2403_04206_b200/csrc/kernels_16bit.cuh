@@ -71,9 +71,10 @@ __device__ __forceinline__ void split_range16(long long b, long long e, int vec_
 }
 
 // Step 1 on 16-bit gradients: same work list, same fp32-run / fp64-combine scheme as sumsq_kernel;
-// a thread's 16-byte load carries 8 elements, each with its own fp32 accumulator.
+// a thread's 16-byte load carries 8 elements, each with its own fp32 accumulator.  Six CTAs per SM
+// (40 registers) like the fp32 kernel: measured 4 % faster than five on the ViT-B/16 table.
 template <typename T, int UNROLL>
-__global__ void __launch_bounds__(kThreads, 5)
+__global__ void __launch_bounds__(kThreads, 6)
 sumsq16_kernel(const __grid_constant__ ConstPtrs grads, StepScratch sc, int items, int vec_ok)
 {
     __shared__ double warp_part[2][kThreads / 32];
