@@ -110,6 +110,30 @@ def test_16bit_pull_extremes_are_bit_exact(grawa, dtype_name):
     assert np.array_equal(r0["center"], r1["center"])
 
 
+@pytest.mark.parametrize("dtype_name", ["bfloat16", "float16"])
+@pytest.mark.parametrize("M", [5, 8, 12, 16])
+def test_16bit_pull_extremes_are_bit_exact_on_the_staged_kernel(grawa, M, dtype_name):
+    """5..16 workers take the kernel that stages its columns through shared memory: the same exact
+    identities at pull 1 and pull 0, and the same bytes as the register kernel it replaces."""
+    cfg = gen.custom_config([7, 5001, 0, 3, 12001, 777, 8, 9, 8192, 8193, 40000], M, seed=400 + M, log10_sigma=(-2.0, 0.0))
+    p, g = gen.make_inputs(cfg)
+    r1 = run_typed(grawa, dtype_name, "lgrawa", p, g, 1.0, cfg.offsets())
+    for w in r1["workers"]:
+        assert np.array_equal(w, r1["center"])
+    r0 = run_typed(grawa, dtype_name, "mgrawa", p, g, 0.0, cfg.offsets())
+    for w, a in zip(r0["workers"], r0["p_img"]):
+        assert np.array_equal(w, a)
+    staged = run_typed(grawa, dtype_name, "lgrawa", p, g, 0.3, cfg.offsets())
+    grawa.grawa_set_option("pull16_staged", 0)
+    try:
+        regs = run_typed(grawa, dtype_name, "lgrawa", p, g, 0.3, cfg.offsets())
+    finally:
+        grawa.grawa_set_option("pull16_staged", 1)
+    assert np.array_equal(staged["center"], regs["center"])
+    for u, v in zip(staged["workers"], regs["workers"]):
+        assert np.array_equal(u, v)
+
+
 def test_16bit_sumsq_bit_exact_on_integer_gradients(grawa):
     sizes = [10, 1000, 8192, 3, 20000, 1, 4097, 70000]
     rng = np.random.default_rng(3)
