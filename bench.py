@@ -341,12 +341,12 @@ STORED_CAPTURES = {
                     "end": "// Steps 4-5 for any M up to",
                     "host_begin": "static grawa_status enqueue_center_pull(StepContext", "host_end": "// Given scores of a step",
                     "kernel_sha256": "9aa1cd15bd94e316e2a45778645f33881e36eaed5ee35a7f1b272d01f6475272",
-                    "host_sha256": "3da8ac05f8a7f1338e0f94cc8aaec33818f4bbe64ec93fb725b53e58e6c35fda"},
+                    "host_sha256": "08f9e8f045b5e0f30219e9a3fc2c79ab3bfb91d23a7c329b7e8c6c8cef465dae"},
     "sumsq": {"M": 16, "dram_bytes": 954845952 + 3118336, "begin": "// Step 1 (Eq. 3 / Eq. 5):",
               "end": "// Steps 4-5, register variant",
               "host_begin": "static grawa_status enqueue_weights_launches(StepContext& c)\n", "host_end": "// Steps 4-5 on 16-bit storage",
               "kernel_sha256": "6c8fcdcd2927db90fe40fdbb204bf18a7a4757f76906c7670ab4625309856fa1",
-              "host_sha256": "d4e501bd1b39f7af71d29a7670c0fa21c05eabf6517be8608e100ac96bc95406"},
+              "host_sha256": "749ab7388e3b22c197354e8780ec470ca204b4568ffb3a038fbabe3a23e9796a"},
 }
 DEFAULT_KNOBS = {"sumsq_tile": 8192, "pull_tile": 0, "pull_variant": 0, "bulk_tile": 0, "sumsq_ctas_per_sm": 0,
                  "pull_prefetch_waves": 3, "sumsq_prefetch_waves": 1,

@@ -319,10 +319,12 @@ int grawa_trace_read(uint64_t *rows_out, int max_rows);
  *   "sumsq_tile"   elements per sum-of-squares work item (multiple of 1024, 1024..1048576)
  *   "pull_tile"    elements per centre+pull work item (multiple of 1024, 1024..1048576);
  *                  0 (default) = what one CTA of the register kernel covers in a single pass,
- *                  8192 / 4096 / 2048 / 1024 elements for M <= 2 / 4 / 8 / more
- *   "pull_variant" 0 = automatic (register kernel up to 16 workers, bulk-copy kernel above),
- *                  1 = register kernel (vector loads), 2 = bulk-copy kernel (shared-memory
- *                  staging by 1-D bulk asynchronous copies and bulk stores)
+ *                  8192 / 4096 / 2048 / 1024 elements for M <= 2 / 4 / 8 / 16; above 16 workers
+ *                  what one CTA of the shared-memory kernel covers (4 elements per thread)
+ *   "pull_variant" 0 and 1 = register kernel (vector loads) up to 16 workers and, above 16, a
+ *                  kernel that stages each thread's 16-byte columns through shared memory by
+ *                  asynchronous copies (both storage widths); 2 = bulk-copy kernel (fp32 only:
+ *                  shared-memory staging by 1-D bulk asynchronous copies and bulk stores)
  *   "bulk_tile"    elements per slice of a bulk-copy stage (multiple of 256, up to 16384);
  *                  0 = chosen from M so that three stages fit in shared memory
  *   "kernel_timing" 1 = every device-buffer step also records CUDA events around its three

@@ -58,8 +58,9 @@ static inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; 
 // Dynamic shared memory the bulk-copy centre+pull kernel may use (one CTA per SM).
 constexpr size_t kBulkSmemBudget = 200 * 1024;
 
-// Does the centre+pull of an M-worker problem take the bulk-copy kernel?
-static bool wants_bulk(int M) { return g_pull_variant == 2 || (g_pull_variant == 0 && M > kMaxRegWorkers); }
+// Does the centre+pull of an M-worker problem take the bulk-copy kernel?  (Only when asked for: the staged
+// kernels replaced it as the vector path for more than 16 workers.)
+static bool wants_bulk(int) { return g_pull_variant == 2; }
 
 // Elements per slice of a bulk-copy stage: the option, or the largest multiple of 256 up to 4096
 // that leaves room for three stages of M+1 slices.
@@ -189,6 +190,7 @@ static grawa_status get_plan(int64_t n, int M, const std::vector<int64_t>& off, 
     p->tile1 = g_sumsq_tile * (4 / elem);
     p->tile2 = p->bulk ? bulk_tile_for(M)
                : (g_pull_tile > 0 ? g_pull_tile
+                  : M > kMaxRegWorkers ? staged_any_threads(M) * (16 / elem)
                   : (elem == 2 ? ((M > 4 && g_pull16_staged) ? pull16s_pass_elems(std::min(M, kMaxRegWorkers)) : pull16_pass_elems(std::min(M, kMaxRegWorkers)))
                                : pull_pass_elems(std::min(M, kMaxRegWorkers))));
     GRAWA_CUDA_TRY(cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, device));
@@ -428,6 +430,21 @@ struct CenterPull16StagedDispatch<T, 4> {
     }
 };
 
+// More than 16 aligned workers, any storage type: the staged kernel with a run-time worker count.
+template <typename T>
+static cudaError_t launch_center_pull_staged_any(bool per_layer, int grid, int item_begin, int item_end, cudaStream_t stream, bool pdl,
+                                                 const MutPtrs& x, T* center, const float* beta, const Segment* segs, long long n,
+                                                 int tile, float pull, int M, int preload)
+{
+    const int threads = staged_any_threads(M);
+    const size_t smem = align_up(sizeof(uint4) * static_cast<size_t>(M) * threads + sizeof(float) * M, 16);
+    auto kernel = per_layer ? center_pull_staged_any_kernel<T, true> : center_pull_staged_any_kernel<T, false>;
+    const cudaError_t err = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 80 * 1024);
+    if (err != cudaSuccess) return err;
+    return launch_kernel_smem(kernel, grid, threads, smem, stream, pdl, x, center, beta, segs, item_begin, item_end, n, tile, pull, M,
+                              preload);
+}
+
 // Device pointers and launch facts of one step, resolved once from the plan and the options.
 struct StepContext {
     Plan* plan = nullptr;
@@ -570,6 +587,9 @@ static grawa_status enqueue_center_pull16_t(StepContext& c, int item_begin, int 
         GRAWA_CUDA_TRY((CenterPull16StagedDispatch<T, kMaxRegWorkers>::run(M, per_layer, grid, item_begin, item_end, c.stream, c.pdl,
                                                                            c.xp, center, c.sc.beta, plan->d_segs2, c.n, tile, c.pull,
                                                                            (c.preload && g_pull_preload) ? 1 : 0)));
+    } else if (c.vec_x && M > kMaxRegWorkers) {
+        GRAWA_CUDA_TRY(launch_center_pull_staged_any<T>(per_layer, grid, item_begin, item_end, c.stream, c.pdl, c.xp, center, c.sc.beta,
+                                                        plan->d_segs2, c.n, tile, c.pull, M, (c.preload && g_pull_preload) ? 1 : 0));
     } else if (c.vec_x && M <= kMaxRegWorkers) {
         GRAWA_CUDA_TRY((CenterPull16Dispatch<T, kMaxRegWorkers>::run(M, per_layer, grid, item_begin, item_end, c.stream, c.pdl, c.xp,
                                                                      center, c.sc.beta, plan->d_segs2, c.n, tile, c.pull)));
@@ -597,7 +617,7 @@ static grawa_status enqueue_center_pull(StepContext& c, int item_begin, int item
     const int tile = static_cast<int>(plan->tile2);
     const float* beta = c.sc.beta;
     if (c.dtype != 0) return enqueue_center_pull16(c, item_begin, item_end);
-    // bulk-copy variant: asked for explicitly, or the only vector path for M > 16
+    // bulk-copy variant: only when asked for
     const size_t stage_bytes = sizeof(float) * static_cast<size_t>(plan->tile2) * (M + 1);
     const int stages = static_cast<int>(std::min<size_t>(kBulkMaxStages, kBulkSmemBudget / stage_bytes));
     if (c.vec_x && plan->bulk && stages >= 2) {
@@ -605,6 +625,9 @@ static grawa_status enqueue_center_pull(StepContext& c, int item_begin, int item
         GRAWA_CUDA_TRY(CenterPullBulkDispatch<kMaxRegWorkers>::run(M <= kMaxRegWorkers ? M : 1, per_layer, gridb, item_begin, item_end,
                                                                    stage_bytes * stages, c.stream, c.pdl, c.xp, c.center, beta,
                                                                    plan->d_segs2, c.n, tile, stages, M, c.pull, c.counter, c.status));
+    } else if (c.vec_x && M > kMaxRegWorkers) {
+        GRAWA_CUDA_TRY(launch_center_pull_staged_any<float>(per_layer, grid, item_begin, item_end, c.stream, c.pdl, c.xp, c.center, beta,
+                                                            plan->d_segs2, c.n, tile, c.pull, M, (c.preload && g_pull_preload) ? 1 : 0));
     } else if (c.vec_x && M <= kMaxRegWorkers) {
         // L2 prefetch of later items during the weights' finalisation: pays on short steps only (a few
         // dozen waves of CTAs); on long ones the window it fills is negligible and the hint costs a little

@@ -162,3 +162,39 @@ def test_typed_entry_with_float32_equals_the_plain_entry(grawa):
         grawa.grawa_step_typed("lgrawa", [t.double() for t in xa], gr, 0.5, off, ca)
     with pytest.raises(TypeError):
         grawa.grawa_step_typed("lgrawa", [t.half() for t in xa], gr, 0.5, off, ca)      # mixed dtypes
+
+
+@pytest.mark.parametrize("dtype_name", ["bfloat16", "float16"])
+@pytest.mark.parametrize("M", [17, 33, 64])
+def test_16bit_many_worker_kernel_is_exact_at_the_pull_extremes_and_matches_the_scalar_kernel(grawa, M, dtype_name):
+    """More than 16 workers take the run-time-M shared-memory kernel: exact identities at pull 1 and
+    pull 0, and (from given norms, so that the weights are the same) the same bytes as the element-wise
+    kernel that bases 2 bytes off alignment fall to."""
+    cfg = gen.custom_config([7, 5001, 0, 3, 12001, 777, 8, 9, 8192, 8193, 40000], M, seed=500 + M, log10_sigma=(-2.0, 0.0))
+    p, g = gen.make_inputs(cfg)
+    r1 = run_typed(grawa, dtype_name, "lgrawa", p, g, 1.0, cfg.offsets())
+    for w in r1["workers"]:
+        assert np.array_equal(w, r1["center"])
+    r0 = run_typed(grawa, dtype_name, "mgrawa", p, g, 0.0, cfg.offsets())
+    for w, a in zip(r0["workers"], r0["p_img"]):
+        assert np.array_equal(w, a)
+    vec = run_typed(grawa, dtype_name, "lgrawa", p, g, 0.3, cfg.offsets())
+    check(vec, dtype_name, "lgrawa", 0.3, cfg.offsets())
+    # same given norms, hence the same weights, through the vector kernel and (bases 2 bytes off) the element-wise one
+    import torch
+    dt = getattr(torch, dtype_name)
+    K = len(cfg.offsets()) - 1
+    norms = torch.from_numpy(np.random.default_rng(M).uniform(0.5, 2.0, size=(K, M))).cuda()
+    got = []
+    for shift in (0, 1):
+        xs = []
+        for a in p:
+            t = torch.zeros(a.size + shift, dtype=dt, device="cuda")
+            t[shift:] = torch.from_numpy(a).cuda().to(dt)
+            xs.append(t[shift:])
+        c = torch.zeros(xs[0].numel() + shift, dtype=dt, device="cuda")[shift:]
+        grawa.grawa_step_from_layer_norms_typed("lgrawa", xs, norms, 0.3, cfg.offsets(), c)
+        assert grawa.grawa_last_step_status() == 0
+        got.append([c.float().cpu().numpy()] + [t.float().cpu().numpy() for t in xs])
+    for u, v in zip(*got):
+        assert np.array_equal(u, v)

@@ -528,13 +528,41 @@ def test_bulk_and_register_variants_agree_bit_for_bit(grawa):
         assert bool((u == v).all())
 
 
-def test_many_workers_take_the_bulk_kernel_by_default(grawa):
-    """More than 16 workers: the automatic choice is the bulk-copy kernel (any M up to 64)."""
+def test_many_workers_take_the_shared_memory_kernel_by_default(grawa):
+    """More than 16 workers: the default is the kernel with a run-time worker count that stages its
+    columns through shared memory (any M up to 64); lambda 0.3 and a 33-element layer between two
+    long ones exercise its edges."""
     cfg = gen.custom_config([100000, 33, 200001], 40, seed=77, log10_sigma=(-2.0, 0.0))
     p, g = gen.make_inputs(cfg)
     res = gpu_step(grawa, "lgrawa", p, g, 0.3, cfg.offsets())
     compare_with_oracle(res, "lgrawa", p, g, 0.3, cfg.offsets())
     assert grawa.grawa_last_step_status() == 0
+
+
+@pytest.mark.parametrize("M", [17, 31, 64])
+def test_many_worker_kernel_matches_the_bulk_kernel_bit_for_bit_and_is_exact_at_the_pull_extremes(grawa, M):
+    """The run-time-M shared-memory kernel takes the same fused multiply-add chain in the same order
+    as the other centre+pull kernels: identical bytes; pull 1 puts every worker on the centre, pull 0
+    leaves every worker untouched."""
+    cfg = gen.custom_config([7, 5001, 0, 3, 12001, 777, 8, 9, 8192, 8193, 40000], M, seed=300 + M, log10_sigma=(-2.0, 0.0))
+    p, g = gen.make_inputs(cfg)
+    off = cfg.offsets()
+    ref = gpu_step(grawa, "lgrawa", p, g, 0.3, off)
+    compare_with_oracle(ref, "lgrawa", p, g, 0.3, off)
+    grawa.grawa_set_option("pull_variant", 2)
+    try:
+        got = gpu_step(grawa, "lgrawa", p, g, 0.3, off)
+    finally:
+        grawa.grawa_set_option("pull_variant", 0)
+    assert bool((ref["center"] == got["center"]).all())
+    for u, v in zip(ref["workers"], got["workers"]):
+        assert bool((u == v).all())
+    full = gpu_step(grawa, "mgrawa", p, g, 1.0, off)
+    for w in full["workers"]:
+        assert bool((w == full["center"]).all())
+    none = gpu_step(grawa, "lgrawa", p, g, 0.0, off)
+    for w, a in zip(none["workers"], p):
+        assert np.array_equal(w.cpu().numpy(), a)
 
 
 # ------------------------------------------------------------------ repeated steps on one plan
