@@ -122,10 +122,18 @@ class ClockSampler:
 
 # ------------------------------------------------------------------ workloads on the device
 
+def with_workers(cfg, M):
+    """The same layer table and value recipe with another number of workers."""
+    return gen.custom_config(np.diff(cfg.offsets()), M, seed=cfg.seed, pull=cfg.pull, grad_recipe=cfg.grad_recipe,
+                             log10_sigma=cfg.log10_sigma, loud_worker_factor=cfg.loud_worker_factor, name=f"{cfg.name}[M={M}]")
+
+
 def workload_config(args):
     """The named workload, or (for small profiling captures) only its first --layers-limit layers
     with the same value recipe."""
     cfg = gen.CONFIGS[args.workload]
+    if args.workers and args.workers != cfg.M:
+        cfg = with_workers(cfg, args.workers)
     if args.layers_limit and args.layers_limit < cfg.K:
         sizes = np.diff(cfg.offsets()[:args.layers_limit + 1])
         cfg = gen.custom_config(sizes, cfg.M, seed=cfg.seed, pull=cfg.pull, grad_recipe=cfg.grad_recipe,
@@ -337,12 +345,12 @@ def whole_job_steps_per_s(world, ms_per_step_max):
 # knob at its default; anything else reports null.
 CAPTURE_ELEMENTS = 14918400
 STORED_CAPTURES = {
-    "center_pull": {"M": 16, "dram_bytes": 955045376 + 958240256, "begin": "// Steps 4-5, register variant",
+    "center_pull": {"M": 16, "dram_bytes": 955075584 + 958193664, "begin": "// Steps 4-5, register variant",
                     "end": "// Steps 4-5 for any M up to",
                     "host_begin": "static grawa_status enqueue_center_pull(StepContext", "host_end": "// Given scores of a step",
                     "kernel_sha256": "9aa1cd15bd94e316e2a45778645f33881e36eaed5ee35a7f1b272d01f6475272",
                     "host_sha256": "08f9e8f045b5e0f30219e9a3fc2c79ab3bfb91d23a7c329b7e8c6c8cef465dae"},
-    "sumsq": {"M": 16, "dram_bytes": 954845952 + 3118336, "begin": "// Step 1 (Eq. 3 / Eq. 5):",
+    "sumsq": {"M": 16, "dram_bytes": 954870016 + 5120512, "begin": "// Step 1 (Eq. 3 / Eq. 5):",
               "end": "// Steps 4-5, register variant",
               "host_begin": "static grawa_status enqueue_weights_launches(StepContext& c)\n", "host_end": "// Steps 4-5 on 16-bit storage",
               "kernel_sha256": "6c8fcdcd2927db90fe40fdbb204bf18a7a4757f76906c7670ab4625309856fa1",
@@ -454,7 +462,7 @@ def run_cuda(args):
         sharded_out = run_sharded(grawa, cfg, variant, args, world, rank, peak, barrier, x, g, center)
 
     ms_max, e2e_ms_max = max_over_ranks([ms, e2e_ms if e2e_ms is not None else 0.0], world, "cuda")
-    ops = targets = small = None
+    ops = targets = small = many = None
     if world == 1 and not args.headline_only:
         ops = side_ops(grawa, cfg, variant, x, g, center, args, peak)
     del call, x, g, center
@@ -462,6 +470,7 @@ def run_cuda(args):
     hp_np, hg_np = [t.numpy() for t in hp], [t.numpy() for t in hg]
     if world == 1 and not args.headline_only:
         targets = target_runs(grawa, args, peak, have=(cfg, hp, hg))
+        many = many_worker_runs(grawa, args, peak)
         small = small_runs(grawa, args)
     clocks = sampler.stop()
 
@@ -507,6 +516,8 @@ def run_cuda(args):
             line["targets"] = targets
         if ops is not None:
             line["ops"] = ops
+        if many is not None:
+            line["many_workers"] = many
         if small is not None:
             line["small"] = small
         if sharded_out is not None:
@@ -578,6 +589,29 @@ def target_runs(grawa, args, peak, have=None):
                 del cb
         del c, x, g, center
         torch.cuda.empty_cache()
+    return out
+
+
+def many_worker_runs(grawa, args, peak):
+    """More workers than the register kernels cover (32, on the ResNet-18 layer table and value recipe;
+    3 GB): the centre+pull kernel with a run-time worker count, fp32 and bfloat16 storage."""
+    import torch
+    M = 32
+    cfg = with_workers(gen.CONFIGS["resnet18_imagenet"], M)
+    x, g = device_inputs(cfg)
+    center = torch.zeros(cfg.n, device="cuda")
+    steps = max(50, min(args.steps, 200))
+    out = []
+    for dtype in ("f32", "bf16"):
+        c = Call(grawa, cfg, "lgrawa", "step", dtype, x, g, center)
+        ms, _, _ = c.time(steps, 3)
+        _, _, ph = c.time(steps, 1, phases=True)
+        out.append(dict(workload=cfg.name, variant="lgrawa", storage=dtype, M=M, n=cfg.n, steps=steps,
+                        algorithmic_bytes=op_bytes(cfg, "step", dtype), kernels=kernel_table(cfg, dtype, ph, peak),
+                        **rates(op_bytes(cfg, "step", dtype), ms, peak)))
+        del c
+    del x, g, center
+    torch.cuda.empty_cache()
     return out
 
 
@@ -689,6 +723,7 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--headline-only", action="store_true", help="skip the short runs of the other workloads and calls")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workers", type=int, default=0, help="override the workload's number of workers (2..64)")
     ap.add_argument("--layers-limit", type=int, default=0, help="use only the first L layers (small profiling captures)")
     ap.add_argument("--option", action="append", default=[], help="library tuning knob, name=value (repeatable)")
     ap.add_argument("--print-source-hashes", action="store_true",
