@@ -447,7 +447,8 @@ template <> struct Col16<float> {
 // 16-byte slots per thread stay within 72 KB of shared memory, so that three CTAs fit on an SM.
 __host__ __device__ constexpr int staged_any_threads(int M)
 {
-    return (4608 / M) / 32 * 32 > 256 ? 256 : ((4608 / M) / 32 * 32 < 32 ? 32 : (4608 / M) / 32 * 32);
+    const int fit = (72 * 1024 / 16) / M / 32 * 32;
+    return fit > 256 ? 256 : (fit < 32 ? 32 : fit);
 }
 
 // Steps 4-5 for 17..64 workers (any storage type): the staging of center_pull16_staged_kernel with the

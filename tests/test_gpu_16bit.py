@@ -198,3 +198,14 @@ def test_16bit_many_worker_kernel_is_exact_at_the_pull_extremes_and_matches_the_
         got.append([c.float().cpu().numpy()] + [t.float().cpu().numpy() for t in xs])
     for u, v in zip(*got):
         assert np.array_equal(u, v)
+
+
+def test_16bit_resnet18_table_with_32_workers_full_size(grawa):
+    """The many-worker case the benchmark times on bfloat16 storage, element by element against the oracle."""
+    base = gen.CONFIGS["resnet18_imagenet"]
+    cfg = gen.custom_config(np.diff(base.offsets()), 32, seed=base.seed, pull=base.pull, grad_recipe=base.grad_recipe,
+                            log10_sigma=base.log10_sigma, loud_worker_factor=base.loud_worker_factor)
+    p, g = gen.make_inputs(cfg)
+    res = run_typed(grawa, "bfloat16", "lgrawa", p, g, cfg.pull, cfg.offsets())
+    del p, g
+    check(res, "bfloat16", "lgrawa", cfg.pull, cfg.offsets())

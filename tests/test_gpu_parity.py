@@ -55,6 +55,21 @@ def test_parity_large_workloads(grawa, name, variant):
         assert 50 < res["beta"][1] / res["beta"][0] < 200
 
 
+def test_parity_resnet18_table_with_32_workers_full_size(grawa):
+    """The many-worker case the benchmark times (ResNet-18 layer table and value recipe, 32 workers):
+    element by element against the oracle, per-layer and flat weights."""
+    base = gen.CONFIGS["resnet18_imagenet"]
+    cfg = gen.custom_config(np.diff(base.offsets()), 32, seed=base.seed, pull=base.pull, grad_recipe=base.grad_recipe,
+                            log10_sigma=base.log10_sigma, loud_worker_factor=base.loud_worker_factor)
+    _inputs_cache.clear()
+    p, g = gen.make_inputs(cfg)
+    for variant in ("lgrawa", "mgrawa"):
+        res = gpu_step(grawa, variant, p, g, cfg.pull, cfg.offsets())
+        compare_with_oracle(res, variant, p, g, cfg.pull, cfg.offsets())
+        assert grawa.grawa_last_step_status() == 0
+        del res
+
+
 @pytest.mark.parametrize("pull", [0.3, 0.7])
 @pytest.mark.parametrize("variant", ["mgrawa", "lgrawa"])
 def test_parity_other_pull_strengths(grawa, variant, pull):
