@@ -229,6 +229,20 @@ class Call:
         return e0.elapsed_time(e1) / steps, launches, ph
 
 
+def per_step_times(call, steps):
+    """Each of `steps` further calls between its own pair of CUDA events: median and minimum."""
+    import torch
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    ev[0].record()
+    for i in range(steps):
+        call.fn()
+        ev[i + 1].record()
+    torch.cuda.synchronize()
+    t = sorted(ev[i].elapsed_time(ev[i + 1]) for i in range(steps))
+    return {"steps": steps, "median_ms": t[steps // 2], "min_ms": t[0], "max_ms": t[-1],
+            "note": "one event pair per call, taken after the timed region; the headline is the K-call region"}
+
+
 def rates(bytes_per_call, ms, peak):
     gbs = bytes_per_call / (ms * 1e-3) / 1e9
     return {"ms_per_step": ms, "steps_per_s": 1e3 / ms, "achieved_gbs": gbs, "frac_of_measured_peak": gbs / peak,
@@ -432,6 +446,7 @@ def run_cuda(args):
     barrier()
     ms, launches, _ = call.time(args.steps, args.warmup)
     barrier()
+    each = per_step_times(call, max(10, min(args.steps, 100)))
     line = None
     alg_bytes = op_bytes(cfg, op, dtype)
     if op == "prox":
@@ -503,7 +518,7 @@ def run_cuda(args):
             "scaling": "weak", "vs_baseline": None, "dtype": dtype, "data": "synthetic",
             "config": describe(cfg, variant, op, dtype, world),
             "step_hbm": {k: step_rates[k] for k in ("achieved_gbs", "frac_of_measured_peak", "frac_of_nominal_8TBs")},
-            "roofline": roof,
+            "roofline": roof, "per_step": each,
             "gpu_launches": launches, "clocks": clocks, "last_step_status": status,
         }
         if e2e_ms is not None:

@@ -12,7 +12,7 @@ LIB_PATH = os.path.join(_HERE, "libgrawa.so")
 DEBUG_LIB_PATH = os.path.join(_HERE, "libgrawa_debug_bounds.so")
 TRACE_LIB_PATH = os.path.join(_HERE, "libgrawa_trace.so")
 SOURCES = [os.path.join(CSRC, "grawa.cu")]
-HEADERS = [os.path.join(CSRC, "kernels.cuh"), os.path.join(CSRC, "center_pull_bulk.cuh"), os.path.join(CSRC, "kernels_16bit.cuh"),
+HEADERS = [os.path.join(CSRC, "kernels.cuh"), os.path.join(CSRC, "center_pull_bulk.cuh"), os.path.join(CSRC, "kernels_16bit.cuh"), os.path.join(CSRC, "center_pull_staged_any.cuh"),
            os.path.join(_ROOT, "include", "grawa.h")]
 
 # IEEE arithmetic throughout: no fast-math.

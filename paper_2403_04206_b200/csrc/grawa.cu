@@ -17,6 +17,7 @@
 #include "kernels.cuh"
 #include "center_pull_bulk.cuh"
 #include "kernels_16bit.cuh"
+#include "center_pull_staged_any.cuh"
 
 namespace grawa {
 

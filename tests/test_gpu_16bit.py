@@ -209,3 +209,23 @@ def test_16bit_resnet18_table_with_32_workers_full_size(grawa):
     res = run_typed(grawa, "bfloat16", "lgrawa", p, g, cfg.pull, cfg.offsets())
     del p, g
     check(res, "bfloat16", "lgrawa", cfg.pull, cfg.offsets())
+
+
+@pytest.mark.parametrize("case", range(24))
+def test_16bit_parity_on_seeded_random_tables(grawa, case):
+    """The same kind of random tables on 16-bit storage, across the register, staged and run-time-M kernels."""
+    rng = np.random.default_rng(7000 + case)
+    K = int(rng.integers(1, 12))
+    kinds = rng.integers(0, 5, size=K)
+    sizes = [int({0: 0, 1: rng.integers(1, 17), 2: rng.integers(17, 3000), 3: 8 * rng.integers(256, 5000),
+                  4: rng.integers(20000, 70000)}[int(k)]) for k in kinds]
+    if sum(sizes) == 0:
+        sizes[-1] = 4321
+    M = int(rng.choice([2, 3, 4, 5, 8, 11, 16, 17, 25, 48, 64]))
+    dtype_name = ["bfloat16", "float16"][case % 2]
+    variant = ["lgrawa", "mgrawa", "grawa"][case % 3]
+    pull = float(rng.choice([0.2, 0.5, 0.8]))
+    cfg = gen.custom_config(sizes, M, seed=7000 + case, log10_sigma=(-2.0, 0.0))
+    p, g = gen.make_inputs(cfg)
+    res = run_typed(grawa, dtype_name, variant, p, g, pull, cfg.offsets(), offset_elems=(8 if case % 4 == 3 else 0))
+    check(res, dtype_name, variant, pull, cfg.offsets())

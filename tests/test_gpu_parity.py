@@ -580,6 +580,27 @@ def test_many_worker_kernel_matches_the_bulk_kernel_bit_for_bit_and_is_exact_at_
         assert np.array_equal(w.cpu().numpy(), a)
 
 
+@pytest.mark.parametrize("case", range(40))
+def test_parity_on_seeded_random_tables(grawa, case):
+    """Random layer tables (empty, tiny, odd and long layers mixed), worker counts across every
+    centre+pull kernel, pull strengths and variants, all drawn from the case number."""
+    rng = np.random.default_rng(9000 + case)
+    K = int(rng.integers(1, 14))
+    kinds = rng.integers(0, 5, size=K)
+    sizes = [int({0: 0, 1: rng.integers(1, 9), 2: rng.integers(9, 3000), 3: 4 * rng.integers(256, 9000),
+                  4: rng.integers(20000, 90000)}[int(k)]) for k in kinds]
+    if sum(sizes) == 0:
+        sizes[-1] = 1234
+    M = int(rng.choice([2, 3, 4, 5, 7, 8, 9, 12, 16, 17, 20, 29, 40, 64]))
+    variant = ["mgrawa", "lgrawa", "grawa"][case % 3]
+    pull = float(rng.choice([0.1, 0.3, 0.5, 0.7, 0.9]))
+    cfg = gen.custom_config(sizes, M, seed=9000 + case, log10_sigma=(-3.0, 0.0))
+    p, g = gen.make_inputs(cfg)
+    res = gpu_step(grawa, variant, p, g, pull, cfg.offsets())
+    compare_with_oracle(res, variant, p, g, pull, cfg.offsets())
+    assert grawa.grawa_last_step_status() == 0
+
+
 # ------------------------------------------------------------------ repeated steps on one plan
 
 @pytest.mark.parametrize("variant", ["mgrawa", "lgrawa", "grawa"])
