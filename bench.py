@@ -660,9 +660,23 @@ def small_runs(grawa, args):
                     graph.replay()
                 e1.record()
                 stream.synchronize()
+                # ten steps in one graph: what a step costs inside a larger captured region (no host launch between steps)
+                graph10 = torch.cuda.CUDAGraph()
+                with torch.cuda.graph(graph10, stream=stream):
+                    for _ in range(10):
+                        c.fn()
+                for _ in range(5):
+                    graph10.replay()
+                f0, f1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                f0.record()
+                for _ in range(100):
+                    graph10.replay()
+                f1.record()
+                stream.synchronize()
             out.append({"workload": name, "variant": variant, "M": cfg.M, "n": cfg.n, "eager_us": eager_ms * 1e3, "eager_prepared_args_us": prepared_ms * 1e3,
-                        "graph_replay_us": e0.elapsed_time(e1), "traffic_time_us_at_8TBs": op_bytes(cfg, "step") / 8e12 * 1e6})
-            del graph
+                        "graph_replay_us": e0.elapsed_time(e1), "step_us_inside_a_graph_of_10_steps": f0.elapsed_time(f1),
+                        "traffic_time_us_at_8TBs": op_bytes(cfg, "step") / 8e12 * 1e6})
+            del graph, graph10
         del x, g, center
     return out
 
