@@ -359,12 +359,12 @@ def whole_job_steps_per_s(world, ms_per_step_max):
 # knob at its default; anything else reports null.
 CAPTURE_ELEMENTS = 14918400
 STORED_CAPTURES = {
-    "center_pull": {"M": 16, "dram_bytes": 955075584 + 958193664, "begin": "// Steps 4-5, register variant",
+    "center_pull": {"M": 16, "dram_bytes": 955075584 + 958193664, "dram_bytes_full": (86567656, 5542392064 + 5844806656), "begin": "// Steps 4-5, register variant",
                     "end": "// Steps 4-5 for any M up to",
                     "host_begin": "static grawa_status enqueue_center_pull(StepContext", "host_end": "// Given scores of a step",
                     "kernel_sha256": "9aa1cd15bd94e316e2a45778645f33881e36eaed5ee35a7f1b272d01f6475272",
                     "host_sha256": "08f9e8f045b5e0f30219e9a3fc2c79ab3bfb91d23a7c329b7e8c6c8cef465dae"},
-    "sumsq": {"M": 16, "dram_bytes": 954870016 + 5120512, "begin": "// Step 1 (Eq. 3 / Eq. 5):",
+    "sumsq": {"M": 16, "dram_bytes": 954870016 + 5120512, "dram_bytes_full": (86567656, 5540708608 + 3944448), "begin": "// Step 1 (Eq. 3 / Eq. 5):",
               "end": "// Steps 4-5, register variant",
               "host_begin": "static grawa_status enqueue_weights_launches(StepContext& c)\n", "host_end": "// Steps 4-5 on 16-bit storage",
               "kernel_sha256": "6c8fcdcd2927db90fe40fdbb204bf18a7a4757f76906c7670ab4625309856fa1",
@@ -394,7 +394,8 @@ def source_hashes(which):
 
 
 def stored_traffic(grawa, which, cfg):
-    """DRAM bytes of one full launch scaled from the stored capture, or None when it does not apply."""
+    """DRAM bytes of one full launch from the stored captures (the one taken at this very size if there
+    is one, else the small one scaled by elements), or None when they do not apply."""
     cap = STORED_CAPTURES[which]
     if cap["dram_bytes"] is None or cfg.M != cap["M"]:
         return None
@@ -402,6 +403,9 @@ def stored_traffic(grawa, which, cfg):
         return None
     if source_hashes(which) != (cap["kernel_sha256"], cap["host_sha256"]):
         return None
+    full = cap.get("dram_bytes_full")
+    if full and full[0] == cfg.n:
+        return float(full[1])
     return cap["dram_bytes"] / CAPTURE_ELEMENTS * cfg.n
 
 
@@ -497,10 +501,10 @@ def run_cuda(args):
             roof = {"bound": "hbm", "kernel": dominant, "achieved": kd["achieved_gbs"], "peak": peak, "peak_source": peak_src,
                     "unit": "GB/s", "frac": kd["frac_of_measured_peak"], "frac_of_nominal_8TBs": kd["achieved_gbs"] / NOMINAL_HBM_GBS,
                     "traffic": stored_traffic(grawa, "center_pull", cfg) if dtype == "f32" else None,
-                    "traffic_source": "stored ncu capture (dram bytes read + written) of a launch over "
-                                      f"{CAPTURE_ELEMENTS} elements at the same M, scaled by elements; null when the kernel, its launch "
-                                      "code or a tuning knob differs from the capture's",
-                    "traffic_scaled_from_n": CAPTURE_ELEMENTS,
+                    "traffic_source": "stored ncu capture (dram bytes read + written) of one launch at the same M: taken at this "
+                                      f"workload's full size when n = 86567656, otherwise a launch over {CAPTURE_ELEMENTS} elements "
+                                      "scaled by elements; null when the kernel, its launch code or a tuning knob differs from the capture's",
+                    "traffic_scaled_from_n": None if cfg.n == 86567656 else CAPTURE_ELEMENTS,
                     "algorithmic_bytes_per_launch": kd["algorithmic_bytes_per_launch"], "kernel_ms": kd["kernel_ms"],
                     "timed_with": "library CUDA events around each kernel in a second K-step region (dependent launch off there)",
                     "other_kernels": {k: v for k, v in kernels.items() if k != "center_pull"},

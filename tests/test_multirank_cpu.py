@@ -88,6 +88,8 @@ def test_stored_ncu_traffic_is_quoted_only_for_the_captured_kernel_and_default_k
         got = bench.stored_traffic(Knobs(), which, vit)
         assert (got is not None) == (same_source and cap["dram_bytes"] is not None)
         if got is not None:
-            assert abs(got / (cap["dram_bytes"] / bench.CAPTURE_ELEMENTS * vit.n) - 1) < 1e-12
+            assert got == cap["dram_bytes_full"][1] and cap["dram_bytes_full"][0] == vit.n    # the capture at this very size
+            part = gen.custom_config([1000, 5_000_000], vit.M)                                # any other size: scaled by elements
+            assert abs(bench.stored_traffic(Knobs(), which, part) / (cap["dram_bytes"] / bench.CAPTURE_ELEMENTS * part.n) - 1) < 1e-12
         assert bench.stored_traffic(Knobs(), which, vgg) is None                      # another M
         assert bench.stored_traffic(Knobs(pull_variant=2), which, vit) is None       # a knob off its default
