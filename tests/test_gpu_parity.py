@@ -601,6 +601,20 @@ def test_parity_on_seeded_random_tables(grawa, case):
     assert grawa.grawa_last_step_status() == 0
 
 
+@pytest.mark.parametrize("variant", ["mgrawa", "lgrawa", "grawa"])
+@pytest.mark.parametrize("M", [5, 64])
+def test_parity_with_thousands_of_tiny_layers(grawa, M, variant):
+    """3000 layers of 0..50 elements: every (layer, worker) row is its own item, the one-CTA
+    finalisation walks long runs of layers per thread, most centre+pull items are ragged."""
+    rng = np.random.default_rng(31)
+    sizes = [int(v) for v in rng.integers(0, 51, size=3000)]
+    cfg = gen.custom_config(sizes, M, seed=640 + M, log10_sigma=(-3.0, 0.0))
+    p, g = gen.make_inputs(cfg)
+    res = gpu_step(grawa, variant, p, g, 0.5, cfg.offsets())
+    compare_with_oracle(res, variant, p, g, 0.5, cfg.offsets())
+    assert grawa.grawa_last_step_status() == 0
+
+
 # ------------------------------------------------------------------ repeated steps on one plan
 
 @pytest.mark.parametrize("variant", ["mgrawa", "lgrawa", "grawa"])
