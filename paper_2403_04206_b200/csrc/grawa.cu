@@ -523,18 +523,30 @@ static grawa_status make_context(int variant, float* const* params, const float*
     return GRAWA_OK;
 }
 
-// Steps 2-3.  LGRAWA from the sums of a sum-of-squares kernel: one warp per layer in as many CTAs
-// as that takes.  Everything else (one weight per worker, or given scores): one CTA.
+// Steps 2-3.  LGRAWA: one warp per layer in as many CTAs as that takes.  One weight per worker: one
+// CTA with a thread per (layer, worker) row when that fits, runs of rows per thread up to
+// kFinSharedOutRows rows, beyond that the rows shared out over several full CTAs.
 static cudaError_t launch_finalize(const StepContext& c)
 {
     const Plan* plan = c.plan;
-    const bool layered = c.variant == kLgrawa && c.sc.given == nullptr;
-    const int warps = kFinThreadsLayered / 32;
-    const int grid = layered ? std::max(1, std::min((plan->K + warps - 1) / warps, 4 * plan->sm_count)) : 1;
-    // the one CTA of the other cases: a thread per (layer, worker) row when that fits
     const int64_t rows = static_cast<int64_t>(plan->K) * c.M;
-    const int flat = static_cast<int>(std::max<int64_t>(128, std::min<int64_t>(kFinThreadsFlat, (rows + 31) / 32 * 32)));
-    const int block = layered ? kFinThreadsLayered : flat;
+    int grid = 1, block = static_cast<int>(std::max<int64_t>(128, std::min<int64_t>(kFinThreadsFlat, (rows + 31) / 32 * 32)));
+    if (c.variant == kLgrawa && c.sc.given == nullptr) {
+        block = kFinThreadsLayered;
+        grid = std::max(1, std::min((plan->K + block / 32 - 1) / (block / 32), 4 * plan->sm_count));
+    } else if (c.variant == kLgrawa) {
+        // given scores: no sum-of-squares kernel has cleared the status words, and several CTAs only
+        // add their flags to them, so they are cleared here when the layers take more than one CTA
+        if (plan->K > kFinGivenLayersOneCta) {
+            block = kFinThreadsFlat;
+            grid = std::min((plan->K + block / 32 - 1) / (block / 32), 4 * plan->sm_count);
+            cudaError_t err = cudaMemsetAsync(c.sc.status, 0, sizeof(int), c.stream);
+            if (err == cudaSuccess && c.sc.status_copy) err = cudaMemsetAsync(c.sc.status_copy, 0, sizeof(int), c.stream);
+            if (err != cudaSuccess) return err;
+        }
+    } else if (rows > kFinSharedOutRows) {
+        grid = static_cast<int>(std::min<int64_t>((rows + kFinThreadsFlat - 1) / kFinThreadsFlat, plan->sm_count));
+    }
     return launch_kernel(finalize_kernel, grid, block, c.stream, c.pdl, c.sc);
 }
 

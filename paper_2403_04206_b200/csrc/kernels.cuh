@@ -359,6 +359,9 @@ __device__ __forceinline__ void store_row(const StepScratch& sc, size_t idx, dou
 constexpr int kFinThreadsLayered = 256;     // LGRAWA: 8 layers per CTA
 constexpr int kFinThreadsFlat = 1024;       // MGRAWA / GRAWA: the one CTA (at most)
 constexpr int kFinGroupSlots = 512;         // >= ceil(sqrt(P)) * M for every P * M <= 1024, M <= 64
+constexpr int kFinSharedOutRows = 4096;     // MGRAWA / GRAWA with more (layer, worker) rows than this: several CTAs
+constexpr int kFinGivenLayersOneCta = 256;  // LGRAWA from given scores with more layers than this: several CTAs
+constexpr int kFinTicketWord = 3;           // word of the scratch's leading block that counts those CTAs' tickets
 
 __global__ void __launch_bounds__(kFinThreadsFlat, 1)
 finalize_kernel(StepScratch sc)
@@ -430,19 +433,56 @@ finalize_kernel(StepScratch sc)
         return;
     }
 
-    // MGRAWA / GRAWA (launched as one CTA)
+    // MGRAWA / GRAWA: one CTA, or (many rows) several CTAs that share the rows out and a last one to
+    // finish, whichever it is, that adds the stored terms in the same fixed order as the one CTA would
     const int P = max(1, min(K, static_cast<int>(blockDim.x) / M));
     const int run = (K + P - 1) / P;
+    const bool shared_out = gridDim.x > 1;
+    if (shared_out) {
+        const long long rows = static_cast<long long>(K) * M;
+        for (long long idx = static_cast<long long>(blockIdx.x) * blockDim.x + tid; idx < rows;
+             idx += static_cast<long long>(gridDim.x) * blockDim.x) {
+            const double s = row_sumsq(sc, bins, static_cast<size_t>(idx));
+            store_row(sc, static_cast<size_t>(idx), s, row_term(sc, static_cast<size_t>(idx), s));
+        }
+        // one ticket per CTA (no CTA waits for another): the rows are fenced before the ticket is
+        // taken, and whoever takes the last one reads all of them behind a fence of its own
+        unsigned* ticket = reinterpret_cast<unsigned*>(sc.next_buf) + kFinTicketWord;
+        __shared__ int last_sm;
+        __threadfence();
+        __syncthreads();
+        if (tid == 0) last_sm = atomicAdd(ticket, 1u) == gridDim.x - 1 ? 1 : 0;
+        __syncthreads();
+        if (!last_sm) {
+            if (keeper && sc.given == nullptr) *sc.next_buf = next;
+            trace.done();
+            return;
+        }
+        __threadfence();
+        if (tid == 0) *ticket = 0u;                              // ready for the next launch
+    }
     if (tid < P * M) {
         const int p = tid / M, m = tid - p * M;
         const int k1 = min(K, (p + 1) * run);
         double a = 0.0;
-        for (int k = p * run; k < k1; ++k) {
-            const size_t idx = static_cast<size_t>(k) * M + m;
-            const double s = row_sumsq(sc, bins, idx);
-            const double term = row_term(sc, idx, s);
-            store_row(sc, idx, s, term);
-            a += term;
+        if (shared_out) {                                        // the stored terms, same order; loads eight at a time
+            int k = p * run;
+            for (; k + 8 <= k1; k += 8) {
+                double t[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) t[u] = __ldcg(sc.A + static_cast<size_t>(k + u) * M + m);
+#pragma unroll
+                for (int u = 0; u < 8; ++u) a += t[u];
+            }
+            for (; k < k1; ++k) a += __ldcg(sc.A + static_cast<size_t>(k) * M + m);
+        } else {
+            for (int k = p * run; k < k1; ++k) {
+                const size_t idx = static_cast<size_t>(k) * M + m;
+                const double s = row_sumsq(sc, bins, idx);
+                const double term = row_term(sc, idx, s);
+                store_row(sc, idx, s, term);
+                a += term;
+            }
         }
         part_sm[tid] = a;
     }

@@ -57,6 +57,21 @@ def main():
     gs = [torch.zeros(cfg.n + 1, device="cuda")[1:] for _ in range(4)]
     gpu_step(grawa, "lgrawa", p, g, 0.5, cfg.offsets(), params_dev=xs, grads_dev=gs)
     out["cases"] += 1
+    # thousands of tiny layers (finalisation over several CTAs) and many workers (run-time-M kernel)
+    rng = np.random.default_rng(3)
+    for M in (5, 33, 64):
+        cfg = gen.custom_config([int(v) for v in rng.integers(0, 41, size=2500)] + [50001], M, seed=900 + M, log10_sigma=(-2.0, 0.0))
+        p, g = gen.make_inputs(cfg)
+        for variant in ("mgrawa", "lgrawa", "grawa"):
+            res = gpu_step(grawa, variant, p, g, 0.5, cfg.offsets())
+            if M == 5:
+                compare_with_oracle(res, variant, p, g, 0.5, cfg.offsets())
+            out["cases"] += 1
+        norms = torch.from_numpy(10.0 ** rng.uniform(-2, 1, size=(cfg.K, M))).cuda()
+        grawa.grawa_step_from_layer_norms("lgrawa", [torch.from_numpy(a).cuda() for a in p], norms, 0.5, cfg.offsets(), None)
+        x16 = [torch.from_numpy(a).cuda().bfloat16() for a in p]
+        grawa.grawa_step_typed("lgrawa", x16, [torch.from_numpy(a).cuda().bfloat16() for a in g], 0.5, cfg.offsets(), None)
+        out["cases"] += 2
     torch.cuda.synchronize()
     out["violations"] = grawa.grawa_debug_bounds_violations()
     print(json.dumps(out))

@@ -89,6 +89,48 @@ def test_step_from_layer_norms_parity(grawa, variant, M):
         assert np.array_equal(x[0].cpu().numpy(), p[0])
 
 
+@pytest.mark.parametrize("variant", ["mgrawa", "lgrawa", "grawa"])
+@pytest.mark.parametrize("M", [3, 64])
+def test_step_from_layer_norms_with_thousands_of_layers(grawa, variant, M):
+    """3000 layers: the finalisation runs as several CTAs (rows shared out and a last CTA that adds the
+    terms; with per-layer weights a warp per layer and status words cleared in front of the launch).
+    Twice in a row, the second time with a non-finite norm: the status says so and the next step is clean."""
+    import torch
+    rng = np.random.default_rng(M)
+    sizes = [int(v) for v in rng.integers(0, 41, size=3000)]
+    cfg = gen.custom_config(sizes, M, seed=170 + M, log10_sigma=(-2.0, 0.0))
+    p, _ = gen.make_inputs(cfg)
+    off = cfg.offsets()
+    norms = 10.0 ** rng.uniform(-3, 1, size=(cfg.K, M))
+    norms[np.diff(off) == 0] = 0.0
+    A = oracle.scores_from_norms(norms, variant)
+    beta_ref, _ = oracle.weights(A)
+    G = cfg.K if variant == "lgrawa" else 1
+    tol = TOL_X_ABS_FACTOR * max(float(np.abs(a).max()) for a in p)
+    word = torch.full((1,), 77, dtype=torch.int32, device="cuda")
+    for trial in range(3):
+        given = norms.copy()
+        if trial == 1:
+            given[1234, 1] = np.inf
+        x = to_device(p)
+        center = torch.empty(cfg.n, device="cuda")
+        beta = torch.empty(G * M, device="cuda")
+        grawa.grawa_step_from_layer_norms(variant, x, torch.from_numpy(given).cuda(), 0.5, off, center, weights_out=beta,
+                                          status_word=word)
+        status = grawa.grawa_last_step_status()
+        if trial == 1:
+            assert status == -3 and word.item() != 0            # GRAWA_ERR_NONFINITE
+            continue
+        assert status == 0 and word.item() == 0
+        got_beta = beta.cpu().numpy().reshape(beta_ref.shape)
+        nz = beta_ref != 0
+        assert np.abs(got_beta[nz] / beta_ref[nz] - 1).max() <= TOL_BETA_REL
+        c_ref, w_ref = oracle.center_pull(p, beta_ref, 0.5, off, want_workers=True)
+        assert np.abs(center.cpu().numpy() - c_ref).max() <= tol
+        for m in range(M):
+            assert np.abs(x[m].cpu().numpy() - w_ref[m]).max() <= tol
+
+
 @pytest.mark.parametrize("variant", ["mgrawa", "lgrawa"])
 def test_norms_then_step_equals_the_gradient_step_bit_for_bit(grawa, variant):
     """Layer norms taken worker by worker and fed back give exactly the step that reads the gradients."""

@@ -613,6 +613,10 @@ def test_parity_with_thousands_of_tiny_layers(grawa, M, variant):
     res = gpu_step(grawa, variant, p, g, 0.5, cfg.offsets())
     compare_with_oracle(res, variant, p, g, 0.5, cfg.offsets())
     assert grawa.grawa_last_step_status() == 0
+    again = gpu_step(grawa, variant, p, g, 0.5, cfg.offsets())            # tickets and digit rows left clean
+    for key in ("S", "A", "beta"):
+        assert np.array_equal(again[key], res[key]), key
+    assert bool((again["center"] == res["center"]).all())
 
 
 # ------------------------------------------------------------------ repeated steps on one plan
