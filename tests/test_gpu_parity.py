@@ -38,7 +38,8 @@ def test_parity_small_and_medium_workloads(grawa, name, variant):
     cfg = gen.CONFIGS[name]
     p, g = inputs(name)
     res = gpu_step(grawa, variant, p, g, cfg.pull, cfg.offsets())
-    compare_with_oracle(res, variant, p, g, cfg.pull, cfg.offsets())
+    stats = compare_with_oracle(res, variant, p, g, cfg.pull, cfg.offsets())
+    print(name, variant, stats)
     assert grawa.grawa_last_step_status() == 0
 
 
