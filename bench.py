@@ -372,7 +372,7 @@ STORED_CAPTURES = {
 }
 DEFAULT_KNOBS = {"sumsq_tile": 8192, "pull_tile": 0, "pull_variant": 0, "bulk_tile": 0, "sumsq_ctas_per_sm": 0,
                  "pull_prefetch_waves": 3, "sumsq_prefetch_waves": 1,
-                 "pull_ctas_per_sm": 0, "dependent_launch": 1, "pull_preload": 1}
+                 "pull_ctas_per_sm": 0, "dependent_launch": 1, "pull_preload": 1, "pull_wide": 1}
 
 
 def code_only(text):

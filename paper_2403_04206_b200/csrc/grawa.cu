@@ -33,6 +33,7 @@ static int64_t g_bulk_tile = 0;           // 0 = chosen from M so that at least 
 static int64_t g_kernel_timing = 0;
 static int64_t g_pdl = 1;
 static int64_t g_pull_preload = 1;
+static int64_t g_pull_wide = 1;             // fp32 register kernel: 32-byte accesses when every base is 32-byte aligned
 static int64_t g_pull16_staged = 1;         // 16-bit storage, 5..16 workers: shared-memory staged kernel (1) or register kernel (0)
 static int64_t g_pull_prefetch_waves = 3;
 static int64_t g_sumsq_prefetch_waves = 1;
@@ -339,15 +340,15 @@ struct CenterPullBulkDispatch<1> {
 };
 
 template <int M>
-static cudaError_t launch_center_pull(bool per_layer, int grid, int item_begin, int item_end, cudaStream_t stream, bool pdl,
+static cudaError_t launch_center_pull(bool per_layer, bool wide, int grid, int item_begin, int item_end, cudaStream_t stream, bool pdl,
                                       const MutPtrs& x, float* center, const float* beta, const Segment* segs, long long n, int tile,
                                       float pull, int preload, int prefetch_stride, int prefetch_waves)
 {
-    if (per_layer)
-        return launch_kernel(center_pull_kernel<M, true>, grid, kThreads, stream, pdl, x, center, beta, segs, item_begin, item_end, n,
-                             tile, pull, 1, preload, prefetch_stride, prefetch_waves);
-    return launch_kernel(center_pull_kernel<M, false>, grid, kThreads, stream, pdl, x, center, beta, segs, item_begin, item_end, n, tile,
-                         pull, 1, preload, prefetch_stride, prefetch_waves);
+    // `wide`: every base is 32-byte aligned, so the columns are moved by 32-byte loads and stores
+    auto kernel = wide ? (per_layer ? center_pull_kernel<M, true, 8> : center_pull_kernel<M, false, 8>)
+                       : (per_layer ? center_pull_kernel<M, true, 4> : center_pull_kernel<M, false, 4>);
+    return launch_kernel(kernel, grid, wide ? pull_threads(M, 8) : pull_threads(M, 4), stream, pdl, x, center, beta, segs, item_begin,
+                         item_end, n, tile, pull, 1, preload, prefetch_stride, prefetch_waves);
 }
 
 template <int M>
@@ -457,6 +458,7 @@ struct StepContext {
     MutPtrs xp{};
     float* center = nullptr;
     bool vec_g = true, vec_x = true, pdl = false;
+    bool wide_x = true;            // parameters and centre are 32-byte aligned as well
     StepScratch sc{};
     int* status = nullptr;
     unsigned* counter = nullptr;
@@ -495,10 +497,12 @@ static grawa_status make_context(int variant, float* const* params, const float*
     g_last_status[{plan->device, stream}] = ctx->status;
     ctx->vec_g = true;
     ctx->vec_x = center_out == nullptr || aligned16(center_out);
+    ctx->wide_x = (reinterpret_cast<uintptr_t>(center_out) & 31u) == 0;
     for (int m = 0; m < M; ++m) {
         ctx->gp.p[m] = grads ? grads[m] : nullptr; ctx->xp.p[m] = params[m];
         ctx->vec_g = ctx->vec_g && grads && aligned16(grads[m]);
         ctx->vec_x = ctx->vec_x && aligned16(params[m]);
+        ctx->wide_x = ctx->wide_x && (reinterpret_cast<uintptr_t>(params[m]) & 31u) == 0;
     }
     StepScratch& sc = ctx->sc;
     sc.segs = plan->d_segs1;
@@ -648,7 +652,7 @@ static grawa_status enqueue_center_pull(StepContext& c, int item_begin, int item
         const int waves = (grid <= 64 * stride) ? static_cast<int>(g_pull_prefetch_waves) : 0;
         const int grid2 = g_pull_ctas_per_sm > 0
                               ? static_cast<int>(std::min<int64_t>(grid, g_pull_ctas_per_sm * plan->sm_count)) : grid;
-        GRAWA_CUDA_TRY(CenterPullDispatch<kMaxRegWorkers>::run(M, per_layer, grid2, item_begin, item_end, c.stream, c.pdl, c.xp,
+        GRAWA_CUDA_TRY(CenterPullDispatch<kMaxRegWorkers>::run(M, per_layer, c.wide_x && g_pull_wide, grid2, item_begin, item_end, c.stream, c.pdl, c.xp,
                                                                c.center, beta, plan->d_segs2, c.n, tile, c.pull,
                                                                (c.preload && g_pull_preload) ? 1 : 0, stride, waves));
     } else {
@@ -1134,13 +1138,18 @@ grawa_status grawa_prox_step_typed(grawa_dtype dtype, void* const* params, const
                                static_cast<const float*>(center), &off, elem_size(dtype));
     if (st != GRAWA_OK || n == 0) return st;
     MutPtrs xp{};
-    bool vec = aligned16(center);
-    for (int m = 0; m < M; ++m) { xp.p[m] = static_cast<float*>(params[m]); vec = vec && aligned16(params[m]); }
+    bool vec = aligned16(center), wide = (reinterpret_cast<uintptr_t>(center) & 31u) == 0;
+    for (int m = 0; m < M; ++m) {
+        xp.p[m] = static_cast<float*>(params[m]);
+        vec = vec && aligned16(params[m]);
+        wide = wide && (reinterpret_cast<uintptr_t>(params[m]) & 31u) == 0;
+    }
     int64_t tile;
     {
         std::lock_guard<std::mutex> lock(g_mutex);
-        // one vector column per thread (measured best): 1024 fp32 or 2048 16-bit elements per CTA
-        tile = g_pull_tile > 0 ? g_pull_tile : (dtype == GRAWA_F32 ? 1024 : 2048);
+        wide = wide && g_pull_wide && dtype == GRAWA_F32;     // (on 16-bit storage 32-byte columns measured no gain)
+        // one vector column per thread (measured best): 16 bytes, or for fp32 32 bytes when every base is 32-byte aligned
+        tile = g_pull_tile > 0 ? g_pull_tile : (wide ? 32 : 16) * kThreads / static_cast<int64_t>(elem_size(dtype));
     }
     const int64_t tiles = (n + tile - 1) / tile;
     if (tiles > 0x7fffffffll) return GRAWA_ERR_INVALID_ARG;
@@ -1150,7 +1159,7 @@ grawa_status grawa_prox_step_typed(grawa_dtype dtype, void* const* params, const
     else if (dtype == GRAWA_F16)
         prox16_kernel<__half><<<grid, kThreads, 0, stream>>>(xp, static_cast<const __half*>(center), n, t, mu_over_tau, M, v);
     else
-        prox_kernel<<<grid, kThreads, 0, stream>>>(xp, static_cast<const float*>(center), n, t, mu_over_tau, M, v);
+        (wide ? prox_kernel<8> : prox_kernel<4>)<<<grid, kThreads, 0, stream>>>(xp, static_cast<const float*>(center), n, t, mu_over_tau, M, v);
     ++g_launches;
     GRAWA_CUDA_TRY(cudaGetLastError());
     return GRAWA_OK;
@@ -1308,6 +1317,11 @@ grawa_status grawa_set_option(const char* name, int64_t value)
         g_pull_preload = value;
         return GRAWA_OK;
     }
+    if (std::strcmp(name, "pull_wide") == 0) {
+        if (value < 0 || value > 1) return GRAWA_ERR_INVALID_ARG;
+        g_pull_wide = value;
+        return GRAWA_OK;
+    }
     if (std::strcmp(name, "pull16_staged") == 0) {
         if (value < 0 || value > 1) return GRAWA_ERR_INVALID_ARG;
         if (value != g_pull16_staged) { g_pull16_staged = value; clear_plans_locked(); }
@@ -1332,6 +1346,7 @@ int64_t grawa_get_option(const char* name)
     if (std::strcmp(name, "kernel_timing") == 0) return g_kernel_timing;
     if (std::strcmp(name, "dependent_launch") == 0) return g_pdl;
     if (std::strcmp(name, "pull_preload") == 0) return g_pull_preload;
+    if (std::strcmp(name, "pull_wide") == 0) return g_pull_wide;
     if (std::strcmp(name, "pull16_staged") == 0) return g_pull16_staged;
     if (std::strcmp(name, "pull_prefetch_waves") == 0) return g_pull_prefetch_waves;
     if (std::strcmp(name, "sumsq_prefetch_waves") == 0) return g_sumsq_prefetch_waves;

@@ -660,14 +660,51 @@ __device__ __forceinline__ void pull_scalar(const MutPtrs& x, float* center, con
 // workers in flight (COLS * M vector loads) and a CTA covers kThreads * COLS * VEC elements per
 // pass.  Measured alternatives: 8-byte columns with more CTAs per SM lose badly at M = 16 and
 // change nothing for M <= 8 (the kernel sits at the mixed read/write rate of the memory system).
-__host__ __device__ constexpr int pull_cols(int M) { return (M <= 2) ? 8 : (M <= 4) ? 4 : (M <= 8) ? 2 : 1; }
-__host__ __device__ constexpr int pull_vec(int) { return 4; }
-__host__ __device__ constexpr int pull_pass_elems(int M) { return kThreads * pull_cols(M) * pull_vec(M); }
+//
+// VEC = 8 (32-byte loads and stores, `ld/st.global.v8.f32`) keeps the same bytes per thread in half
+// as many columns and needs 32-byte aligned bases; an arithmetic-free copy of this access shape runs
+// 1.2-1.4 % faster with 32-byte than with 16-byte accesses at M = 4, 8 and 16.  Above 8 workers
+// a 32-byte column of all workers takes about 210 registers, so those CTAs have 128 threads (two per
+// SM, the same bytes in flight).  A pass covers the same number of elements for either width.
+__host__ __device__ constexpr int pull_cols(int M, int VEC = 4)
+{
+    return VEC == 8 ? ((M <= 2) ? 4 : (M <= 4) ? 2 : 1) : ((M <= 2) ? 8 : (M <= 4) ? 4 : (M <= 8) ? 2 : 1);
+}
+__host__ __device__ constexpr int pull_threads(int M, int VEC = 4) { return (VEC == 8 && M > 8) ? kThreads / 2 : kThreads; }
+__host__ __device__ constexpr int pull_pass_elems(int M) { return kThreads * pull_cols(M) * 4; }
+static_assert(pull_threads(16, 8) * pull_cols(16, 8) * 8 == pull_pass_elems(16) && pull_threads(8, 8) * pull_cols(8, 8) * 8 == pull_pass_elems(8) &&
+              pull_threads(4, 8) * pull_cols(4, 8) * 8 == pull_pass_elems(4) && pull_threads(2, 8) * pull_cols(2, 8) * 8 == pull_pass_elems(2),
+              "a pass covers the same elements for both access widths");
+
+// [b, e) split into scalar head, body aligned to VEC elements, scalar tail (everything head without vec_ok).
+template <int VEC>
+__device__ __forceinline__ void split_range_vec(long long b, long long e, int vec_ok, long long& hb, long long& te)
+{
+    if (vec_ok) {
+        hb = min((b + (VEC - 1)) & ~static_cast<long long>(VEC - 1), e);
+        te = max(e & ~static_cast<long long>(VEC - 1), hb);
+    } else {
+        hb = e;
+        te = e;
+    }
+}
 
 template <int VEC> struct VecIO;
 template <> struct VecIO<4> {
     static __device__ __forceinline__ void ld(const float* p, float (&o)[4]) { const float4 t = __ldcs(reinterpret_cast<const float4*>(p)); o[0] = t.x; o[1] = t.y; o[2] = t.z; o[3] = t.w; }
     static __device__ __forceinline__ void st(float* p, const float (&o)[4]) { __stcs(reinterpret_cast<float4*>(p), make_float4(o[0], o[1], o[2], o[3])); }
+};
+template <> struct VecIO<8> {
+    static __device__ __forceinline__ void ld(const float* p, float (&o)[8])
+    {
+        asm volatile("ld.global.cs.v8.f32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=f"(o[0]), "=f"(o[1]), "=f"(o[2]), "=f"(o[3]), "=f"(o[4]), "=f"(o[5]), "=f"(o[6]), "=f"(o[7]) : "l"(p) : "memory");
+    }
+    static __device__ __forceinline__ void st(float* p, const float (&o)[8])
+    {
+        asm volatile("st.global.cs.v8.f32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                     :: "l"(p), "f"(o[0]), "f"(o[1]), "f"(o[2]), "f"(o[3]), "f"(o[4]), "f"(o[5]), "f"(o[6]), "f"(o[7]) : "memory");
+    }
 };
 template <> struct VecIO<2> {
     static __device__ __forceinline__ void ld(const float* p, float (&o)[2]) { const float2 t = __ldcs(reinterpret_cast<const float2*>(p)); o[0] = t.x; o[1] = t.y; }
@@ -686,14 +723,14 @@ template <> struct VecIO<2> {
 // 2 * `prefetch_stride`, ... further on to be brought into L2: while the weights are being finalised
 // DRAM has nothing else to do, and the CTAs that take those items later find them in L2.  A
 // prefetch is a hint without architectural effect, and L2 is the GPU's point of coherence.
-template <int M, bool PER_LAYER>
-__global__ void __launch_bounds__(kThreads, 2)
+template <int M, bool PER_LAYER, int VEC>
+__global__ void __launch_bounds__(pull_threads(M, VEC), 2)
 center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restrict__ beta,
                    const Segment* __restrict__ segs, int item_begin, int item_end, long long n, int tile, float lambda,
                    int vec_ok, int preload, int prefetch_stride, int prefetch_waves)
 {
-    constexpr int COLS = pull_cols(M);
-    constexpr int VEC = pull_vec(M);
+    constexpr int COLS = pull_cols(M, VEC);
+    constexpr int THREADS = pull_threads(M, VEC);
     const int tid = threadIdx.x;
     int item = item_begin + blockIdx.x;
     // the work list belongs to the plan, not to the kernel before this one: fetch the first item early
@@ -709,14 +746,14 @@ center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restric
             b = static_cast<long long>(it) * tile;
             e = min(n, b + tile);
         }
-        split_range(b, e, vec_ok, hb, te);
-        ncol = static_cast<int>((te - hb) / VEC);               // te - hb is a multiple of 4
+        split_range_vec<VEC>(b, e, vec_ok, hb, te);
+        ncol = static_cast<int>((te - hb) / VEC);               // te - hb is a multiple of VEC
     };
     float v[COLS][M][VEC];
     auto load_chunk = [&](int c0) {
 #pragma unroll
         for (int q = 0; q < COLS; ++q) {
-            const int c = c0 + q * kThreads + tid;
+            const int c = c0 + q * THREADS + tid;
             if (c < ncol && in_bounds(hb + static_cast<long long>(c) * VEC, VEC, b, e, n)) {
 #pragma unroll
                 for (int m = 0; m < M; ++m) VecIO<VEC>::ld(x.p[m] + hb + static_cast<long long>(c) * VEC, v[q][m]);
@@ -741,7 +778,7 @@ center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restric
                         pb = it * tile;
                         pe = min(n, pb + tile);
                     }
-                    split_range(pb, pe, vec_ok, phb, pte);
+                    split_range_vec<VEC>(pb, pe, vec_ok, phb, pte);
                     const unsigned bytes = static_cast<unsigned>(pte - phb) * 4u;       // a multiple of 16
                     const float* base = x.p[0];
 #pragma unroll
@@ -769,12 +806,12 @@ center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restric
 #pragma unroll
             for (int m = 0; m < M; ++m) w[m] = bt[m];
         }
-        for (int c0 = 0; c0 < ncol; c0 += kThreads * COLS) {
+        for (int c0 = 0; c0 < ncol; c0 += THREADS * COLS) {
             if (!loaded) load_chunk(c0);
             loaded = false;
 #pragma unroll
             for (int q = 0; q < COLS; ++q) {
-                const int c = c0 + q * kThreads + tid;
+                const int c = c0 + q * THREADS + tid;
                 if (c < ncol && in_bounds(hb + static_cast<long long>(c) * VEC, VEC, b, e, n)) {
                     float cc[VEC];
 #pragma unroll
@@ -796,9 +833,9 @@ center_pull_kernel(MutPtrs x, float* __restrict__ center, const float* __restric
             }
         }
         loaded = false;                                  // an item without a vector body used nothing
-        for (long long i = b + tid; i < hb; i += kThreads)
+        for (long long i = b + tid; i < hb; i += THREADS)
             if (in_bounds(i, 1, b, e, n)) pull_scalar<M>(x, center, w, lambda, oml, i);
-        for (long long i = te + tid; i < e; i += kThreads)
+        for (long long i = te + tid; i < e; i += THREADS)
             if (in_bounds(i, 1, b, e, n)) pull_scalar<M>(x, center, w, lambda, oml, i);
         item += gridDim.x;
         if (item < item_end) locate(item);
@@ -868,7 +905,9 @@ copy_kernel(const float* __restrict__ src, float* __restrict__ dst, long long n,
 }
 
 // Proximity step (the "Prox." update of Algorithms 1-2): x_m <- fmaf(a, x_C, (1-a) x_m), a = mu/tau.
-// One CTA per flat tile; the centre column is loaded once and reused for all M workers.
+// One CTA per flat tile; the centre column is loaded once and reused for all M workers.  VEC = 4
+// (16-byte columns) or 8 (32-byte columns, bases 32-byte aligned).
+template <int VEC>
 __global__ void __launch_bounds__(kThreads)
 prox_kernel(MutPtrs x, const float* __restrict__ center, long long n, int tile, float a, int M, int vec_ok)
 {
@@ -877,30 +916,31 @@ prox_kernel(MutPtrs x, const float* __restrict__ center, long long n, int tile, 
     const long long e = min(n, b + tile);
     const float oma = 1.0f - a;
     long long hb, te;
-    split_range(b, e, vec_ok, hb, te);
-    const int ncol = static_cast<int>((te - hb) >> 2);
+    split_range_vec<VEC>(b, e, vec_ok, hb, te);
+    const int ncol = static_cast<int>((te - hb) / VEC);
     for (int c = threadIdx.x; c < ncol; c += kThreads) {
-        if (!in_bounds(hb + 4LL * c, 4, b, e, n)) continue;
-        const float4 cc = ld_stream4(reinterpret_cast<const float4*>(center + hb) + c);
+        const long long j = hb + static_cast<long long>(VEC) * c;
+        if (!in_bounds(j, VEC, b, e, n)) continue;
+        float cc[VEC];
+        VecIO<VEC>::ld(center + j, cc);
         int m = 0;
         for (; m + 4 <= M; m += 4) {
-            float4 v[4];
+            float v[4][VEC];
 #pragma unroll
-            for (int q = 0; q < 4; ++q) v[q] = ld_stream4(reinterpret_cast<const float4*>(x.p[m + q] + hb) + c);
+            for (int q = 0; q < 4; ++q) VecIO<VEC>::ld(x.p[m + q] + j, v[q]);
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
-                float4 o;
-                o.x = fmaf(a, cc.x, oma * v[q].x); o.y = fmaf(a, cc.y, oma * v[q].y);
-                o.z = fmaf(a, cc.z, oma * v[q].z); o.w = fmaf(a, cc.w, oma * v[q].w);
-                st_stream4(reinterpret_cast<float4*>(x.p[m + q] + hb) + c, o);
+#pragma unroll
+                for (int t = 0; t < VEC; ++t) v[q][t] = fmaf(a, cc[t], oma * v[q][t]);
+                VecIO<VEC>::st(x.p[m + q] + j, v[q]);
             }
         }
         for (; m < M; ++m) {
-            const float4 v = ld_stream4(reinterpret_cast<const float4*>(x.p[m] + hb) + c);
-            float4 o;
-            o.x = fmaf(a, cc.x, oma * v.x); o.y = fmaf(a, cc.y, oma * v.y);
-            o.z = fmaf(a, cc.z, oma * v.z); o.w = fmaf(a, cc.w, oma * v.w);
-            st_stream4(reinterpret_cast<float4*>(x.p[m] + hb) + c, o);
+            float v[VEC];
+            VecIO<VEC>::ld(x.p[m] + j, v);
+#pragma unroll
+            for (int t = 0; t < VEC; ++t) v[t] = fmaf(a, cc[t], oma * v[t]);
+            VecIO<VEC>::st(x.p[m] + j, v);
         }
     }
     for (int pass = 0; pass < 2; ++pass) {

@@ -620,6 +620,41 @@ def test_parity_with_thousands_of_tiny_layers(grawa, M, variant):
     assert bool((again["center"] == res["center"]).all())
 
 
+@pytest.mark.parametrize("M", [2, 3, 4, 7, 8, 9, 13, 16])
+def test_32_byte_and_16_byte_accesses_agree_bit_for_bit(grawa, M):
+    """Bases aligned to 32 bytes take 32-byte loads and stores, bases aligned to 16 bytes only (here
+    every vector starts 16 bytes into its allocation) the 16-byte ones: same arithmetic, same bytes out,
+    for the averaging step and for the proximity step; both against the oracle."""
+    import torch
+    cfg = gen.custom_config([7, 5001, 0, 3, 12001, 777, 8, 9, 8192, 8193, 40000], M, seed=700 + M, log10_sigma=(-2.0, 0.0))
+    p, g = gen.make_inputs(cfg)
+    off = cfg.offsets()
+
+    def shifted(arrs):
+        out = []
+        for a in arrs:
+            t = torch.zeros(a.size + 4, device="cuda")[4:]
+            assert t.data_ptr() % 32 == 16
+            t.copy_(torch.from_numpy(a))
+            out.append(t)
+        return out
+    for variant in ("lgrawa", "mgrawa"):
+        wide = gpu_step(grawa, variant, p, g, 0.3, off)
+        compare_with_oracle(wide, variant, p, g, 0.3, off)
+        narrow = gpu_step(grawa, variant, p, g, 0.3, off, params_dev=shifted(p), grads_dev=shifted(g))
+        compare_with_oracle(narrow, variant, p, g, 0.3, off)
+        assert bool((wide["center"] == narrow["center"]).all())
+        for u, v in zip(wide["workers"], narrow["workers"]):
+            assert bool((u == v).all())
+    xa, xb = to_device(p), shifted(p)
+    ca, cb = to_device([g[0]])[0], shifted([g[0]])[0]
+    grawa.grawa_prox_step(xa, ca, 0.05 / 16)
+    grawa.grawa_prox_step(xb, cb, 0.05 / 16)
+    torch.cuda.synchronize()
+    for u, v in zip(xa, xb):
+        assert bool((u == v).all())
+
+
 # ------------------------------------------------------------------ repeated steps on one plan
 
 @pytest.mark.parametrize("variant", ["mgrawa", "lgrawa", "grawa"])
