@@ -359,12 +359,12 @@ def whole_job_steps_per_s(world, ms_per_step_max):
 # knob at its default; anything else reports null.
 CAPTURE_ELEMENTS = 14918400
 STORED_CAPTURES = {
-    "center_pull": {"M": 16, "dram_bytes": 955075584 + 958193664, "dram_bytes_full": (86567656, 5542392064 + 5844806656), "begin": "// Steps 4-5, register variant",
+    "center_pull": {"M": 16, "dram_bytes": 955067392 + 953410560, "dram_bytes_full": (86567656, 5541940224 + 5825000448), "begin": "// Steps 4-5, register variant",
                     "end": "// Steps 4-5 for any M up to",
                     "host_begin": "static grawa_status enqueue_center_pull(StepContext", "host_end": "// Given scores of a step",
-                    "kernel_sha256": "9aa1cd15bd94e316e2a45778645f33881e36eaed5ee35a7f1b272d01f6475272",
-                    "host_sha256": "08f9e8f045b5e0f30219e9a3fc2c79ab3bfb91d23a7c329b7e8c6c8cef465dae"},
-    "sumsq": {"M": 16, "dram_bytes": 954870016 + 5120512, "dram_bytes_full": (86567656, 5540708608 + 3944448), "begin": "// Step 1 (Eq. 3 / Eq. 5):",
+                    "kernel_sha256": "444a286cacebaa8d7c93389e88c2d8b630a66fc7505a9c644cc49f3a9e74fd66",
+                    "host_sha256": "81b9d1b33c91036008ffb4b6a8cd8b72799b0b9f18d617d2a2a48f7b9d052c65"},
+    "sumsq": {"M": 16, "dram_bytes": 954848768 + 3460864, "dram_bytes_full": (86567656, 5540634624 + 3330048), "begin": "// Step 1 (Eq. 3 / Eq. 5):",
               "end": "// Steps 4-5, register variant",
               "host_begin": "static grawa_status enqueue_weights_launches(StepContext& c)\n", "host_end": "// Steps 4-5 on 16-bit storage",
               "kernel_sha256": "6c8fcdcd2927db90fe40fdbb204bf18a7a4757f76906c7670ab4625309856fa1",
