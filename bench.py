@@ -732,10 +732,11 @@ def run_reference(args):
     base, sec = oracle_timing(cfg, variant, p, g, budget_s=150.0, steps_wanted=max(1, args.steps), warmup=max(0, args.warmup))
     value = 1.0 / sec
     base = {k: base[k] for k in ("value", "unit", "cores", "kind", "sample", "whole_steps")}
-    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": 1,
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "steps/s", "n_gpus": world,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": sec * 1e3, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-            "config": describe(cfg, variant, "step", "f32", 1),
+            "config": describe(cfg, variant, "step", "f32", world),      # rank 0 alone runs the oracle, one problem
             "cpu_baseline": base,
             "e2e": {"value": value, "unit": "steps/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
     print(json.dumps(line), flush=True)
