@@ -655,6 +655,54 @@ def test_32_byte_and_16_byte_accesses_agree_bit_for_bit(grawa, M):
         assert bool((u == v).all())
 
 
+def test_two_host_threads_on_their_own_streams_and_buffers(grawa):
+    """Calls with different streams and disjoint buffers may run concurrently: two host threads, each
+    with its own stream, problem shape and variant, forty steps each from fresh parameters; every
+    result equals the one the same call gives alone, bit for bit."""
+    import threading
+    import torch
+    jobs = [("lgrawa", gen.custom_config([7, 50001, 0, 3, 120001, 777], 5, seed=801, log10_sigma=(-2.0, 0.0))),
+            ("mgrawa", gen.custom_config([4096, 64, 65536, 300001], 8, seed=802, log10_sigma=(-2.0, 0.0)))]
+    data, alone = [], []
+    for variant, cfg in jobs:
+        p, g = gen.make_inputs(cfg)
+        data.append((p, g))
+        res = gpu_step(grawa, variant, p, g, 0.4, cfg.offsets())
+        compare_with_oracle(res, variant, p, g, 0.4, cfg.offsets())
+        alone.append(res)
+    out, errors = [None, None], []
+
+    def run(i):
+        try:
+            variant, cfg = jobs[i]
+            stream = torch.cuda.Stream()
+            with torch.cuda.stream(stream):
+                x0, g = to_device(data[i][0]), to_device(data[i][1])
+                x = [t.clone() for t in x0]
+                center = torch.empty(cfg.n, device="cuda")
+                step = grawa.grawa_lgrawa_step if variant == "lgrawa" else grawa.grawa_mgrawa_step
+                for _ in range(40):
+                    for t, t0 in zip(x, x0):
+                        t.copy_(t0)
+                    step(x, g, 0.4, cfg.offsets(), center, stream=stream)
+                stream.synchronize()
+                assert grawa.grawa_last_step_status(stream) == 0
+            out[i] = (x, center)
+        except Exception as exc:                                  # surfaced in the main thread
+            errors.append(exc)
+    threads = [threading.Thread(target=run, args=(i,)) for i in range(2)]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join()
+    assert not errors, errors
+    for i in range(2):
+        x, center = out[i]
+        assert bool((center == alone[i]["center"]).all())
+        for u, v in zip(x, alone[i]["workers"]):
+            assert bool((u == v).all())
+
+
 # ------------------------------------------------------------------ repeated steps on one plan
 
 @pytest.mark.parametrize("variant", ["mgrawa", "lgrawa", "grawa"])
