@@ -22,6 +22,13 @@ template <> struct Pair16<__nv_bfloat16> {
         const __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
         return *reinterpret_cast<const unsigned*>(&v);
     }
+    // lo += w.lo^2, hi += w.hi^2: fused multiply-add with 16-bit sources and an fp32 accumulator (the
+    // sources are widened exactly, one rounding: the value of fmaf on the unpacked elements)
+    static __device__ __forceinline__ void square_add(unsigned w, float& lo, float& hi)
+    {
+        asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\tfma.rn.f32.bf16 %0, l, l, %0;\n\tfma.rn.f32.bf16 %1, h, h, %1;\n\t}"
+            : "+f"(lo), "+f"(hi) : "r"(w));
+    }
     static __device__ __forceinline__ float load1(const __nv_bfloat16* p) { return __bfloat162float(*p); }
     static __device__ __forceinline__ void store1(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
 };
@@ -36,6 +43,11 @@ template <> struct Pair16<__half> {
     {
         const __half2 v = __floats2half2_rn(lo, hi);
         return *reinterpret_cast<const unsigned*>(&v);
+    }
+    static __device__ __forceinline__ void square_add(unsigned w, float& lo, float& hi)
+    {
+        asm("{\n\t.reg .b16 l, h;\n\tmov.b32 {l, h}, %2;\n\tfma.rn.f32.f16 %0, l, l, %0;\n\tfma.rn.f32.f16 %1, h, h, %1;\n\t}"
+            : "+f"(lo), "+f"(hi) : "r"(w));
     }
     static __device__ __forceinline__ float load1(const __half* p) { return __half2float(*p); }
     static __device__ __forceinline__ void store1(__half* p, float v) { *p = __float2half_rn(v); }
@@ -129,10 +141,10 @@ sumsq16_kernel(const __grid_constant__ ConstPtrs grads, StepScratch sc, int item
             for (int t = 0; t < 8; ++t) a[t] = 0.f;
 #pragma unroll
             for (int u = 0; u < UNROLL; ++u) {
-                float v[8];
-                unpack8<T>(raw[u], v);
-#pragma unroll
-                for (int t = 0; t < 8; ++t) a[t] = fmaf(v[t], v[t], a[t]);
+                Pair16<T>::square_add(raw[u].x, a[0], a[1]);
+                Pair16<T>::square_add(raw[u].y, a[2], a[3]);
+                Pair16<T>::square_add(raw[u].z, a[4], a[5]);
+                Pair16<T>::square_add(raw[u].w, a[6], a[7]);
             }
             dacc += ((static_cast<double>(a[0]) + static_cast<double>(a[1])) + (static_cast<double>(a[2]) + static_cast<double>(a[3]))) +
                     ((static_cast<double>(a[4]) + static_cast<double>(a[5])) + (static_cast<double>(a[6]) + static_cast<double>(a[7])));
