@@ -137,7 +137,9 @@ typedef enum grawa_dtype { GRAWA_F32 = 0, GRAWA_BF16 = 1, GRAWA_F16 = 2 } grawa_
  * centre, and each result is rounded to nearest-even once, on its store (pull = 1 still makes
  * every worker bit-equal to center_out, pull = 0 leaves them untouched).
  * params, grads: HOST arrays of M DEVICE pointers to n elements of `dtype`, aligned to the element
- * size (16-byte aligned bases take the vector kernels); center_out: DEVICE, n elements, or NULL.
+ * size (16-byte aligned bases take the vector kernels; fp32 bases aligned to 32 bytes, as every
+ * allocator's are, the 32-byte accesses of the centre+pull and proximity kernels); center_out: DEVICE,
+ * n elements, or NULL.
  * GRAWA_F32 is exactly the three step entry points above. */
 grawa_status grawa_step_typed(grawa_dtype dtype, grawa_variant variant, void *const *params,
                               const void *const *grads, int64_t n, int M, float pull,
