@@ -342,8 +342,9 @@ int grawa_trace_read(uint64_t *rows_out, int max_rows);
  *                  that are resident when a kernel starts hint the data of the items that many
  *                  grid-fuls further on into L2 while they wait for the kernel in front; 0 = off.
  *   "pull_wide"     1 (default) = when every parameter vector and the centre are 32-byte aligned, the fp32
- *                  centre+pull kernel for up to 16 workers and the fp32 proximity step move their columns
- *                  by 32-byte loads and stores; 0 = 16-byte accesses always.  Same results bit for bit.
+ *                  centre+pull kernel for up to 16 workers, the 16-bit one for up to 4 workers and the
+ *                  fp32 proximity step move their columns by 32-byte loads and stores; 0 = 16-byte
+ *                  accesses always.  Same results bit for bit.
  *   "pull16_staged" 1 (default) = on 16-bit storage with 5..16 workers the centre+pull kernel stages
  *                  its columns through shared memory (per-thread asynchronous 16-byte copies);
  *                  0 = the register kernel for every worker count.  Drops the cached plans.

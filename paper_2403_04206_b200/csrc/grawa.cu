@@ -371,15 +371,14 @@ struct CenterPullDispatch<1> {
 
 // 16-bit storage: register kernel for 2..16 aligned workers.
 template <typename T, int M>
-static cudaError_t launch_center_pull16(bool per_layer, int grid, int item_begin, int item_end, cudaStream_t stream, bool pdl,
+static cudaError_t launch_center_pull16(bool per_layer, bool wide, int grid, int item_begin, int item_end, cudaStream_t stream, bool pdl,
                                         const MutPtrs& x, T* center, const float* beta, const Segment* segs, long long n,
                                         int tile, float pull)
 {
-    if (per_layer)
-        return launch_kernel(center_pull16_kernel<T, M, true>, grid, kThreads, stream, pdl, x, center, beta, segs, item_begin,
-                             item_end, n, tile, pull, 1);
-    return launch_kernel(center_pull16_kernel<T, M, false>, grid, kThreads, stream, pdl, x, center, beta, segs, item_begin, item_end,
-                         n, tile, pull, 1);
+    constexpr bool kCanWide = M <= 4;               // 32-byte columns: up to 4 workers
+    auto kernel = (wide && kCanWide) ? (per_layer ? center_pull16_kernel<T, M, true, kCanWide> : center_pull16_kernel<T, M, false, kCanWide>)
+                                     : (per_layer ? center_pull16_kernel<T, M, true, false> : center_pull16_kernel<T, M, false, false>);
+    return launch_kernel(kernel, grid, kThreads, stream, pdl, x, center, beta, segs, item_begin, item_end, n, tile, pull, 1);
 }
 
 template <typename T, int M>
@@ -608,7 +607,7 @@ static grawa_status enqueue_center_pull16_t(StepContext& c, int item_begin, int 
         GRAWA_CUDA_TRY(launch_center_pull_staged_any<T>(per_layer, grid, item_begin, item_end, c.stream, c.pdl, c.xp, center, c.sc.beta,
                                                         plan->d_segs2, c.n, tile, c.pull, M, (c.preload && g_pull_preload) ? 1 : 0));
     } else if (c.vec_x && M <= kMaxRegWorkers) {
-        GRAWA_CUDA_TRY((CenterPull16Dispatch<T, kMaxRegWorkers>::run(M, per_layer, grid, item_begin, item_end, c.stream, c.pdl, c.xp,
+        GRAWA_CUDA_TRY((CenterPull16Dispatch<T, kMaxRegWorkers>::run(M, per_layer, c.wide_x && g_pull_wide, grid, item_begin, item_end, c.stream, c.pdl, c.xp,
                                                                      center, c.sc.beta, plan->d_segs2, c.n, tile, c.pull)));
     } else {
         GRAWA_CUDA_TRY(launch_kernel(center_pull16_generic_kernel<T>, grid, kThreads, c.stream, c.pdl, c.xp, center, c.sc.beta,

@@ -193,6 +193,18 @@ template <> struct Words<4> {
     }
     static __device__ __forceinline__ void st(void* p, const unsigned (&o)[4]) { __stcs(reinterpret_cast<uint4*>(p), make_uint4(o[0], o[1], o[2], o[3])); }
 };
+template <> struct Words<8> {                       // one 256-bit access; the address is 32-byte aligned
+    static __device__ __forceinline__ void ld(const void* p, unsigned (&o)[8])
+    {
+        asm volatile("ld.global.cs.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
+                     : "=r"(o[0]), "=r"(o[1]), "=r"(o[2]), "=r"(o[3]), "=r"(o[4]), "=r"(o[5]), "=r"(o[6]), "=r"(o[7]) : "l"(p) : "memory");
+    }
+    static __device__ __forceinline__ void st(void* p, const unsigned (&o)[8])
+    {
+        asm volatile("st.global.cs.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};"
+                     :: "l"(p), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+    }
+};
 template <> struct Words<2> {
     static __device__ __forceinline__ void ld(const void* p, unsigned (&o)[2])
     {
@@ -219,16 +231,18 @@ __device__ __forceinline__ void pull16_scalar(const MutPtrs& x, T* center, const
 
 // Steps 4-5 on 16-bit parameters: same arithmetic as center_pull_kernel (fp32 FMA chain over
 // m = 0..M-1, pull from the unrounded fp32 centre), one rounding on each store.
-template <typename T, int M, bool PER_LAYER>
+// WIDE (up to 4 workers, every base 32-byte aligned): 32-byte columns, half as many per thread.
+template <typename T, int M, bool PER_LAYER, bool WIDE>
 __global__ void __launch_bounds__(kThreads, 2)
 center_pull16_kernel(MutPtrs x, T* __restrict__ center, const float* __restrict__ beta, const Segment* __restrict__ segs,
                      int item_begin, int item_end, long long n, int tile, float lambda, int vec_ok)
 {
+    static_assert(!WIDE || M <= 4, "32-byte columns are for up to 4 workers");
     Segment first_sg = Segment{0, 0, 0};           // plan data: independent of the kernel before this one
     if (PER_LAYER && item_begin + static_cast<int>(blockIdx.x) < item_end) first_sg = segs[item_begin + blockIdx.x];
     grid_dependency_sync();
-    constexpr int COLS = pull16_cols(M);
-    constexpr int WORDS = pull16_words(M);
+    constexpr int COLS = WIDE ? pull16_cols(M) / 2 : pull16_cols(M);
+    constexpr int WORDS = WIDE ? 8 : pull16_words(M);
     constexpr int VEC = 2 * WORDS;                 // elements per column
     const float oml = 1.0f - lambda;
     const int tid = threadIdx.x;
@@ -250,9 +264,12 @@ center_pull16_kernel(MutPtrs x, T* __restrict__ center, const float* __restrict_
             b = static_cast<long long>(item) * tile;
             e = min(n, b + tile);
         }
-        long long hb, te;
-        split_range16(b, e, vec_ok, hb, te);
-        const int ncol = static_cast<int>((te - hb) / VEC);      // te - hb is a multiple of 8
+        long long hb = e, te = e;                                 // body aligned to a column (VEC is 4, 8 or 16 elements)
+        if (vec_ok) {
+            hb = min((b + (WIDE ? 15 : 7)) & ~static_cast<long long>(WIDE ? 15 : 7), e);
+            te = max(e & ~static_cast<long long>(WIDE ? 15 : 7), hb);
+        }
+        const int ncol = static_cast<int>((te - hb) / VEC);      // te - hb is a multiple of 8 (16 when WIDE)
         for (int c0 = 0; c0 < ncol; c0 += kThreads * COLS) {
             unsigned raw[COLS][M][WORDS];
 #pragma unroll
@@ -268,42 +285,45 @@ center_pull16_kernel(MutPtrs x, T* __restrict__ center, const float* __restrict_
             for (int q = 0; q < COLS; ++q) {
                 const int c = c0 + q * kThreads + tid;
                 if (c < ncol && in_bounds(hb + static_cast<long long>(c) * VEC, VEC, b, e, n)) {
-                    // centre of the column's elements (fp32 FMA chain over the workers)
-                    float cc[VEC];
+                    // the column in pieces of at most 8 elements: centre (fp32 FMA chain over the workers),
+                    // then the pulled workers packed back in place; stores of whole columns at the end
+                    constexpr int HW = WORDS < 4 ? WORDS : 4;      // words per piece
+                    unsigned oc[WORDS];
 #pragma unroll
-                    for (int k = 0; k < WORDS; ++k) {
-                        float lo, hi;
-                        Pair16<T>::unpack(raw[q][0][k], lo, hi);
-                        cc[2 * k] = w[0] * lo;
-                        cc[2 * k + 1] = w[0] * hi;
-                    }
+                    for (int h = 0; h < WORDS / HW; ++h) {
+                        float cc[2 * HW];
 #pragma unroll
-                    for (int m = 1; m < M; ++m) {
-#pragma unroll
-                        for (int k = 0; k < WORDS; ++k) {
+                        for (int k = 0; k < HW; ++k) {
                             float lo, hi;
-                            Pair16<T>::unpack(raw[q][m][k], lo, hi);
-                            cc[2 * k] = fmaf(w[m], lo, cc[2 * k]);
-                            cc[2 * k + 1] = fmaf(w[m], hi, cc[2 * k + 1]);
+                            Pair16<T>::unpack(raw[q][0][h * HW + k], lo, hi);
+                            cc[2 * k] = w[0] * lo;
+                            cc[2 * k + 1] = w[0] * hi;
+                        }
+#pragma unroll
+                        for (int m = 1; m < M; ++m) {
+#pragma unroll
+                            for (int k = 0; k < HW; ++k) {
+                                float lo, hi;
+                                Pair16<T>::unpack(raw[q][m][h * HW + k], lo, hi);
+                                cc[2 * k] = fmaf(w[m], lo, cc[2 * k]);
+                                cc[2 * k + 1] = fmaf(w[m], hi, cc[2 * k + 1]);
+                            }
+                        }
+#pragma unroll
+                        for (int k = 0; k < HW; ++k) oc[h * HW + k] = Pair16<T>::pack(cc[2 * k], cc[2 * k + 1]);
+#pragma unroll
+                        for (int m = 0; m < M; ++m) {
+#pragma unroll
+                            for (int k = 0; k < HW; ++k) {
+                                float lo, hi;
+                                Pair16<T>::unpack(raw[q][m][h * HW + k], lo, hi);
+                                raw[q][m][h * HW + k] = Pair16<T>::pack(fmaf(lambda, cc[2 * k], oml * lo), fmaf(lambda, cc[2 * k + 1], oml * hi));
+                            }
                         }
                     }
-                    if (center) {
-                        unsigned o[WORDS];
+                    if (center) Words<WORDS>::st(center + hb + static_cast<long long>(c) * VEC, oc);
 #pragma unroll
-                        for (int k = 0; k < WORDS; ++k) o[k] = Pair16<T>::pack(cc[2 * k], cc[2 * k + 1]);
-                        Words<WORDS>::st(center + hb + static_cast<long long>(c) * VEC, o);
-                    }
-#pragma unroll
-                    for (int m = 0; m < M; ++m) {
-                        unsigned o[WORDS];
-#pragma unroll
-                        for (int k = 0; k < WORDS; ++k) {
-                            float lo, hi;
-                            Pair16<T>::unpack(raw[q][m][k], lo, hi);
-                            o[k] = Pair16<T>::pack(fmaf(lambda, cc[2 * k], oml * lo), fmaf(lambda, cc[2 * k + 1], oml * hi));
-                        }
-                        Words<WORDS>::st(reinterpret_cast<T*>(x.p[m]) + hb + static_cast<long long>(c) * VEC, o);
-                    }
+                    for (int m = 0; m < M; ++m) Words<WORDS>::st(reinterpret_cast<T*>(x.p[m]) + hb + static_cast<long long>(c) * VEC, raw[q][m]);
                 }
             }
         }

@@ -229,3 +229,20 @@ def test_16bit_parity_on_seeded_random_tables(grawa, case):
     p, g = gen.make_inputs(cfg)
     res = run_typed(grawa, dtype_name, variant, p, g, pull, cfg.offsets(), offset_elems=(8 if case % 4 == 3 else 0))
     check(res, dtype_name, variant, pull, cfg.offsets())
+
+
+@pytest.mark.parametrize("dtype_name", ["bfloat16", "float16"])
+@pytest.mark.parametrize("M", [2, 3, 4])
+def test_16bit_32_byte_and_16_byte_columns_agree_bit_for_bit(grawa, M, dtype_name):
+    """Up to 4 workers: bases aligned to 32 bytes take 32-byte columns, bases 16 bytes into their
+    allocation the 16-byte ones; same arithmetic, same bytes out, both against the oracle."""
+    cfg = gen.custom_config([7, 5001, 0, 3, 12001, 777, 8, 9, 8192, 8193, 40000, 16, 17], M, seed=900 + M, log10_sigma=(-2.0, 0.0))
+    p, g = gen.make_inputs(cfg)
+    for variant in ("lgrawa", "mgrawa"):
+        wide = run_typed(grawa, dtype_name, variant, p, g, 0.3, cfg.offsets())
+        check(wide, dtype_name, variant, 0.3, cfg.offsets())
+        narrow = run_typed(grawa, dtype_name, variant, p, g, 0.3, cfg.offsets(), offset_elems=8)
+        check(narrow, dtype_name, variant, 0.3, cfg.offsets())
+        assert np.array_equal(wide["center"], narrow["center"])
+        for u, v in zip(wide["workers"], narrow["workers"]):
+            assert np.array_equal(u, v)
