@@ -246,3 +246,33 @@ def test_16bit_32_byte_and_16_byte_columns_agree_bit_for_bit(grawa, M, dtype_nam
         assert np.array_equal(wide["center"], narrow["center"])
         for u, v in zip(wide["workers"], narrow["workers"]):
             assert np.array_equal(u, v)
+
+
+@pytest.mark.parametrize("name", ["vgg16", "vit_b16"])
+def test_16bit_parity_large_workloads_full_size(grawa, name):
+    """bfloat16 LGRAWA on the two largest workloads at full size, element by element against the oracle
+    run on the fp32 images of the rounded inputs (comparison in chunks, as for fp32 storage)."""
+    import torch
+    from gpu_util import compare_with_oracle
+    cfg = gen.CONFIGS[name]
+    p, g = gen.make_inputs(cfg)
+    off = cfg.offsets()
+    x, gr = [], []
+    for m in range(cfg.M):                                      # round to storage; the oracle sees what the GPU sees
+        t = torch.from_numpy(p[m]).cuda().bfloat16()
+        p[m][:] = t.float().cpu().numpy()
+        x.append(t)
+        t = torch.from_numpy(g[m]).cuda().bfloat16()
+        g[m][:] = t.float().cpu().numpy()
+        gr.append(t)
+    K, M = cfg.K, cfg.M
+    beta = torch.empty(K * M, device="cuda")
+    scores = torch.empty(K * M, dtype=torch.float64, device="cuda")
+    sumsq = torch.empty(K * M, dtype=torch.float64, device="cuda")
+    center = torch.zeros(cfg.n, dtype=torch.bfloat16, device="cuda")
+    grawa.grawa_step_typed("lgrawa", x, gr, cfg.pull, off, center, weights_out=beta, scores_out=scores, sumsq_out=sumsq)
+    assert grawa.grawa_last_step_status() == 0
+    res = {"workers": x, "center": center, "beta": beta.cpu().numpy().reshape(K, M), "A": scores.cpu().numpy().reshape(K, M),
+           "S": sumsq.cpu().numpy().reshape(K, M)}
+    stats = compare_with_oracle(res, "lgrawa", p, g, cfg.pull, off, half_ulp=HALF_ULP["bfloat16"])
+    print(name, "bfloat16 lgrawa", stats)
