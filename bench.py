@@ -481,7 +481,7 @@ def run_cuda(args):
         sharded_out = run_sharded(grawa, cfg, variant, args, world, rank, peak, barrier, x, g, center)
 
     ms_max, e2e_ms_max = max_over_ranks([ms, e2e_ms if e2e_ms is not None else 0.0], world, "cuda")
-    ops = targets = small = many = None
+    ops = targets = small = many = trace = None
     if world == 1 and not args.headline_only:
         ops = side_ops(grawa, cfg, variant, x, g, center, args, peak)
     del call, x, g, center
@@ -491,6 +491,8 @@ def run_cuda(args):
         targets = target_runs(grawa, args, peak, have=(cfg, hp, hg))
         many = many_worker_runs(grawa, args, peak)
         small = small_runs(grawa, args)
+        if args.trace_finalize:
+            trace = trace_breakdown("resnet18_imagenet")
     clocks = sampler.stop()
 
     if rank == 0:
@@ -539,6 +541,8 @@ def run_cuda(args):
             line["many_workers"] = many
         if small is not None:
             line["small"] = small
+        if trace is not None:
+            line["in_step_finalize"] = trace
         if sharded_out is not None:
             line["sharded"] = sharded_out
         if world == 1 and not args.no_cpu_baseline and op == "step":
@@ -632,6 +636,52 @@ def many_worker_runs(grawa, args, peak):
     del x, g, center
     torch.cuda.empty_cache()
     return out
+
+
+def trace_child(name):
+    """Runs in a child process with the trace build selected: eager back-to-back steps of one workload,
+    both variants; prints the medians of the device-side stamps as one JSON line."""
+    import torch
+    import paper_2403_04206_b200 as grawa
+    cfg = gen.CONFIGS[name]
+    x, g = device_inputs(cfg)
+    center = torch.empty(cfg.n, device="cuda")
+    out = {}
+    steps = 24
+    for variant in ("lgrawa", "mgrawa"):
+        fn = grawa.PreparedStep(variant, x, g, cfg.pull, cfg.offsets(), center)
+        for _ in range(5):
+            fn()
+        torch.cuda.synchronize()
+        if grawa.grawa_trace_read() is None:
+            print(json.dumps({"unavailable": "not the trace build"}))
+            return
+        for _ in range(steps):
+            fn()
+        torch.cuda.synchronize()
+        t = grawa.grawa_trace_read().astype(np.int64)[:steps]          # [step, kernel, stamp] in ns
+        med = lambda a: float(np.median(a[2:])) / 1e3
+        out[variant] = {"finalize_us": med(t[:, 1, 3] - t[:, 1, 1]),
+                        "sumsq_exit_to_finalize_start_us": med(t[:, 1, 1] - t[:, 0, 3]),
+                        "finalize_exit_to_center_pull_start_us": med(t[:, 2, 1] - t[:, 1, 3])}
+    print(json.dumps(out))
+
+
+def trace_breakdown(name):
+    """The finalisation kernel and the two hand-overs around it as they run inside a step (dependent
+    launch on), from `%globaltimer` stamps of the library's trace build in a child process.  The stamps
+    slow the sum-of-squares kernel down, so only these three short intervals are reported.  The kernel's
+    duration here is not what it adds to a step: while it runs, the centre+pull kernel's early loads and
+    L2 hints keep DRAM busy (that is their purpose), which lengthens this kernel's few memory round trips."""
+    import subprocess
+    env = dict(os.environ, GRAWA_TRACE="1")
+    try:
+        r = subprocess.run([sys.executable, os.path.abspath(__file__), "--trace-child", name], env=env, capture_output=True,
+                           text=True, timeout=300)
+        line = [l for l in r.stdout.splitlines() if l.startswith("{")][-1]
+        return dict(workload=name, source="trace build of the library, device-side stamps, medians of 22 eager steps", **json.loads(line))
+    except Exception as exc:                                     # a diagnostic: never fails the run
+        return {"workload": name, "unavailable": repr(exc)[:200]}
 
 
 def small_runs(grawa, args):
@@ -760,11 +810,17 @@ def main():
     ap.add_argument("--workers", type=int, default=0, help="override the workload's number of workers (2..64)")
     ap.add_argument("--layers-limit", type=int, default=0, help="use only the first L layers (small profiling captures)")
     ap.add_argument("--option", action="append", default=[], help="library tuning knob, name=value (repeatable)")
+    ap.add_argument("--trace-finalize", action="store_true",
+                    help="add device-side stamps of the finalisation kernel inside ResNet-18 steps (trace build, child process)")
+    ap.add_argument("--trace-child", default=None, help=argparse.SUPPRESS)
     ap.add_argument("--print-source-hashes", action="store_true",
                     help="print the hashes that tie a stored ncu capture to the kernel source, and exit")
     args = ap.parse_args()
     if args.print_source_hashes:
         print(json.dumps({k: source_hashes(k) for k in STORED_CAPTURES}))
+        return
+    if args.trace_child:
+        trace_child(args.trace_child)
         return
     args.warmup = max(args.warmup, 3) if args.impl == "cuda" else args.warmup
     if args.impl == "reference":
