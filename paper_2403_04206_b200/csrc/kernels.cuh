@@ -634,8 +634,8 @@ sumsq_kernel(const __grid_constant__ ConstPtrs grads, StepScratch sc, int items,
 }
 
 // ---------------------------------------------------------------------------------------------
-// Steps 4-5, register variant: one thread owns a 16-byte column of all M workers, so each
-// parameter is read once and M independent vector loads are in flight per column.
+// Steps 4-5, register variant: one thread owns a 16-byte (VEC = 4) or 32-byte (VEC = 8) column of
+// all M workers, so each parameter is read once and M independent vector loads are in flight per column.
 //   x_C = sum_m beta_m x_m   (fp32 FMA chain, m = 0..M-1)      x_m <- fmaf(pull, x_C, (1-pull) x_m)
 // PER_LAYER: the items are the Segments, weights of the segment's layer (Eq. 7); otherwise flat
 // tiles of `tile` elements and one weight per worker (Eq. 2 / Eq. 4).  The launch covers items
