@@ -2,6 +2,8 @@
 ("replicas only"), so what has to work across ranks is the timing reduction (max over ranks), the
 whole-job aggregate, and the reference arm's rule that only rank 0 works."""
 import json
+
+import numpy as np
 import os
 import subprocess
 import sys
@@ -93,3 +95,17 @@ def test_stored_ncu_traffic_is_quoted_only_for_the_captured_kernel_and_default_k
             assert abs(bench.stored_traffic(Knobs(), which, part) / (cap["dram_bytes"] / bench.CAPTURE_ELEMENTS * part.n) - 1) < 1e-12
         assert bench.stored_traffic(Knobs(), which, vgg) is None                      # another M
         assert bench.stored_traffic(Knobs(pull_variant=2), which, vit) is None       # a knob off its default
+
+
+def test_workers_override_keeps_the_layer_table_and_recipe():
+    import argparse
+    import bench
+    import gen
+    base = gen.CONFIGS["resnet18_imagenet"]
+    args = argparse.Namespace(workload="resnet18_imagenet", workers=32, layers_limit=0)
+    cfg = bench.workload_config(args)
+    assert cfg.M == 32 and cfg.n == base.n and cfg.K == base.K and np.array_equal(cfg.offsets(), base.offsets())
+    assert (cfg.seed, cfg.pull, cfg.grad_recipe, cfg.log10_sigma) == (base.seed, base.pull, base.grad_recipe, base.log10_sigma)
+    assert bench.op_bytes(cfg, "step") == (3 * 32 + 1) * 4 * base.n and bench.op_bytes(cfg, "step", "bf16") == (3 * 32 + 1) * 2 * base.n
+    small = bench.workload_config(argparse.Namespace(workload="vit_b16", workers=0, layers_limit=28))
+    assert small.K == 28 and small.M == gen.CONFIGS["vit_b16"].M and small.n == 14918400 == bench.CAPTURE_ELEMENTS
