@@ -2,12 +2,11 @@
 ("replicas only"), so what has to work across ranks is the timing reduction (max over ranks), the
 whole-job aggregate, and the reference arm's rule that only rank 0 works."""
 import json
-
-import numpy as np
 import os
 import subprocess
 import sys
 
+import numpy as np
 import pytest
 import torch
 import torch.distributed as dist
